@@ -1,0 +1,184 @@
+"""Plain decoder forward: the function the rollout policy pi_theta evaluates.
+
+The paper names the policy models only; the architecture is the one the benchmark
+configurations spell out: pre-norm decoder, RMSNorm (eps inside the root, gains g),
+grouped-query attention with rotate-half RoPE, SwiGLU feed-forward, no biases, untied
+embedding and output head.  For a token string t_0..t_{n-1}:
+
+    x_t   = E[t_t]
+    h     = rmsnorm(x, g1);  q, k, v = h Wq^T, h Wk^T, h Wv^T;  RoPE(q, k; position t)
+    s_tu  = q_t . k_u / sqrt(dh) for u <= t, query head i reads kv head i // (Hq/Hkv)
+    x    += softmax(s) v Wo^T
+    h     = rmsnorm(x, g2);  x += (silu(h Wg^T) * (h Wu^T)) Wd^T
+    logits_t = rmsnorm(x_t, gf) W_lm^T
+
+Three routines compute it: `forward_full` (dense recompute, the definition),
+`Incremental` (token-by-token with a growing K/V list) and `SharedPrefix` (one K/V of
+the cached prefix reused by all G samples of a sampling group, Eq. 3).  The tests pin
+the second and third to the first.
+"""
+from dataclasses import dataclass
+import numpy as np
+
+
+@dataclass(frozen=True)
+class Shape:
+    n_layers: int
+    d_model: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    d_ffn: int
+    vocab: int
+    rope_base: float = 10000.0
+    rms_eps: float = 1e-6
+    dtype: str = "fp32"          # "fp32" | "bf16": storage type of the matrices
+
+
+def mat(w, name, dt):
+    """Matrix `name` as dtype dt (widening compact bf16 bit patterns if needed)."""
+    t = w[name]
+    if t.dtype == np.uint16:
+        t = (t.astype(np.uint32) << np.uint32(16)).view(np.float32)
+    return t.astype(dt, copy=False)
+
+
+def rmsnorm(x, g, eps):
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x / np.sqrt(ms + eps) * g
+
+
+def rope_angles(pos, head_dim, base):
+    """[len(pos), head_dim/2] angles pos * base^(-2i/head_dim), in float64."""
+    i = np.arange(head_dim // 2, dtype=np.float64)
+    theta = np.float64(base) ** (-2.0 * i / head_dim)
+    return np.asarray(pos, dtype=np.float64)[:, None] * theta[None, :]
+
+
+def rope(x, pos, base):
+    """Rotate-half RoPE. x: [T, H, dh]; dimension i pairs with i + dh/2."""
+    dh = x.shape[-1]
+    ang = rope_angles(pos, dh, base)
+    c = np.cos(ang)[:, None, :].astype(x.dtype)
+    s = np.sin(ang)[:, None, :].astype(x.dtype)
+    x1, x2 = x[..., : dh // 2], x[..., dh // 2:]
+    return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
+
+
+def silu(x):
+    return x / (1.0 + np.exp(-x))
+
+
+def attend(q, k, v, visible):
+    """q [T,Hq,dh], k/v [U,Hkv,dh], visible [T,U] bool -> [T,Hq,dh]."""
+    T, hq, dh = q.shape
+    hkv = k.shape[1]
+    rep = hq // hkv
+    out = np.empty_like(q)
+    scale = 1.0 / np.sqrt(dh)
+    for h in range(hq):
+        s = (q[:, h, :] @ k[:, h // rep, :].T) * scale
+        s = np.where(visible, s, -np.inf)
+        s = s - s.max(axis=-1, keepdims=True)
+        p = np.exp(s)
+        p = p / p.sum(axis=-1, keepdims=True)
+        out[:, h, :] = p @ v[:, h // rep, :]
+    return out
+
+
+def _qkv(w, shape, l, x, pos, dt):
+    hq, hkv, dh = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+    h = rmsnorm(x, mat(w, f"layers.{l}.g1", dt), shape.rms_eps)
+    q = (h @ mat(w, f"layers.{l}.wq", dt).T).reshape(-1, hq, dh)
+    k = (h @ mat(w, f"layers.{l}.wk", dt).T).reshape(-1, hkv, dh)
+    v = (h @ mat(w, f"layers.{l}.wv", dt).T).reshape(-1, hkv, dh)
+    return rope(q, pos, shape.rope_base), rope(k, pos, shape.rope_base), v
+
+
+def _finish_layer(w, shape, l, x, a, dt):
+    x = x + a.reshape(x.shape[0], -1) @ mat(w, f"layers.{l}.wo", dt).T
+    h = rmsnorm(x, mat(w, f"layers.{l}.g2", dt), shape.rms_eps)
+    act = silu(h @ mat(w, f"layers.{l}.wg", dt).T) * (h @ mat(w, f"layers.{l}.wu", dt).T)
+    return x + act @ mat(w, f"layers.{l}.wd", dt).T
+
+
+def head(w, shape, x, dt):
+    return rmsnorm(x, mat(w, "gf", dt), shape.rms_eps) @ mat(w, "lm_head", dt).T
+
+
+def forward_full(w, shape, tokens, dt=np.float64, pos0=0, return_hidden=False):
+    """Logits [T, V] at every position of one token string (dense causal recompute)."""
+    tokens = np.asarray(tokens)
+    T = tokens.size
+    pos = np.arange(pos0, pos0 + T)
+    x = mat(w, "embed", dt)[tokens]
+    causal = np.tril(np.ones((T, T), dtype=bool))
+    for l in range(shape.n_layers):
+        q, k, v = _qkv(w, shape, l, x, pos, dt)
+        x = _finish_layer(w, shape, l, x, attend(q, k, v, causal), dt)
+    return x if return_hidden else head(w, shape, x, dt)
+
+
+class Incremental:
+    """Token-by-token decode of one sequence with a growing K/V list per layer."""
+
+    def __init__(self, w, shape, dt=np.float64):
+        self.w, self.shape, self.dt = w, shape, dt
+        self.k = [[] for _ in range(shape.n_layers)]
+        self.v = [[] for _ in range(shape.n_layers)]
+        self.n = 0
+
+    def step(self, token):
+        """Feed one token at position self.n; return the logits [V] after it."""
+        w, shape, dt = self.w, self.shape, self.dt
+        x = mat(w, "embed", dt)[np.asarray([token])]
+        for l in range(shape.n_layers):
+            q, k, v = _qkv(w, shape, l, x, [self.n], dt)
+            self.k[l].append(k[0]); self.v[l].append(v[0])
+            K = np.stack(self.k[l]); V = np.stack(self.v[l])
+            a = attend(q, K, V, np.ones((1, K.shape[0]), dtype=bool))
+            x = _finish_layer(w, shape, l, x, a, dt)
+        self.n += 1
+        return head(w, shape, x, dt)[0]
+
+
+class SharedPrefix:
+    """K/V of a cached prefix, computed once and read by all G samples of a group."""
+
+    def __init__(self, w, shape, prefix_tokens, dt=np.float64):
+        self.w, self.shape, self.dt = w, shape, dt
+        prefix_tokens = np.asarray(prefix_tokens)
+        self.P = P = prefix_tokens.size
+        x = mat(w, "embed", dt)[prefix_tokens]
+        causal = np.tril(np.ones((P, P), dtype=bool))
+        self.k, self.v = [], []
+        for l in range(shape.n_layers):
+            q, k, v = _qkv(w, shape, l, x, np.arange(P), dt)
+            self.k.append(k); self.v.append(v)
+            x = _finish_layer(w, shape, l, x, attend(q, k, v, causal), dt)
+        self.x_last = x[-1:].copy()                      # residual stream at the last prefix token
+
+    def step0_logits(self):
+        """Logits for suffix position 0 (shared by the whole group)."""
+        return head(self.w, self.shape, self.x_last, self.dt)[0]
+
+    def teacher_forced_hidden(self, suffix):
+        """Residual stream after feeding suffix tokens [S'] (one sample) at positions P.."""
+        w, shape, dt, P = self.w, self.shape, self.dt, self.P
+        suffix = np.asarray(suffix)
+        n = suffix.size
+        x = mat(w, "embed", dt)[suffix]
+        vis = np.concatenate([np.ones((n, P), dtype=bool), np.tril(np.ones((n, n), dtype=bool))], axis=1)
+        for l in range(shape.n_layers):
+            q, k, v = _qkv(w, shape, l, x, np.arange(P, P + n), dt)
+            K = np.concatenate([self.k[l], k]); V = np.concatenate([self.v[l], v])
+            x = _finish_layer(w, shape, l, x, attend(q, K, V, vis), dt)
+        return x
+
+    def teacher_forced_logits(self, suffix):
+        """Logits [len(suffix), V]: row j is the distribution of o_j given prefix, o_<j."""
+        suffix = np.asarray(suffix)
+        xs = self.x_last
+        if suffix.size > 1:
+            xs = np.concatenate([xs, self.teacher_forced_hidden(suffix[:-1])])
+        return head(self.w, self.shape, xs, self.dt)
