@@ -1,0 +1,205 @@
+/*
+ * rpo.h -- C ABI of the B200 rollout library for RPO (Reinforcement Fine-Tuning with
+ * Partial Reasoning Optimization).
+ *
+ * The library implements the rollout stage of the method: for every question q_k the
+ * cached response a_k is truncated and the policy generates G continuations of the
+ * prefix (Section 3.2 "Rollout", Eq. 3; Algorithm 1, inner loop over g = 1..G), and the
+ * per-token probabilities pi_theta(o_{i,j} | q, o_{i,<j}) that the probability ratio
+ * r_{i,j} of Eq. 7 is built from.  The caller hands over token arrays only: the prefix
+ * is the already concatenated string q_k || a_k^{[0:-m]}.
+ *
+ * Conventions
+ *  - Every function returns RPO_OK (0) or a negative RPO_ERR_* code; nothing throws or
+ *    aborts across this boundary.  rpo_strerror() names a code.
+ *  - Pointer prefixes: d_ = device memory owned by the caller (e.g. a torch tensor's
+ *    data pointer), h_ = host memory owned by the caller.  The library never frees or
+ *    keeps caller memory beyond the call, except that work reading/writing d_ buffers is
+ *    *enqueued* on the stream given to rpo_create and may still be running on return;
+ *    synchronise that stream before reading outputs or reusing inputs.
+ *  - All kernels run on the one CUDA stream passed at creation (0 = legacy default).
+ *  - There is no CPU fallback: without a CUDA device every compute call fails with
+ *    RPO_ERR_CUDA.
+ *  - Matrices are stored [out_features, in_features]; y = x W^T.
+ *  - Sequence number of sample i of group g, for the random stream: group_id * G + i.
+ */
+#ifndef RPO_H_
+#define RPO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define RPO_OK 0
+#define RPO_ERR_INVALID_ARG (-1)     /* NULL pointer, negative size, bad flag                      */
+#define RPO_ERR_SHAPE (-2)           /* decoder shape not supported by the kernels                */
+#define RPO_ERR_KV_POOL (-3)         /* not enough free KV blocks / group or sequence slots       */
+#define RPO_ERR_CUDA (-4)            /* a CUDA runtime call failed (no device, out of memory...)  */
+#define RPO_ERR_DEVICE_TIMEOUT (-5)  /* a bounded device-side wait ran out (see rpo_device_status)*/
+#define RPO_ERR_NOT_INITIALISED (-6) /* weights not initialised / group handle not live           */
+#define RPO_ERR_LIMIT (-7)           /* request exceeds a limit fixed at rpo_create               */
+
+#define RPO_DTYPE_FP32 0
+#define RPO_DTYPE_BF16 1
+
+typedef struct rpo_ctx rpo_ctx; /* opaque: weights, paged KV pool, block tables, workspaces */
+
+/* Decoder shape (the paper names the policy models only; these fields describe the
+ * pre-norm GQA decoder of the benchmark configurations). */
+typedef struct rpo_shape {
+  int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
+  float rope_base; /* theta_i = rope_base^(-2i/head_dim), rotate-half pairing           */
+  float rms_eps;   /* inside the square root                                            */
+  int32_t dtype;   /* RPO_DTYPE_*: storage type of matrices, K/V and GEMM inputs        */
+  int32_t kv_block_tokens; /* tokens per KV block; must be 16                           */
+} rpo_shape;
+
+/* Capacity fixed at creation. */
+typedef struct rpo_limits {
+  int64_t kv_pool_blocks;   /* KV blocks of kv_block_tokens tokens (all layers each)      */
+  int32_t max_groups;       /* live prompt groups                                         */
+  int32_t max_seqs;         /* sequences decoded in one rpo_decode_suffix call (n_groups*G)*/
+  int32_t max_chunk_tokens; /* rows one prefill / log-prob pass works on; a prefix must fit*/
+  int32_t max_positions;    /* prefix_len + max_new upper bound (RoPE table, block tables) */
+} rpo_limits;
+
+/* Sampler of pi_theta(. | q_k, prefix, o_<j) (Eq. 3).  temperature > 0; 0 <= top_p <= 1.
+ * greedy != 0: lowest token id among the maximal logits.  eos_id < 0: no early stop. */
+typedef struct rpo_sampler {
+  float temperature;
+  float top_p;
+  int32_t greedy;
+  int32_t eos_id;
+  uint64_t seed;
+} rpo_sampler;
+
+/* Handle of a prefilled prompt group (plain data, caller-held). */
+typedef struct rpo_group {
+  int32_t group_id;   /* caller's id; decides the random streams of the group's samples   */
+  int32_t prefix_len; /* tokens of the cached prefix held in shared KV blocks             */
+  int32_t slot;       /* library slot; do not modify                                      */
+  int32_t n_blocks;   /* shared KV blocks held by the group                               */
+} rpo_group;
+
+const char* rpo_strerror(int code);
+
+/* Fill *out with a named decoder shape: "tiny", "qwen1.5b-class", "qwen7b-class".
+ * Returns RPO_ERR_INVALID_ARG for an unknown name. */
+int rpo_shape_preset(const char* name, rpo_shape* out);
+
+/* Create a context on the current CUDA device: allocates the weight arena, the paged KV
+ * pool ([layer][K|V][kv_head][block][16][head_dim]), block tables and workspaces.
+ * cuda_stream is a cudaStream_t (may be NULL).  *out is owned by the caller until
+ * rpo_destroy.  Errors: RPO_ERR_SHAPE (head_dim not 64/128, d_model or d_ffn not a
+ * multiple of 8, n_q_heads not a multiple of n_kv_heads, kv_block_tokens != 16),
+ * RPO_ERR_CUDA (allocation failed). */
+int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limits* limits, void* cuda_stream);
+int rpo_destroy(rpo_ctx* ctx);
+
+/* Seeded random initialisation of the named decoder shape: every matrix element is
+ * float32(std) * z with z a standard normal taken from the Philox4x32-10 block
+ * (element_index / 4) of stream (seed, tensor id); bf16 models round to nearest even.
+ * RMSNorm gains are set to 1.  (The paper trains DeepSeek-R1-Distill-Qwen checkpoints,
+ * Section 4; random weights of the same shape stand in for them.) */
+int rpo_init_weights(rpo_ctx* ctx, uint64_t seed, float std);
+
+/* Copy one tensor to / from host memory in its storage type (float for fp32 models and
+ * for gains, uint16 bf16 bit patterns otherwise), logical layout [out, in].  Names:
+ * "embed", "lm_head", "gf", "layers.<l>.{wq,wk,wv,wo,wg,wu,wd,g1,g2}".  bytes must equal
+ * the tensor size.  Synchronises the stream. */
+int rpo_read_tensor(rpo_ctx* ctx, const char* name, void* h_dst, size_t bytes);
+int rpo_write_tensor(rpo_ctx* ctx, const char* name, const void* h_src, size_t bytes);
+
+/* Prefill: run the decoder over the cached prefix q_k || a_k^{[0:-m]} of each group ONCE
+ * and keep its K/V in KV blocks that all G samples of the group will read (Eq. 3; "the
+ * same response prefix is shared during the sampling phase", Section 3.4).
+ *   d_tokens   device int32, the n_groups prefixes concatenated
+ *   h_offsets  host int32 [n_groups+1], prefix g = d_tokens[h_offsets[g] .. h_offsets[g+1])
+ *   h_group_ids host int32 [n_groups] or NULL (ids 0..n_groups-1)
+ *   h_groups_out host [n_groups], filled before return (no device sync needed)
+ * Each prefix needs 1 <= len <= max_chunk_tokens and len < max_positions.
+ * Errors: RPO_ERR_KV_POOL (blocks or slots exhausted; nothing is kept), RPO_ERR_LIMIT,
+ * RPO_ERR_INVALID_ARG (token ids are NOT range-checked on the host; out-of-range ids are
+ * clamped on the device and flagged in rpo_device_status). */
+int rpo_prefill_prefix(rpo_ctx* ctx, int32_t n_groups, const int32_t* d_tokens, const int32_t* h_offsets,
+                       const int32_t* h_group_ids, rpo_group* h_groups_out);
+
+/* Decode: G continuations per group over the shared prefix KV (Eq. 3; Algorithm 1).
+ * Sequence b = g_index*G + i.  Step 0 draws all G samples of a group from the logits of
+ * the group's last prefix token; step j feeds token j-1.  A sequence that emits eos_id
+ * stops: the EOS token and its log-prob are recorded, later slots hold eos_id / 0.0 and
+ * d_lens_out counts tokens up to and including EOS.
+ *   d_forced_tokens  NULL, or device int32 [B*max_new]: teacher forcing -- these tokens
+ *                    are emitted instead of sampled ones (log-probs still computed)
+ *   d_tokens_out     device int32 [B*max_new]
+ *   d_lens_out       device int32 [B]
+ *   d_logprobs_out   NULL or device float [B*max_new]: log pi(o_j | ...), full vocabulary,
+ *                    at the sampler's temperature
+ *   d_logits_dbg     NULL or device float [B*max_new*vocab]: the float32 logits every
+ *                    step was drawn from (tests only; large)
+ * Private suffix KV blocks are taken from the pool for the duration of the call.
+ * Errors: RPO_ERR_LIMIT (B > max_seqs, prefix_len+max_new > max_positions),
+ * RPO_ERR_KV_POOL, RPO_ERR_NOT_INITIALISED (stale handle), RPO_ERR_INVALID_ARG. */
+int rpo_decode_suffix(rpo_ctx* ctx, int32_t n_groups, const rpo_group* h_groups, int32_t G, int32_t max_new,
+                      const rpo_sampler* sampler, const int32_t* d_forced_tokens, int32_t* d_tokens_out,
+                      int32_t* d_lens_out, float* d_logprobs_out, float* d_logits_dbg);
+
+/* Token log-probabilities log pi_theta(o_{i,j} | q, o_{i,<j}) of given suffixes (numerator
+ * and denominator of r_{i,j}, Eq. 7), teacher-forced over the shared prefix KV:
+ *   d_tokens [B*max_new], d_lens [B] as written by rpo_decode_suffix
+ *   z = logits * inv_temperature; normalisation over the full vocabulary
+ *   d_logprobs_out device float [B*max_new]; entries j >= len are 0
+ *   d_logits_dbg NULL or device float [B*max_new*vocab] (tests only)
+ * The [B*max_new, vocab] logits are produced in bounded row chunks, never whole. */
+int rpo_token_logprobs(rpo_ctx* ctx, int32_t n_groups, const rpo_group* h_groups, int32_t G, int32_t max_new,
+                       const int32_t* d_tokens, const int32_t* d_lens, float inv_temperature,
+                       float* d_logprobs_out, float* d_logits_dbg);
+
+/* Return the groups' shared KV blocks and slots to the pool (host bookkeeping; work
+ * already enqueued on the stream is unaffected because later work is ordered after it). */
+int rpo_release_groups(rpo_ctx* ctx, int32_t n_groups, const rpo_group* h_groups);
+
+/* Whole rollout with HOST buffers (the call an application makes once per batch):
+ * copies the prefix tokens to the device, prefills, decodes, optionally computes the
+ * teacher-forced log-probs (want_policy_logprobs != 0 -> h_policy_logprobs_out), copies
+ * the results back, releases the groups and synchronises the stream.
+ * h_tokens_out [B*max_new], h_lens_out [B], h_logprobs_out [B*max_new] or NULL. */
+int rpo_rollout_host(rpo_ctx* ctx, int32_t n_groups, const int32_t* h_tokens, const int32_t* h_offsets,
+                     const int32_t* h_group_ids, int32_t G, int32_t max_new, const rpo_sampler* sampler,
+                     int32_t* h_tokens_out, int32_t* h_lens_out, float* h_logprobs_out,
+                     int32_t want_policy_logprobs, float* h_policy_logprobs_out);
+
+/* The sampler alone, on caller-supplied float32 logits [n_rows, vocab] (row r belongs to
+ * sequence d_seq_ids[r], draw number `step`): used to test the sampler in isolation.
+ * d_tokens_out int32 [n_rows]; d_logprobs_out NULL or float [n_rows]. */
+int rpo_sample_rows(rpo_ctx* ctx, int32_t n_rows, int32_t vocab, const float* d_logits, const rpo_sampler* sampler,
+                    const int64_t* d_seq_ids, int32_t step, int32_t* d_tokens_out, float* d_logprobs_out);
+
+/* Dense product C[M,N] = A[M,K] * W[N,K]^T through the same GEMM kernel the layers use
+ * (storage type of the context; C is float32).  For kernel-level parity tests.
+ * impl: 0 = the kernel the context would choose, 1 = plain CUDA-core kernel,
+ * 2 = tcgen05/TMA kernel (bf16 only; RPO_ERR_SHAPE if K % 64 != 0 or N % 16 != 0). */
+int rpo_gemm(rpo_ctx* ctx, int32_t impl, int32_t M, int32_t N, int32_t K, const void* d_A, const void* d_W,
+             float* d_C);
+
+/* Device status word, sticky until read: 0 = clean; bit 0 = a bounded wait expired
+ * (TMA / MMA pipeline), bit 1 = token id out of range (clamped), bit 2 = block-table
+ * index out of range (access skipped).  Synchronises the stream; *out receives the word
+ * and the word is cleared. */
+int rpo_device_status(rpo_ctx* ctx, int32_t* out);
+
+/* Counters since creation: kernels launched by the library, free KV blocks. */
+int rpo_counters(rpo_ctx* ctx, int64_t* kernel_launches, int64_t* free_kv_blocks);
+
+/* Runtime switches (tests/benchmarks): name = "use_tcgen05" (bf16 GEMMs on the tensor-core
+ * kernel, default 1), "use_tc_attention" (tensor-core attention kernels, default 1),
+ * "use_graph" (CUDA graph per decode step, default 1). */
+int rpo_set_option(rpo_ctx* ctx, const char* name, int32_t value);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RPO_H_ */

@@ -1,0 +1,87 @@
+// Host-side state of one rollout context.
+#pragma once
+#include <cuda_runtime.h>
+#include <map>
+#include <string>
+#include <vector>
+
+#include "../../include/rpo.h"
+
+namespace rpo {
+
+struct TensorInfo {
+  void* ptr = nullptr;     // physical base
+  int rows = 0, cols = 0;  // logical [out, in]
+  int row_mul = 1;         // logical row r lives at physical row r*row_mul + row_add of `ptr`
+  int row_add = 0;
+  bool gain = false;       // float32 vector
+  uint32_t tensor_id = 0;
+};
+
+struct LayerWeights {
+  void *wqkv, *wo, *wgu, *wd;  // fused [q|k|v] rows; gate/up rows interleaved
+  float *g1, *g2;
+};
+
+struct GroupState {
+  bool live = false;
+  int32_t group_id = 0, prefix_len = 0;
+  std::vector<int32_t> blocks;
+};
+
+struct Workspace {
+  float* x = nullptr;      // [R, d] residual stream
+  void* h = nullptr;       // [R, d]
+  void* qkv = nullptr;     // [R, (Hq+2Hkv)*dh]
+  void* attn = nullptr;    // [R, Hq*dh]
+  void* gu = nullptr;      // [R, 2F]
+  void* act = nullptr;     // [R, F]
+  float* xh = nullptr;     // [HR, d] head input rows
+  void* hh = nullptr;      // [HR, d]
+  float* logits = nullptr; // [HR, V]
+  float* partial = nullptr;      // split-K partial sums
+  size_t partial_elems = 0;
+  float* attn_part = nullptr;    // decode attention partials
+  size_t attn_part_elems = 0;
+  int32_t *row_seq = nullptr, *row_t = nullptr, *row_tok = nullptr;
+  void* seqs = nullptr;    // SeqDesc[]
+  int32_t *done = nullptr, *lens = nullptr, *cur_tok = nullptr, *logit_row = nullptr, *slot_idx = nullptr;
+  int64_t* seq_ids = nullptr;
+  int R = 0, HR = 0;
+};
+
+}  // namespace rpo
+
+struct rpo_ctx {
+  rpo_shape shape;
+  rpo_limits lim;
+  cudaStream_t stream = nullptr;
+  bool bf16 = false;
+  size_t esz = 4;
+  int qkv_cols = 0;
+  // weights
+  std::vector<void*> allocations;
+  std::map<std::string, rpo::TensorInfo> tensors;
+  std::vector<rpo::LayerWeights> layers;
+  void *embed = nullptr, *lm_head = nullptr;
+  float* gf = nullptr;
+  bool weights_ready = false;
+  // paged KV
+  void* kv_base = nullptr;
+  int64_t kv_layer_stride = 0, kv_kv_stride = 0, kv_head_stride = 0;
+  std::vector<int32_t> free_blocks;
+  int32_t* d_block_table = nullptr;
+  int tbl_stride = 0;
+  std::vector<int32_t> free_slots;
+  std::vector<rpo::GroupState> groups;
+  float* d_x_last = nullptr;   // [max_groups, d]
+  void* d_rope = nullptr;      // float2 [max_positions, dh/2]
+  rpo::Workspace ws;
+  int* d_status = nullptr;
+  int64_t launches = 0;
+  int sm_count = 148;
+  // options
+  int use_tcgen05 = 1, use_tc_attention = 1, use_graph = 1;
+  // tcgen05 GEMM state (tensor maps are built per call; see gemm_tc.cuh)
+  void* tc_state = nullptr;
+};

@@ -1,0 +1,274 @@
+// Elementwise / row kernels of the rollout path: seeded init, embedding gather, RMSNorm (with the
+// split-K reduction and residual add folded in), RoPE + paged K/V write, SwiGLU, row gathers and
+// the log-probability row kernel.  T is the storage type (float or bf16); statistics are float32.
+#pragma once
+#include "common.cuh"
+
+namespace rpo {
+
+// Per-sequence view of the paged KV cache: a shared segment (the group's prefix blocks, fully
+// visible) followed by a private segment (causal).  Offsets index the int32 block table.
+struct SeqDesc {
+  int32_t shared_tbl;  // first block-table entry of the shared segment, -1 if none
+  int32_t shared_len;  // tokens in the shared segment
+  int32_t priv_tbl;    // first block-table entry of the private segment
+  int32_t reserved;
+};
+
+template <typename T>
+struct KVPool {
+  T* base;
+  int64_t layer_stride, kv_stride, head_stride;  // elements
+  int32_t n_blocks, head_dim;
+  __device__ __forceinline__ T* at(int layer, int kv, int head, int block, int off) const {
+    return base + layer * layer_stride + kv * kv_stride + head * head_stride +
+           ((int64_t)block * KV_BLOCK + off) * head_dim;
+  }
+};
+
+// --------------------------------------------------------------------------------------------
+// Seeded N(0, std^2) init.  Thread = one Philox block = 4 consecutive logical elements.
+// Logical element e = row*cols + col lands at dst[(row*row_mul + row_add)*cols + col], which
+// lets gate/up rows interleave and q/k/v rows stack inside fused matrices.
+// --------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void init_normal_kernel(T* __restrict__ dst, int64_t n_elems, int cols, int row_mul, int row_add,
+                                   uint32_t k0, uint32_t k1, uint32_t tensor_id, float stdv) {
+  const int64_t n_blocks = (n_elems + 3) / 4;
+  for (int64_t blk = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; blk < n_blocks;
+       blk += (int64_t)gridDim.x * blockDim.x) {
+    const U4 r = philox4x32_10((uint32_t)blk, (uint32_t)((uint64_t)blk >> 32), tensor_id, 1u, k0, k1);
+    float z[4];
+    const uint32_t xa[2] = {r.x, r.z}, xb[2] = {r.y, r.w};
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const float u1 = rmul(radd((float)(xa[j] >> 9), 0.5f), 1.1920928955078125e-07f);  // 2^-23
+      const float rad = __fsqrt_rn(rmul(-2.0f, ln_unit(u1)));
+      float sn, cs;
+      sincos_turn24(xb[j] >> 8, &sn, &cs);
+      z[2 * j] = rmul(rad, cs);
+      z[2 * j + 1] = rmul(rad, sn);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int64_t e = blk * 4 + j;
+      if (e < n_elems) {
+        const int64_t row = e / cols, col = e % cols;
+        dst[(row * row_mul + row_add) * cols + col] = from_f32<T>(rmul(z[j], stdv));
+      }
+    }
+  }
+}
+
+template <typename T>
+__global__ void fill_kernel(T* dst, int64_t n, float v) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+    dst[i] = from_f32<T>(v);
+}
+
+// cos/sin table [max_positions][head_dim/2], angles in float64.
+__global__ void rope_table_kernel(float2* __restrict__ tab, int max_pos, int half, double base) {
+  const int64_t n = (int64_t)max_pos * half;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    const int pos = (int)(i / half), j = (int)(i % half);
+    const double theta = pow(base, -2.0 * (double)j / (double)(2 * half));
+    double s, c;
+    sincos((double)pos * theta, &s, &c);
+    tab[i] = make_float2((float)c, (float)s);
+  }
+}
+
+// x[r,:] = E[tok[r],:]  (float32 residual stream).
+template <typename T>
+__global__ void embed_kernel(const int32_t* __restrict__ tokens, const T* __restrict__ E, float* __restrict__ x,
+                             int rows, int d, int vocab, int* status) {
+  const int r = blockIdx.x;
+  if (r >= rows) return;
+  int tok = tokens[r];
+  if (tok < 0 || tok >= vocab) {
+    if (threadIdx.x == 0) atomicOr(status, STATUS_BAD_TOKEN);
+    tok = min(max(tok, 0), vocab - 1);
+  }
+  const T* src = E + (int64_t)tok * d;
+  float* dst = x + (int64_t)r * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = to_f32(src[i]);
+}
+
+// dst[r,:] = src[idx[r],:]  (float32 rows; idx may be NULL = identity)
+__global__ void gather_rows_f32_kernel(const float* __restrict__ src, const int32_t* __restrict__ idx,
+                                       float* __restrict__ dst, int rows, int d) {
+  const int r = blockIdx.x;
+  if (r >= rows) return;
+  const int s = idx ? idx[r] : r;
+  if (s < 0) {
+    for (int i = threadIdx.x; i < d; i += blockDim.x) dst[(int64_t)r * d + i] = 0.f;
+    return;
+  }
+  for (int i = threadIdx.x; i < d; i += blockDim.x) dst[(int64_t)r * d + i] = src[(int64_t)s * d + i];
+}
+
+// RMSNorm of the float32 residual stream, one CTA per row:
+//   x[r,:] += sum_s partial[s][r,:]   (optional split-K partial sums of the previous GEMM)
+//   h[r,:]  = x[r,:] / sqrt(mean(x^2) + eps) * g
+template <typename T>
+__global__ void rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ gain, T* __restrict__ h, int rows,
+                               int d, float eps, const float* __restrict__ partial, int n_splits,
+                               int64_t split_stride) {
+  extern __shared__ float srow[];
+  __shared__ float red[32];
+  const int r = blockIdx.x;
+  if (r >= rows) return;
+  float* xr = x + (int64_t)r * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    float v = xr[i];
+    if (partial) {
+      for (int s = 0; s < n_splits; ++s) v += partial[s * split_stride + (int64_t)r * d + i];
+      xr[i] = v;
+    }
+    srow[i] = v;
+    ss += v * v;
+  }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float v = (threadIdx.x < (blockDim.x >> 5)) ? red[threadIdx.x] : 0.f;
+    v = warp_sum(v);
+    if (threadIdx.x == 0) red[0] = v;
+  }
+  __syncthreads();
+  const float inv = 1.0f / sqrtf(red[0] / (float)d + eps);
+  T* hr = h + (int64_t)r * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) hr[i] = from_f32<T>(srow[i] * inv * gain[i]);
+}
+
+// RoPE (rotate-half) on q and k, then K/V written to the row's slot of its private segment.
+// qkv row layout: [q heads | k heads | v heads] x head_dim.  Grid: (rows, Hq + 2*Hkv).
+template <typename T>
+__global__ void rope_kv_kernel(T* __restrict__ qkv, const int32_t* __restrict__ row_seq,
+                               const int32_t* __restrict__ row_t, const SeqDesc* __restrict__ seqs,
+                               const int32_t* __restrict__ block_table, const float2* __restrict__ rope_tab,
+                               KVPool<T> pool, int layer, int rows, int hq, int hkv, int max_pos, int* status) {
+  const int r = blockIdx.x, head = blockIdx.y;
+  if (r >= rows) return;
+  const int t = row_t[r];
+  if (t < 0) return;
+  const int dh = pool.head_dim, half = dh / 2;
+  const SeqDesc sd = seqs[row_seq[r]];
+  const int pos = sd.shared_len + t;
+  if (pos >= max_pos) { if (threadIdx.x == 0) atomicOr(status, STATUS_BAD_BLOCK); return; }
+  T* src = qkv + (int64_t)r * (hq + 2 * hkv) * dh + (int64_t)head * dh;
+  T* dst = nullptr;
+  if (head >= hq) {
+    const int kv = (head - hq) / hkv, kh = (head - hq) % hkv;
+    const int blk = block_table[sd.priv_tbl + t / KV_BLOCK];
+    if (blk < 0 || blk >= pool.n_blocks) { if (threadIdx.x == 0) atomicOr(status, STATUS_BAD_BLOCK); return; }
+    dst = pool.at(layer, kv, kh, blk, t % KV_BLOCK);
+  }
+  if (head < hq + hkv) {  // q or k: rotate
+    for (int i = threadIdx.x; i < half; i += blockDim.x) {
+      const float2 cs = rope_tab[(int64_t)pos * half + i];
+      const float a = to_f32(src[i]), b = to_f32(src[i + half]);
+      const T o1 = from_f32<T>(a * cs.x - b * cs.y), o2 = from_f32<T>(b * cs.x + a * cs.y);
+      if (dst) { dst[i] = o1; dst[i + half] = o2; } else { src[i] = o1; src[i + half] = o2; }
+    }
+  } else {
+    for (int i = threadIdx.x; i < dh; i += blockDim.x) dst[i] = src[i];
+  }
+}
+
+// act[r, j] = silu(gu[r, 2j]) * gu[r, 2j+1]   (gate/up interleaved by the fused weight layout)
+template <typename T>
+__global__ void swiglu_kernel(const T* __restrict__ gu, T* __restrict__ act, int64_t n_out) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_out; i += (int64_t)gridDim.x * blockDim.x) {
+    const float g = to_f32(gu[2 * i]), u = to_f32(gu[2 * i + 1]);
+    act[i] = from_f32<T>(g / (1.0f + __expf(-g)) * u);
+  }
+}
+
+// Row metadata of a teacher-forced pass: row (s, j), j in [0, S-1), feeds token j of sequence s at
+// private index j; it is active when j < len[s]-1.  Also the input token of the row.
+__global__ void build_teacher_rows_kernel(const int32_t* __restrict__ tokens, const int32_t* __restrict__ lens,
+                                          int seq0, int n_seq, int S, int32_t* __restrict__ row_seq,
+                                          int32_t* __restrict__ row_t, int32_t* __restrict__ row_tok) {
+  const int n = n_seq * (S - 1);
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    const int s = i / (S - 1), j = i % (S - 1);
+    const int len = lens[seq0 + s];
+    row_seq[i] = s;
+    row_t[i] = (j < len - 1) ? j : -1;
+    row_tok[i] = (j < len - 1) ? tokens[(int64_t)(seq0 + s) * S + j] : 0;
+  }
+}
+
+// Gather index for the head of a teacher-forced pass over head-rows (s, j), j in [0,S):
+// j = 0 reads the group's last-prefix residual (index = -(1 + x_last slot) encoded), j >= 1 reads
+// layer-stack row (s, j-1).  Here we simply materialise the head input rows.
+__global__ void gather_head_rows_kernel(const float* __restrict__ x, const float* __restrict__ x_last,
+                                        const int32_t* __restrict__ seq_slot, int row0, int n_rows, int S, int d,
+                                        float* __restrict__ dst) {
+  const int i = blockIdx.x;
+  if (i >= n_rows) return;
+  const int hr = row0 + i, s = hr / S, j = hr % S;
+  const float* src = (j == 0) ? x_last + (int64_t)seq_slot[s] * d : x + ((int64_t)s * (S - 1) + (j - 1)) * d;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) dst[(int64_t)i * d + c] = src[c];
+}
+
+__device__ __forceinline__ float block_reduce_max(float v, float* red) {
+  v = warp_max(v);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float w = (threadIdx.x < (blockDim.x >> 5)) ? red[threadIdx.x] : -INFINITY;
+    w = warp_max(w);
+    if (threadIdx.x == 0) red[0] = w;
+  }
+  __syncthreads();
+  const float out = red[0];
+  __syncthreads();
+  return out;
+}
+__device__ __forceinline__ float block_reduce_sum(float v, float* red) {
+  v = warp_sum(v);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float w = (threadIdx.x < (blockDim.x >> 5)) ? red[threadIdx.x] : 0.f;
+    w = warp_sum(w);
+    if (threadIdx.x == 0) red[0] = w;
+  }
+  __syncthreads();
+  const float out = red[0];
+  __syncthreads();
+  return out;
+}
+
+// log-prob of the given token per head-row of a teacher-forced pass (full-vocabulary
+// normalisation, z = logits * inv_T); rows with j >= len get 0.
+__global__ void logprob_rows_kernel(const float* __restrict__ logits, int row0, int n_rows, int V, int S,
+                                    const int32_t* __restrict__ tokens, const int32_t* __restrict__ lens, int seq0,
+                                    float inv_T, float* __restrict__ out, float* __restrict__ logits_dbg) {
+  __shared__ float red[32];
+  const int i = blockIdx.x;
+  if (i >= n_rows) return;
+  const int hr = row0 + i, s = hr / S, j = hr % S;
+  const int64_t o = (int64_t)(seq0 + s) * S + j;
+  const float* row = logits + (int64_t)i * V;
+  if (logits_dbg)
+    for (int c = threadIdx.x; c < V; c += blockDim.x) logits_dbg[o * V + c] = row[c];
+  if (j >= lens[seq0 + s]) { if (threadIdx.x == 0) out[o] = 0.f; return; }
+  float m = -INFINITY;
+  for (int c = threadIdx.x; c < V; c += blockDim.x) m = fmaxf(m, row[c] * inv_T);
+  m = block_reduce_max(m, red);
+  float sum = 0.f;
+  for (int c = threadIdx.x; c < V; c += blockDim.x) sum += __expf(row[c] * inv_T - m);
+  sum = block_reduce_sum(sum, red);
+  if (threadIdx.x == 0) {
+    int tok = tokens[o];
+    tok = min(max(tok, 0), V - 1);
+    out[o] = (row[tok] * inv_T - m) - logf(sum);
+  }
+}
+
+}  // namespace rpo

@@ -1,0 +1,726 @@
+// C ABI of the rollout library: context, weights, paged KV bookkeeping and the orchestration of
+// prefill (Eq. 3: prefix computed once per group), suffix decode (G samples per group, Algorithm 1
+// rollout loop) and teacher-forced token log-probabilities (Eq. 7).
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "context.h"
+#include "gemm_tc.cuh"
+#include "kernels.cuh"
+#include "ref_kernels.cuh"
+#include "sampler.cuh"
+
+using namespace rpo;
+
+#define CUDA_TRY(expr)                                                              \
+  do {                                                                              \
+    cudaError_t e_ = (expr);                                                        \
+    if (e_ != cudaSuccess) {                                                        \
+      fprintf(stderr, "[rpo] CUDA error %s at %s:%d: %s\n", cudaGetErrorName(e_), __FILE__, __LINE__, \
+              cudaGetErrorString(e_));                                              \
+      return RPO_ERR_CUDA;                                                          \
+    }                                                                               \
+  } while (0)
+
+#define RPO_TRY(expr)            \
+  do {                           \
+    int r_ = (expr);             \
+    if (r_ != RPO_OK) return r_; \
+  } while (0)
+
+#define LAUNCH(ctx, kern, grid, block, smem, ...)                         \
+  do {                                                                    \
+    kern<<<(grid), (block), (smem), (ctx)->stream>>>(__VA_ARGS__);        \
+    (ctx)->launches++;                                                    \
+    CUDA_TRY(cudaGetLastError());                                         \
+  } while (0)
+
+static inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
+static inline int grid_for(int64_t n, int block, int cap = 148 * 16) {
+  return (int)std::max<int64_t>(1, std::min<int64_t>((n + block - 1) / block, cap));
+}
+
+extern "C" const char* rpo_strerror(int code) {
+  switch (code) {
+    case RPO_OK: return "ok";
+    case RPO_ERR_INVALID_ARG: return "invalid argument";
+    case RPO_ERR_SHAPE: return "unsupported decoder shape";
+    case RPO_ERR_KV_POOL: return "KV pool, group slots or sequence slots exhausted";
+    case RPO_ERR_CUDA: return "CUDA runtime error";
+    case RPO_ERR_DEVICE_TIMEOUT: return "bounded device-side wait expired";
+    case RPO_ERR_NOT_INITIALISED: return "weights not initialised or group handle not live";
+    case RPO_ERR_LIMIT: return "request exceeds a limit fixed at rpo_create";
+    default: return "unknown error code";
+  }
+}
+
+extern "C" int rpo_shape_preset(const char* name, rpo_shape* out) {
+  if (!name || !out) return RPO_ERR_INVALID_ARG;
+  rpo_shape s;
+  memset(&s, 0, sizeof(s));
+  s.rms_eps = 1e-6f;
+  s.kv_block_tokens = KV_BLOCK;
+  if (!strcmp(name, "tiny")) {
+    s.n_layers = 2; s.d_model = 256; s.n_q_heads = 4; s.n_kv_heads = 2; s.head_dim = 64; s.d_ffn = 688;
+    s.vocab = 1024; s.rope_base = 10000.f; s.dtype = RPO_DTYPE_FP32;
+  } else if (!strcmp(name, "qwen1.5b-class")) {
+    s.n_layers = 28; s.d_model = 1536; s.n_q_heads = 12; s.n_kv_heads = 2; s.head_dim = 128; s.d_ffn = 8960;
+    s.vocab = 151936; s.rope_base = 1e6f; s.dtype = RPO_DTYPE_BF16;
+  } else if (!strcmp(name, "qwen7b-class")) {
+    s.n_layers = 28; s.d_model = 3584; s.n_q_heads = 28; s.n_kv_heads = 4; s.head_dim = 128; s.d_ffn = 18944;
+    s.vocab = 152064; s.rope_base = 1e6f; s.dtype = RPO_DTYPE_BF16;
+  } else {
+    return RPO_ERR_INVALID_ARG;
+  }
+  *out = s;
+  return RPO_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// creation
+// ---------------------------------------------------------------------------------------------
+static int dev_alloc(rpo_ctx* c, void** p, size_t bytes) {
+  *p = nullptr;
+  if (bytes == 0) bytes = 16;
+  cudaError_t e = cudaMalloc(p, bytes);
+  if (e != cudaSuccess) {
+    fprintf(stderr, "[rpo] cudaMalloc(%zu) failed: %s\n", bytes, cudaGetErrorString(e));
+    cudaGetLastError();
+    return RPO_ERR_CUDA;
+  }
+  c->allocations.push_back(*p);
+  return RPO_OK;
+}
+
+static void add_tensor(rpo_ctx* c, const std::string& name, void* ptr, int rows, int cols, int row_mul, int row_add,
+                       bool gain, uint32_t id) {
+  TensorInfo t;
+  t.ptr = ptr; t.rows = rows; t.cols = cols; t.row_mul = row_mul; t.row_add = row_add; t.gain = gain; t.tensor_id = id;
+  c->tensors[name] = t;
+}
+
+extern "C" int rpo_destroy(rpo_ctx* ctx) {
+  if (!ctx) return RPO_ERR_INVALID_ARG;
+  cudaStreamSynchronize(ctx->stream);
+  tc_destroy(ctx);
+  for (void* p : ctx->allocations) cudaFree(p);
+  delete ctx;
+  return RPO_OK;
+}
+
+extern "C" int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limits* lim, void* cuda_stream) {
+  if (!out || !shape || !lim) return RPO_ERR_INVALID_ARG;
+  *out = nullptr;
+  const rpo_shape& s = *shape;
+  if (s.n_layers < 0 || s.d_model <= 0 || s.n_q_heads <= 0 || s.n_kv_heads <= 0 || s.d_ffn <= 0 || s.vocab <= 0)
+    return RPO_ERR_SHAPE;
+  if ((s.head_dim != 64 && s.head_dim != 128) || s.n_q_heads % s.n_kv_heads || s.kv_block_tokens != KV_BLOCK ||
+      s.d_model % 8 || s.d_ffn % 8 || (s.dtype != RPO_DTYPE_FP32 && s.dtype != RPO_DTYPE_BF16) || s.rms_eps < 0)
+    return RPO_ERR_SHAPE;
+  if (lim->kv_pool_blocks <= 0 || lim->max_groups <= 0 || lim->max_seqs <= 0 || lim->max_chunk_tokens <= 0 ||
+      lim->max_positions <= 1)
+    return RPO_ERR_INVALID_ARG;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
+    cudaGetLastError();
+    fprintf(stderr, "[rpo] no CUDA device: this library has no CPU path\n");
+    return RPO_ERR_CUDA;
+  }
+  rpo_ctx* c = new (std::nothrow) rpo_ctx();
+  if (!c) return RPO_ERR_CUDA;
+  c->shape = s; c->lim = *lim; c->stream = (cudaStream_t)cuda_stream;
+  c->bf16 = s.dtype == RPO_DTYPE_BF16; c->esz = c->bf16 ? 2 : 4;
+  c->qkv_cols = (s.n_q_heads + 2 * s.n_kv_heads) * s.head_dim;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev);
+  const size_t e = c->esz;
+  const int d = s.d_model, dh = s.head_dim, F = s.d_ffn, V = s.vocab, qo = s.n_q_heads * dh;
+  int rc = RPO_OK;
+#define ALLOC(ptr, bytes)                                         \
+  if (rc == RPO_OK) rc = dev_alloc(c, (void**)&(ptr), (size_t)(bytes));
+  // ---- weights
+  ALLOC(c->embed, (size_t)V * d * e);
+  ALLOC(c->lm_head, (size_t)V * d * e);
+  ALLOC(c->gf, (size_t)d * 4);
+  c->layers.resize(s.n_layers);
+  for (int l = 0; l < s.n_layers && rc == RPO_OK; ++l) {
+    LayerWeights& L = c->layers[l];
+    ALLOC(L.wqkv, (size_t)c->qkv_cols * d * e);
+    ALLOC(L.wo, (size_t)d * qo * e);
+    ALLOC(L.wgu, (size_t)2 * F * d * e);
+    ALLOC(L.wd, (size_t)d * F * e);
+    ALLOC(L.g1, (size_t)d * 4);
+    ALLOC(L.g2, (size_t)d * 4);
+    if (rc != RPO_OK) break;
+    const std::string p = "layers." + std::to_string(l) + ".";
+    const uint32_t id = 16 + 8 * l;
+    char* qkv = (char*)L.wqkv;
+    add_tensor(c, p + "wq", qkv, qo, d, 1, 0, false, id + 0);
+    add_tensor(c, p + "wk", qkv + (size_t)qo * d * e, s.n_kv_heads * dh, d, 1, 0, false, id + 1);
+    add_tensor(c, p + "wv", qkv + (size_t)(qo + s.n_kv_heads * dh) * d * e, s.n_kv_heads * dh, d, 1, 0, false, id + 2);
+    add_tensor(c, p + "wo", L.wo, d, qo, 1, 0, false, id + 3);
+    add_tensor(c, p + "wg", L.wgu, F, d, 2, 0, false, id + 4);
+    add_tensor(c, p + "wu", L.wgu, F, d, 2, 1, false, id + 5);
+    add_tensor(c, p + "wd", L.wd, d, F, 1, 0, false, id + 6);
+    add_tensor(c, p + "g1", L.g1, 1, d, 1, 0, true, 0);
+    add_tensor(c, p + "g2", L.g2, 1, d, 1, 0, true, 0);
+  }
+  if (rc == RPO_OK) {
+    add_tensor(c, "embed", c->embed, V, d, 1, 0, false, 0);
+    add_tensor(c, "lm_head", c->lm_head, V, d, 1, 0, false, 1);
+    add_tensor(c, "gf", c->gf, 1, d, 1, 0, true, 0);
+  }
+  // ---- paged KV pool [layer][K|V][kv head][block][16][dh]
+  c->kv_head_stride = (int64_t)lim->kv_pool_blocks * KV_BLOCK * dh;
+  c->kv_kv_stride = c->kv_head_stride * s.n_kv_heads;
+  c->kv_layer_stride = c->kv_kv_stride * 2;
+  ALLOC(c->kv_base, (size_t)std::max(1, s.n_layers) * c->kv_layer_stride * e);
+  c->free_blocks.resize(lim->kv_pool_blocks);
+  for (int64_t i = 0; i < lim->kv_pool_blocks; ++i) c->free_blocks[i] = (int32_t)(lim->kv_pool_blocks - 1 - i);
+  c->tbl_stride = ceil_div(lim->max_positions, KV_BLOCK);
+  ALLOC(c->d_block_table, (size_t)(lim->max_groups + lim->max_seqs) * c->tbl_stride * 4);
+  c->groups.resize(lim->max_groups);
+  for (int i = lim->max_groups - 1; i >= 0; --i) c->free_slots.push_back(i);
+  ALLOC(c->d_x_last, (size_t)lim->max_groups * d * 4);
+  ALLOC(c->d_rope, (size_t)lim->max_positions * (dh / 2) * sizeof(float2));
+  ALLOC(c->d_status, 16);
+  // ---- workspaces
+  Workspace& w = c->ws;
+  w.R = std::max(lim->max_chunk_tokens, lim->max_seqs);
+  w.HR = std::max(std::max(lim->max_seqs, lim->max_groups), std::min(1024, std::max(lim->max_chunk_tokens, 1)));
+  ALLOC(w.x, (size_t)w.R * d * 4);
+  ALLOC(w.h, (size_t)w.R * d * e);
+  ALLOC(w.qkv, (size_t)w.R * c->qkv_cols * e);
+  ALLOC(w.attn, (size_t)w.R * qo * e);
+  ALLOC(w.gu, (size_t)w.R * 2 * F * e);
+  ALLOC(w.act, (size_t)w.R * F * e);
+  ALLOC(w.xh, (size_t)w.HR * d * 4);
+  ALLOC(w.hh, (size_t)w.HR * d * e);
+  ALLOC(w.logits, (size_t)w.HR * V * 4);
+  ALLOC(w.row_seq, (size_t)w.R * 4);
+  ALLOC(w.row_t, (size_t)w.R * 4);
+  ALLOC(w.row_tok, (size_t)w.R * 4);
+  const int nseq = std::max(lim->max_seqs, lim->max_groups);
+  ALLOC(w.seqs, (size_t)nseq * sizeof(SeqDesc));
+  ALLOC(w.done, (size_t)nseq * 4);
+  ALLOC(w.lens, (size_t)nseq * 4);
+  ALLOC(w.cur_tok, (size_t)nseq * 4);
+  ALLOC(w.logit_row, (size_t)nseq * 4);
+  ALLOC(w.slot_idx, (size_t)nseq * 4);
+  ALLOC(w.seq_ids, (size_t)nseq * 8);
+  if (rc == RPO_OK) rc = tc_create(c);
+#undef ALLOC
+  if (rc != RPO_OK) { rpo_destroy(c); return rc; }
+  cudaMemsetAsync(c->d_status, 0, 16, c->stream);
+  rope_table_kernel<<<grid_for((int64_t)lim->max_positions * (dh / 2), 256), 256, 0, c->stream>>>(
+      (float2*)c->d_rope, lim->max_positions, dh / 2, (double)s.rope_base);
+  c->launches++;
+  if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(c->stream) != cudaSuccess) {
+    rpo_destroy(c);
+    return RPO_ERR_CUDA;
+  }
+  *out = c;
+  return RPO_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// weights
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+static int init_weights_t(rpo_ctx* c, uint64_t seed, float stdv) {
+  const uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+  for (auto& kv : c->tensors) {
+    const TensorInfo& t = kv.second;
+    const int64_t n = (int64_t)t.rows * t.cols;
+    if (t.gain) {
+      LAUNCH(c, fill_kernel<float>, grid_for(n, 256), 256, 0, (float*)t.ptr, n, 1.0f);
+    } else {
+      LAUNCH(c, init_normal_kernel<T>, grid_for((n + 3) / 4, 256, 148 * 32), 256, 0, (T*)t.ptr, n, t.cols, t.row_mul,
+             t.row_add, k0, k1, t.tensor_id, stdv);
+    }
+  }
+  return RPO_OK;
+}
+
+extern "C" int rpo_init_weights(rpo_ctx* c, uint64_t seed, float stdv) {
+  if (!c || !(stdv >= 0.f)) return RPO_ERR_INVALID_ARG;
+  RPO_TRY(c->bf16 ? init_weights_t<bf16>(c, seed, stdv) : init_weights_t<float>(c, seed, stdv));
+  c->weights_ready = true;
+  return RPO_OK;
+}
+
+static int tensor_io(rpo_ctx* c, const char* name, void* host, size_t bytes, bool write) {
+  if (!c || !name || !host) return RPO_ERR_INVALID_ARG;
+  auto it = c->tensors.find(name);
+  if (it == c->tensors.end()) return RPO_ERR_INVALID_ARG;
+  const TensorInfo& t = it->second;
+  const size_t e = t.gain ? 4 : c->esz;
+  if (bytes != (size_t)t.rows * t.cols * e) return RPO_ERR_INVALID_ARG;
+  const size_t row_bytes = (size_t)t.cols * e;
+  char* base = (char*)t.ptr + (size_t)t.row_add * row_bytes;
+  const size_t pitch = row_bytes * t.row_mul;
+  if (write)
+    CUDA_TRY(cudaMemcpy2DAsync(base, pitch, host, row_bytes, row_bytes, t.rows, cudaMemcpyHostToDevice, c->stream));
+  else
+    CUDA_TRY(cudaMemcpy2DAsync(host, row_bytes, base, pitch, row_bytes, t.rows, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(cudaStreamSynchronize(c->stream));
+  if (write) c->weights_ready = true;
+  return RPO_OK;
+}
+extern "C" int rpo_read_tensor(rpo_ctx* c, const char* name, void* h_dst, size_t bytes) {
+  return tensor_io(c, name, h_dst, bytes, false);
+}
+extern "C" int rpo_write_tensor(rpo_ctx* c, const char* name, const void* h_src, size_t bytes) {
+  return tensor_io(c, name, const_cast<void*>(h_src), bytes, true);
+}
+
+// ---------------------------------------------------------------------------------------------
+// building blocks
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+static KVPool<T> kv_pool(rpo_ctx* c) {
+  KVPool<T> p;
+  p.base = (T*)c->kv_base; p.layer_stride = c->kv_layer_stride; p.kv_stride = c->kv_kv_stride;
+  p.head_stride = c->kv_head_stride; p.n_blocks = (int32_t)c->lim.kv_pool_blocks; p.head_dim = c->shape.head_dim;
+  return p;
+}
+
+// C = A W^T with the chosen epilogue.  impl: 0 auto, 1 CUDA cores, 2 tcgen05.
+template <typename T>
+static int gemm(rpo_ctx* c, const T* A, const T* W, void* C, int M, int N, int K, int epi, int impl = 0) {
+  if (M <= 0) return RPO_OK;
+  if (impl != 1 && tc_gemm_supported<T>(c, M, N, K) && (impl == 2 || c->use_tcgen05))
+    return tc_gemm<T>(c, A, W, C, M, N, K, epi);
+  if (impl == 2) return RPO_ERR_SHAPE;
+  dim3 grid(ceil_div(N, 64), ceil_div(M, 64));
+  if (epi == EPI_STORE_T) LAUNCH(c, (gemm_ref_kernel<T, EPI_STORE_T>), grid, 256, 0, A, W, C, M, N, K, (int64_t)N);
+  else if (epi == EPI_STORE_F32) LAUNCH(c, (gemm_ref_kernel<T, EPI_STORE_F32>), grid, 256, 0, A, W, C, M, N, K, (int64_t)N);
+  else LAUNCH(c, (gemm_ref_kernel<T, EPI_ADD_F32>), grid, 256, 0, A, W, C, M, N, K, (int64_t)N);
+  return RPO_OK;
+}
+
+template <typename T>
+static int rmsnorm(rpo_ctx* c, float* x, const float* g, T* h, int rows) {
+  if (rows <= 0) return RPO_OK;
+  const int d = c->shape.d_model;
+  LAUNCH(c, rmsnorm_kernel<T>, rows, 256, (size_t)d * 4, x, g, h, rows, d, c->shape.rms_eps, (const float*)nullptr, 0,
+         (int64_t)0);
+  return RPO_OK;
+}
+
+template <typename T>
+static int attention(rpo_ctx* c, int layer, int rows) {
+  const rpo_shape& s = c->shape;
+  Workspace& w = c->ws;
+  const float scale = 1.0f / sqrtf((float)s.head_dim);
+  const int grid = ceil_div((int64_t)rows * s.n_q_heads, 4);
+  if (s.head_dim == 64)
+    LAUNCH(c, (attn_ref_kernel<T, 64>), grid, 128, 0, (const T*)w.qkv, (T*)w.attn, w.row_seq, w.row_t,
+           (const SeqDesc*)w.seqs, c->d_block_table, kv_pool<T>(c), layer, rows, s.n_q_heads, s.n_kv_heads, scale,
+           c->d_status);
+  else
+    LAUNCH(c, (attn_ref_kernel<T, 128>), grid, 128, 0, (const T*)w.qkv, (T*)w.attn, w.row_seq, w.row_t,
+           (const SeqDesc*)w.seqs, c->d_block_table, kv_pool<T>(c), layer, rows, s.n_q_heads, s.n_kv_heads, scale,
+           c->d_status);
+  return RPO_OK;
+}
+
+// The layer stack over `rows` rows of ws.x, whose (sequence, private index) metadata sits in
+// ws.row_seq / ws.row_t and whose sequence descriptors sit in ws.seqs.
+template <typename T>
+static int run_layers(rpo_ctx* c, int rows) {
+  const rpo_shape& s = c->shape;
+  Workspace& w = c->ws;
+  const int d = s.d_model, F = s.d_ffn, qo = s.n_q_heads * s.head_dim;
+  for (int l = 0; l < s.n_layers; ++l) {
+    const LayerWeights& L = c->layers[l];
+    RPO_TRY(rmsnorm<T>(c, w.x, L.g1, (T*)w.h, rows));
+    RPO_TRY(gemm<T>(c, (const T*)w.h, (const T*)L.wqkv, w.qkv, rows, c->qkv_cols, d, EPI_STORE_T));
+    LAUNCH(c, rope_kv_kernel<T>, dim3(rows, s.n_q_heads + 2 * s.n_kv_heads), 64, 0, (T*)w.qkv, w.row_seq, w.row_t,
+           (const SeqDesc*)w.seqs, c->d_block_table, (const float2*)c->d_rope, kv_pool<T>(c), l, rows, s.n_q_heads,
+           s.n_kv_heads, c->lim.max_positions, c->d_status);
+    RPO_TRY(attention<T>(c, l, rows));
+    RPO_TRY(gemm<T>(c, (const T*)w.attn, (const T*)L.wo, w.x, rows, d, qo, EPI_ADD_F32));
+    RPO_TRY(rmsnorm<T>(c, w.x, L.g2, (T*)w.h, rows));
+    RPO_TRY(gemm<T>(c, (const T*)w.h, (const T*)L.wgu, w.gu, rows, 2 * F, d, EPI_STORE_T));
+    LAUNCH(c, swiglu_kernel<T>, grid_for((int64_t)rows * F, 256), 256, 0, (const T*)w.gu, (T*)w.act, (int64_t)rows * F);
+    RPO_TRY(gemm<T>(c, (const T*)w.act, (const T*)L.wd, w.x, rows, d, F, EPI_ADD_F32));
+  }
+  return RPO_OK;
+}
+
+// logits[n, V] (float32, ws.logits) from n residual rows in ws.xh.
+template <typename T>
+static int head(rpo_ctx* c, int n) {
+  Workspace& w = c->ws;
+  RPO_TRY(rmsnorm<T>(c, w.xh, c->gf, (T*)w.hh, n));
+  return gemm<T>(c, (const T*)w.hh, (const T*)c->lm_head, w.logits, n, c->shape.vocab, c->shape.d_model, EPI_STORE_F32);
+}
+
+static int take_blocks(rpo_ctx* c, int n, std::vector<int32_t>& out) {
+  if ((int64_t)c->free_blocks.size() < n) return RPO_ERR_KV_POOL;
+  for (int i = 0; i < n; ++i) { out.push_back(c->free_blocks.back()); c->free_blocks.pop_back(); }
+  return RPO_OK;
+}
+static void give_blocks(rpo_ctx* c, std::vector<int32_t>& b) {
+  for (auto it = b.rbegin(); it != b.rend(); ++it) c->free_blocks.push_back(*it);
+  b.clear();
+}
+
+static int check_groups(rpo_ctx* c, int n_groups, const rpo_group* g) {
+  for (int i = 0; i < n_groups; ++i) {
+    if (g[i].slot < 0 || g[i].slot >= c->lim.max_groups) return RPO_ERR_NOT_INITIALISED;
+    const GroupState& gs = c->groups[g[i].slot];
+    if (!gs.live || gs.group_id != g[i].group_id || gs.prefix_len != g[i].prefix_len) return RPO_ERR_NOT_INITIALISED;
+  }
+  return RPO_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// prefill
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+static int prefill_chunk(rpo_ctx* c, const int32_t* d_tokens, int tok0, const std::vector<int>& slots,
+                         const std::vector<int>& lens) {
+  Workspace& w = c->ws;
+  const int n = (int)slots.size();
+  int rows = 0;
+  for (int l : lens) rows += l;
+  std::vector<int32_t> row_seq(rows), row_t(rows), last(n);
+  std::vector<SeqDesc> sd(n);
+  int r = 0;
+  for (int i = 0; i < n; ++i) {
+    sd[i].shared_tbl = -1; sd[i].shared_len = 0; sd[i].priv_tbl = slots[i] * c->tbl_stride; sd[i].reserved = 0;
+    for (int t = 0; t < lens[i]; ++t, ++r) { row_seq[r] = i; row_t[r] = t; }
+    last[i] = r - 1;
+    const GroupState& gs = c->groups[slots[i]];
+    CUDA_TRY(cudaMemcpyAsync(c->d_block_table + (size_t)slots[i] * c->tbl_stride, gs.blocks.data(),
+                             gs.blocks.size() * 4, cudaMemcpyHostToDevice, c->stream));
+  }
+  CUDA_TRY(cudaMemcpyAsync(w.row_seq, row_seq.data(), (size_t)rows * 4, cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(cudaMemcpyAsync(w.row_t, row_t.data(), (size_t)rows * 4, cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(cudaMemcpyAsync(w.seqs, sd.data(), (size_t)n * sizeof(SeqDesc), cudaMemcpyHostToDevice, c->stream));
+  LAUNCH(c, embed_kernel<T>, rows, 128, 0, d_tokens + tok0, (const T*)c->embed, w.x, rows, c->shape.d_model,
+         c->shape.vocab, c->d_status);
+  RPO_TRY(run_layers<T>(c, rows));
+  // keep the residual stream of every group's last prefix token: step-0 logits come from it
+  for (int i = 0; i < n; ++i)
+    CUDA_TRY(cudaMemcpyAsync(c->d_x_last + (size_t)slots[i] * c->shape.d_model, w.x + (size_t)last[i] * c->shape.d_model,
+                             (size_t)c->shape.d_model * 4, cudaMemcpyDeviceToDevice, c->stream));
+  return RPO_OK;
+}
+
+extern "C" int rpo_prefill_prefix(rpo_ctx* c, int32_t n_groups, const int32_t* d_tokens, const int32_t* h_offsets,
+                                  const int32_t* h_group_ids, rpo_group* h_groups_out) {
+  if (!c || n_groups < 0 || (n_groups > 0 && (!d_tokens || !h_offsets || !h_groups_out))) return RPO_ERR_INVALID_ARG;
+  if (!c->weights_ready) return RPO_ERR_NOT_INITIALISED;
+  int64_t need_blocks = 0;
+  for (int g = 0; g < n_groups; ++g) {
+    const int len = h_offsets[g + 1] - h_offsets[g];
+    if (len < 1) return RPO_ERR_INVALID_ARG;
+    if (len > c->lim.max_chunk_tokens || len >= c->lim.max_positions) return RPO_ERR_LIMIT;
+    need_blocks += ceil_div(len, KV_BLOCK);
+  }
+  if (need_blocks > (int64_t)c->free_blocks.size() || n_groups > (int)c->free_slots.size()) return RPO_ERR_KV_POOL;
+  std::vector<int> slots(n_groups), lens(n_groups);
+  for (int g = 0; g < n_groups; ++g) {
+    const int slot = c->free_slots.back();
+    c->free_slots.pop_back();
+    GroupState& gs = c->groups[slot];
+    gs.live = true; gs.group_id = h_group_ids ? h_group_ids[g] : g; gs.prefix_len = h_offsets[g + 1] - h_offsets[g];
+    gs.blocks.clear();
+    take_blocks(c, ceil_div(gs.prefix_len, KV_BLOCK), gs.blocks);
+    slots[g] = slot; lens[g] = gs.prefix_len;
+    h_groups_out[g].group_id = gs.group_id; h_groups_out[g].prefix_len = gs.prefix_len;
+    h_groups_out[g].slot = slot; h_groups_out[g].n_blocks = (int32_t)gs.blocks.size();
+  }
+  int rc = RPO_OK;
+  int g0 = 0;
+  while (g0 < n_groups && rc == RPO_OK) {
+    int g1 = g0, rows = 0;
+    while (g1 < n_groups && rows + lens[g1] <= c->lim.max_chunk_tokens) rows += lens[g1++];
+    std::vector<int> cs(slots.begin() + g0, slots.begin() + g1), cl(lens.begin() + g0, lens.begin() + g1);
+    rc = c->bf16 ? prefill_chunk<bf16>(c, d_tokens, h_offsets[g0], cs, cl)
+                 : prefill_chunk<float>(c, d_tokens, h_offsets[g0], cs, cl);
+    g0 = g1;
+  }
+  if (rc != RPO_OK) rpo_release_groups(c, n_groups, h_groups_out);
+  return rc;
+}
+
+extern "C" int rpo_release_groups(rpo_ctx* c, int32_t n_groups, const rpo_group* g) {
+  if (!c || n_groups < 0 || (n_groups > 0 && !g)) return RPO_ERR_INVALID_ARG;
+  int rc = RPO_OK;
+  for (int i = 0; i < n_groups; ++i) {
+    if (g[i].slot < 0 || g[i].slot >= c->lim.max_groups || !c->groups[g[i].slot].live) { rc = RPO_ERR_NOT_INITIALISED; continue; }
+    GroupState& gs = c->groups[g[i].slot];
+    give_blocks(c, gs.blocks);
+    gs.live = false;
+    c->free_slots.push_back(g[i].slot);
+  }
+  return rc;
+}
+
+// ---------------------------------------------------------------------------------------------
+// decode
+// ---------------------------------------------------------------------------------------------
+static SamplerArgs sampler_args(rpo_ctx* c, const rpo_sampler* sp) {
+  SamplerArgs a;
+  memset(&a, 0, sizeof(a));
+  a.V = c->shape.vocab;
+  a.temperature = sp->temperature;
+  a.top_p24 = (uint32_t)floorf(sp->top_p * 16777216.0f);
+  a.greedy = sp->greedy; a.eos_id = sp->eos_id; a.seed = sp->seed;
+  return a;
+}
+
+static int check_sampler(const rpo_sampler* sp) {
+  if (!sp || !(sp->temperature > 0.f) || !(sp->top_p >= 0.f && sp->top_p <= 1.f)) return RPO_ERR_INVALID_ARG;
+  return RPO_OK;
+}
+
+template <typename T>
+static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, int S, const rpo_sampler* sp,
+                    const int32_t* d_forced, int32_t* d_tokens_out, int32_t* d_lens_out, float* d_logprobs_out,
+                    float* d_logits_dbg, std::vector<int32_t>& priv_blocks) {
+  Workspace& w = c->ws;
+  const int B = n_groups * G, d = c->shape.d_model;
+  const int per_seq = ceil_div(std::max(S - 1, 0), KV_BLOCK);
+  RPO_TRY(take_blocks(c, B * per_seq, priv_blocks));
+  std::vector<SeqDesc> sd(B);
+  std::vector<int32_t> tbl((size_t)B * c->tbl_stride, -1), logit_row(B), slot_idx(n_groups), zero(B, 0), seq_of_row(B);
+  std::vector<int64_t> seq_ids(B);
+  for (int g = 0; g < n_groups; ++g) {
+    slot_idx[g] = groups[g].slot;
+    for (int i = 0; i < G; ++i) {
+      const int b = g * G + i;
+      sd[b].shared_tbl = groups[g].slot * c->tbl_stride; sd[b].shared_len = groups[g].prefix_len;
+      sd[b].priv_tbl = (c->lim.max_groups + b) * c->tbl_stride; sd[b].reserved = 0;
+      for (int k = 0; k < per_seq; ++k) tbl[(size_t)b * c->tbl_stride + k] = priv_blocks[(size_t)b * per_seq + k];
+      logit_row[b] = g; seq_of_row[b] = b;
+      seq_ids[b] = (int64_t)groups[g].group_id * G + i;
+    }
+  }
+  cudaStream_t st = c->stream;
+  CUDA_TRY(cudaMemcpyAsync(w.seqs, sd.data(), (size_t)B * sizeof(SeqDesc), cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemcpyAsync(c->d_block_table + (size_t)c->lim.max_groups * c->tbl_stride, tbl.data(), tbl.size() * 4,
+                           cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemcpyAsync(w.logit_row, logit_row.data(), (size_t)B * 4, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemcpyAsync(w.slot_idx, slot_idx.data(), (size_t)n_groups * 4, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemcpyAsync(w.row_seq, seq_of_row.data(), (size_t)B * 4, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemcpyAsync(w.seq_ids, seq_ids.data(), (size_t)B * 8, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemsetAsync(w.done, 0, (size_t)B * 4, st));
+  CUDA_TRY(cudaMemsetAsync(w.lens, 0, (size_t)B * 4, st));
+  CUDA_TRY(cudaMemsetAsync(w.row_t, 0xFF, (size_t)B * 4, st));
+
+  SamplerArgs a = sampler_args(c, sp);
+  a.seq_ids = w.seq_ids; a.out_stride = S; a.forced = d_forced; a.tokens_out = d_tokens_out;
+  a.logprobs_out = d_logprobs_out; a.done = w.done; a.lens = w.lens; a.cur_tok = w.cur_tok; a.row_t = w.row_t;
+  a.logits_dbg = d_logits_dbg; a.logits = w.logits;
+
+  // step 0: the G samples of a group draw from the logits of the group's last prefix token
+  LAUNCH(c, gather_rows_f32_kernel, n_groups, 128, 0, (const float*)c->d_x_last, (const int32_t*)w.slot_idx, w.xh,
+         n_groups, d);
+  RPO_TRY(head<T>(c, n_groups));
+  a.logit_row = w.logit_row; a.step = 0; a.out_col = 0; a.last_step = (S == 1);
+  LAUNCH(c, sampler_kernel, B, 1024, 0, a);
+  a.logit_row = nullptr;
+  for (int j = 1; j < S; ++j) {
+    LAUNCH(c, embed_kernel<T>, B, 128, 0, (const int32_t*)w.cur_tok, (const T*)c->embed, w.x, B, d, c->shape.vocab,
+           c->d_status);
+    RPO_TRY(run_layers<T>(c, B));
+    CUDA_TRY(cudaMemcpyAsync(w.xh, w.x, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, st));
+    RPO_TRY(head<T>(c, B));
+    a.step = j; a.out_col = j; a.last_step = (j == S - 1);
+    LAUNCH(c, sampler_kernel, B, 1024, 0, a);
+  }
+  CUDA_TRY(cudaMemcpyAsync(d_lens_out, w.lens, (size_t)B * 4, cudaMemcpyDeviceToDevice, st));
+  return RPO_OK;
+}
+
+extern "C" int rpo_decode_suffix(rpo_ctx* c, int32_t n_groups, const rpo_group* h_groups, int32_t G, int32_t max_new,
+                                 const rpo_sampler* sp, const int32_t* d_forced, int32_t* d_tokens_out,
+                                 int32_t* d_lens_out, float* d_logprobs_out, float* d_logits_dbg) {
+  if (!c || n_groups <= 0 || !h_groups || G <= 0 || max_new <= 0 || !d_tokens_out || !d_lens_out) return RPO_ERR_INVALID_ARG;
+  RPO_TRY(check_sampler(sp));
+  if (!c->weights_ready) return RPO_ERR_NOT_INITIALISED;
+  RPO_TRY(check_groups(c, n_groups, h_groups));
+  if ((int64_t)n_groups * G > c->lim.max_seqs) return RPO_ERR_LIMIT;
+  for (int g = 0; g < n_groups; ++g)
+    if (h_groups[g].prefix_len + max_new > c->lim.max_positions) return RPO_ERR_LIMIT;
+  std::vector<int32_t> priv;
+  int rc = c->bf16 ? decode_t<bf16>(c, n_groups, h_groups, G, max_new, sp, d_forced, d_tokens_out, d_lens_out,
+                                    d_logprobs_out, d_logits_dbg, priv)
+                   : decode_t<float>(c, n_groups, h_groups, G, max_new, sp, d_forced, d_tokens_out, d_lens_out,
+                                     d_logprobs_out, d_logits_dbg, priv);
+  give_blocks(c, priv);   // stream order protects the blocks until the enqueued work is done
+  return rc;
+}
+
+// ---------------------------------------------------------------------------------------------
+// teacher-forced token log-probabilities
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+static int logprobs_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, int S, const int32_t* d_tokens,
+                      const int32_t* d_lens, float inv_T, float* d_out, float* d_logits_dbg) {
+  Workspace& w = c->ws;
+  const int B = n_groups * G, d = c->shape.d_model, V = c->shape.vocab;
+  const int in_rows = std::max(S - 1, 1);                       // layer-stack rows per sequence
+  const int seq_per_chunk = std::min(std::min(c->lim.max_chunk_tokens / in_rows, c->lim.max_seqs), B);
+  if (seq_per_chunk < 1) return RPO_ERR_LIMIT;
+  const int per_seq = ceil_div(std::max(S - 1, 0), KV_BLOCK);
+  cudaStream_t st = c->stream;
+  for (int s0 = 0; s0 < B; s0 += seq_per_chunk) {
+    const int ns = std::min(seq_per_chunk, B - s0);
+    std::vector<int32_t> priv;
+    RPO_TRY(take_blocks(c, ns * per_seq, priv));
+    std::vector<SeqDesc> sd(ns);
+    std::vector<int32_t> tbl((size_t)ns * c->tbl_stride, -1), slot_of_seq(ns);
+    for (int i = 0; i < ns; ++i) {
+      const rpo_group& g = groups[(s0 + i) / G];
+      sd[i].shared_tbl = g.slot * c->tbl_stride; sd[i].shared_len = g.prefix_len;
+      sd[i].priv_tbl = (c->lim.max_groups + i) * c->tbl_stride; sd[i].reserved = 0;
+      for (int k = 0; k < per_seq; ++k) tbl[(size_t)i * c->tbl_stride + k] = priv[(size_t)i * per_seq + k];
+      slot_of_seq[i] = g.slot;
+    }
+    int rc = RPO_OK;
+    do {
+      if (cudaMemcpyAsync(w.seqs, sd.data(), (size_t)ns * sizeof(SeqDesc), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+          cudaMemcpyAsync(c->d_block_table + (size_t)c->lim.max_groups * c->tbl_stride, tbl.data(), tbl.size() * 4,
+                          cudaMemcpyHostToDevice, st) != cudaSuccess ||
+          cudaMemcpyAsync(w.slot_idx, slot_of_seq.data(), (size_t)ns * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        rc = RPO_ERR_CUDA; break;
+      }
+      const int rows = ns * (S - 1);
+      if (rows > 0) {
+        build_teacher_rows_kernel<<<grid_for(rows, 256), 256, 0, st>>>(d_tokens, d_lens, s0, ns, S, w.row_seq, w.row_t,
+                                                                      w.row_tok);
+        c->launches++;
+        embed_kernel<T><<<rows, 128, 0, st>>>((const int32_t*)w.row_tok, (const T*)c->embed, w.x, rows, d, V, c->d_status);
+        c->launches++;
+        if ((rc = run_layers<T>(c, rows)) != RPO_OK) break;
+      }
+      const int head_rows = ns * S;
+      for (int r0 = 0; r0 < head_rows && rc == RPO_OK; r0 += w.HR) {
+        const int nr = std::min(w.HR, head_rows - r0);
+        gather_head_rows_kernel<<<nr, 128, 0, st>>>(w.x, c->d_x_last, w.slot_idx, r0, nr, S, d, w.xh);
+        c->launches++;
+        if ((rc = head<T>(c, nr)) != RPO_OK) break;
+        logprob_rows_kernel<<<nr, 512, 0, st>>>(w.logits, r0, nr, V, S, d_tokens, d_lens, s0, inv_T, d_out, d_logits_dbg);
+        c->launches++;
+      }
+      if (rc == RPO_OK && cudaGetLastError() != cudaSuccess) rc = RPO_ERR_CUDA;
+    } while (0);
+    give_blocks(c, priv);
+    if (rc != RPO_OK) return rc;
+  }
+  return RPO_OK;
+}
+
+extern "C" int rpo_token_logprobs(rpo_ctx* c, int32_t n_groups, const rpo_group* h_groups, int32_t G, int32_t max_new,
+                                  const int32_t* d_tokens, const int32_t* d_lens, float inv_temperature,
+                                  float* d_logprobs_out, float* d_logits_dbg) {
+  if (!c || n_groups <= 0 || !h_groups || G <= 0 || max_new <= 0 || !d_tokens || !d_lens || !d_logprobs_out ||
+      !(inv_temperature > 0.f))
+    return RPO_ERR_INVALID_ARG;
+  if (!c->weights_ready) return RPO_ERR_NOT_INITIALISED;
+  RPO_TRY(check_groups(c, n_groups, h_groups));
+  for (int g = 0; g < n_groups; ++g)
+    if (h_groups[g].prefix_len + max_new > c->lim.max_positions) return RPO_ERR_LIMIT;
+  return c->bf16 ? logprobs_t<bf16>(c, n_groups, h_groups, G, max_new, d_tokens, d_lens, inv_temperature,
+                                    d_logprobs_out, d_logits_dbg)
+                 : logprobs_t<float>(c, n_groups, h_groups, G, max_new, d_tokens, d_lens, inv_temperature,
+                                     d_logprobs_out, d_logits_dbg);
+}
+
+// ---------------------------------------------------------------------------------------------
+// whole rollout with host buffers
+// ---------------------------------------------------------------------------------------------
+extern "C" int rpo_rollout_host(rpo_ctx* c, int32_t n_groups, const int32_t* h_tokens, const int32_t* h_offsets,
+                                const int32_t* h_group_ids, int32_t G, int32_t max_new, const rpo_sampler* sp,
+                                int32_t* h_tokens_out, int32_t* h_lens_out, float* h_logprobs_out,
+                                int32_t want_policy, float* h_policy_out) {
+  if (!c || n_groups <= 0 || !h_tokens || !h_offsets || G <= 0 || max_new <= 0 || !h_tokens_out || !h_lens_out ||
+      (want_policy && !h_policy_out))
+    return RPO_ERR_INVALID_ARG;
+  RPO_TRY(check_sampler(sp));
+  const size_t n_tok = (size_t)h_offsets[n_groups], B = (size_t)n_groups * G, BS = B * max_new;
+  int32_t *d_tok = nullptr, *d_out = nullptr, *d_lens = nullptr;
+  float *d_lp = nullptr, *d_pol = nullptr;
+  std::vector<rpo_group> groups(n_groups);
+  int rc = RPO_OK;
+  bool prefilled = false;
+  do {
+    if (cudaMalloc(&d_tok, std::max<size_t>(n_tok, 1) * 4) != cudaSuccess || cudaMalloc(&d_out, BS * 4) != cudaSuccess ||
+        cudaMalloc(&d_lens, B * 4) != cudaSuccess || cudaMalloc(&d_lp, BS * 4) != cudaSuccess ||
+        (want_policy && cudaMalloc(&d_pol, BS * 4) != cudaSuccess)) { rc = RPO_ERR_CUDA; break; }
+    if (cudaMemcpyAsync(d_tok, h_tokens, n_tok * 4, cudaMemcpyHostToDevice, c->stream) != cudaSuccess) { rc = RPO_ERR_CUDA; break; }
+    if ((rc = rpo_prefill_prefix(c, n_groups, d_tok, h_offsets, h_group_ids, groups.data())) != RPO_OK) break;
+    prefilled = true;
+    if ((rc = rpo_decode_suffix(c, n_groups, groups.data(), G, max_new, sp, nullptr, d_out, d_lens, d_lp, nullptr)) != RPO_OK) break;
+    if (want_policy &&
+        (rc = rpo_token_logprobs(c, n_groups, groups.data(), G, max_new, d_out, d_lens, 1.0f / sp->temperature, d_pol,
+                                 nullptr)) != RPO_OK) break;
+    cudaMemcpyAsync(h_tokens_out, d_out, BS * 4, cudaMemcpyDeviceToHost, c->stream);
+    cudaMemcpyAsync(h_lens_out, d_lens, B * 4, cudaMemcpyDeviceToHost, c->stream);
+    if (h_logprobs_out) cudaMemcpyAsync(h_logprobs_out, d_lp, BS * 4, cudaMemcpyDeviceToHost, c->stream);
+    if (want_policy) cudaMemcpyAsync(h_policy_out, d_pol, BS * 4, cudaMemcpyDeviceToHost, c->stream);
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) rc = RPO_ERR_CUDA;
+  } while (0);
+  if (rc != RPO_OK) { cudaStreamSynchronize(c->stream); cudaGetLastError(); }
+  if (prefilled) rpo_release_groups(c, n_groups, groups.data());
+  cudaFree(d_tok); cudaFree(d_out); cudaFree(d_lens); cudaFree(d_lp); cudaFree(d_pol);
+  return rc;
+}
+
+// ---------------------------------------------------------------------------------------------
+// test / introspection entry points
+// ---------------------------------------------------------------------------------------------
+extern "C" int rpo_sample_rows(rpo_ctx* c, int32_t n_rows, int32_t vocab, const float* d_logits, const rpo_sampler* sp,
+                               const int64_t* d_seq_ids, int32_t step, int32_t* d_tokens_out, float* d_logprobs_out) {
+  if (!c || n_rows < 0 || vocab <= 0 || !d_logits || !d_seq_ids || !d_tokens_out || step < 0) return RPO_ERR_INVALID_ARG;
+  RPO_TRY(check_sampler(sp));
+  if (n_rows == 0) return RPO_OK;
+  SamplerArgs a = sampler_args(c, sp);
+  a.V = vocab; a.logits = d_logits; a.seq_ids = d_seq_ids; a.step = step; a.out_stride = 1; a.out_col = 0;
+  a.tokens_out = d_tokens_out; a.logprobs_out = d_logprobs_out; a.eos_id = -1;
+  LAUNCH(c, sampler_kernel, n_rows, 1024, 0, a);
+  return RPO_OK;
+}
+
+extern "C" int rpo_gemm(rpo_ctx* c, int32_t impl, int32_t M, int32_t N, int32_t K, const void* d_A, const void* d_W,
+                        float* d_C) {
+  if (!c || M < 0 || N <= 0 || K <= 0 || !d_A || !d_W || !d_C || impl < 0 || impl > 2) return RPO_ERR_INVALID_ARG;
+  return c->bf16 ? gemm<bf16>(c, (const bf16*)d_A, (const bf16*)d_W, d_C, M, N, K, EPI_STORE_F32, impl)
+                 : gemm<float>(c, (const float*)d_A, (const float*)d_W, d_C, M, N, K, EPI_STORE_F32, impl);
+}
+
+extern "C" int rpo_device_status(rpo_ctx* c, int32_t* out) {
+  if (!c || !out) return RPO_ERR_INVALID_ARG;
+  int v = 0;
+  CUDA_TRY(cudaMemcpyAsync(&v, c->d_status, 4, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(cudaStreamSynchronize(c->stream));
+  CUDA_TRY(cudaMemsetAsync(c->d_status, 0, 4, c->stream));
+  *out = v;
+  return RPO_OK;
+}
+
+extern "C" int rpo_counters(rpo_ctx* c, int64_t* launches, int64_t* free_blocks) {
+  if (!c) return RPO_ERR_INVALID_ARG;
+  if (launches) *launches = c->launches;
+  if (free_blocks) *free_blocks = (int64_t)c->free_blocks.size();
+  return RPO_OK;
+}
+
+extern "C" int rpo_set_option(rpo_ctx* c, const char* name, int32_t value) {
+  if (!c || !name) return RPO_ERR_INVALID_ARG;
+  if (!strcmp(name, "use_tcgen05")) c->use_tcgen05 = value;
+  else if (!strcmp(name, "use_tc_attention")) c->use_tc_attention = value;
+  else if (!strcmp(name, "use_graph")) c->use_graph = value;
+  else return RPO_ERR_INVALID_ARG;
+  return RPO_OK;
+}
