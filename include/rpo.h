@@ -196,8 +196,16 @@ int rpo_counters(rpo_ctx* ctx, int64_t* kernel_launches, int64_t* free_kv_blocks
 
 /* Runtime switches (tests/benchmarks): name = "use_tcgen05" (bf16 GEMMs on the tensor-core
  * kernel, default 1), "use_tc_attention" (tensor-core attention kernels, default 1),
- * "use_graph" (CUDA graph per decode step, default 1). */
+ * "use_graph" (CUDA graph per decode step, default 1), "profile" (see rpo_profile_read). */
 int rpo_set_option(rpo_ctx* ctx, const char* name, int32_t value);
+
+/* Per-kernel timing.  With option "profile" = 1 every kernel launch is bracketed by a pair of
+ * CUDA events on the context's stream (this serialises nothing but adds event overhead, and
+ * turns CUDA-graph replay off).  rpo_profile_read synchronises, sums the elapsed times and
+ * launch counts since the last read into ms_out / count_out [3 phases x 6 classes], index
+ * phase*6 + class; phases: 0 prefill, 1 decode, 2 token log-probs; classes: 0 other, 1 GEMM,
+ * 2 attention, 3 sampler, 4 RMSNorm, 5 RoPE + KV write.  n >= 18. */
+int rpo_profile_read(rpo_ctx* ctx, double* ms_out, int64_t* count_out, int32_t n);
 
 #ifdef __cplusplus
 }

@@ -14,7 +14,7 @@ _LIB = None
 EXPORTED_SYMBOLS = [
     "rpo_strerror", "rpo_shape_preset", "rpo_create", "rpo_destroy", "rpo_init_weights", "rpo_read_tensor",
     "rpo_write_tensor", "rpo_prefill_prefix", "rpo_decode_suffix", "rpo_token_logprobs", "rpo_release_groups",
-    "rpo_rollout_host", "rpo_sample_rows", "rpo_gemm", "rpo_device_status", "rpo_counters", "rpo_set_option",
+    "rpo_rollout_host", "rpo_sample_rows", "rpo_gemm", "rpo_device_status", "rpo_counters", "rpo_set_option", "rpo_profile_read",
 ]
 
 
@@ -75,6 +75,7 @@ def load_library(path=None):
     lib.rpo_device_status.argtypes = [vp, C.POINTER(i32)]
     lib.rpo_counters.argtypes = [vp, C.POINTER(i64), C.POINTER(i64)]
     lib.rpo_set_option.argtypes = [vp, C.c_char_p, i32]
+    lib.rpo_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64), i32]
     for name in EXPORTED_SYMBOLS:
         if name != "rpo_strerror":
             getattr(lib, name).restype = C.c_int
@@ -231,3 +232,14 @@ class Context:
 
     def set_option(self, name, value):
         _check(self.lib.rpo_set_option(self.handle, name.encode(), int(value)), f"rpo_set_option({name})")
+
+    PHASES = ("prefill", "decode", "logprobs")
+    CLASSES = ("other", "gemm", "attention", "sampler", "rmsnorm", "rope_kv")
+
+    def profile_read(self):
+        """{phase: {class: (total_ms, launches)}} since the last read (needs option profile=1)."""
+        n = len(self.PHASES) * len(self.CLASSES)
+        ms = (C.c_double * n)(); cnt = (C.c_int64 * n)()
+        _check(self.lib.rpo_profile_read(self.handle, ms, cnt, n), "rpo_profile_read")
+        return {p: {k: (ms[i * len(self.CLASSES) + j], cnt[i * len(self.CLASSES) + j])
+                    for j, k in enumerate(self.CLASSES)} for i, p in enumerate(self.PHASES)}

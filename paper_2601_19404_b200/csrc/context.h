@@ -82,6 +82,10 @@ struct rpo_ctx {
   int sm_count = 148;
   // options
   int use_tcgen05 = 1, use_tc_attention = 1, use_graph = 1;
+  // optional per-kernel timing: event pairs around every launch, tagged class + 16*phase
+  struct ProfEvent { cudaEvent_t a, b; int tag; };
+  int profile = 0, prof_class = 0, prof_phase = 0;
+  std::vector<ProfEvent> prof_events;
   // tcgen05 GEMM state (tensor maps are built per call; see gemm_tc.cuh)
   void* tc_state = nullptr;
 };

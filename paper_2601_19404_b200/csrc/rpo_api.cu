@@ -31,9 +31,32 @@ using namespace rpo;
     if (r_ != RPO_OK) return r_; \
   } while (0)
 
+// Kernel classes for the optional per-kernel timing (rpo_set_option "profile").
+enum KClass { KC_OTHER = 0, KC_GEMM = 1, KC_ATTN = 2, KC_SAMPLER = 3, KC_NORM = 4, KC_ROPE = 5, KC_COUNT = 6 };
+
+struct ProfScope {
+  rpo_ctx* c; int prev;
+  ProfScope(rpo_ctx* c_, int k) : c(c_), prev(c_->prof_class) { c->prof_class = k; }
+  ~ProfScope() { c->prof_class = prev; }
+};
+
+static void prof_begin(rpo_ctx* c) {
+  if (!c->profile) return;
+  cudaEvent_t a, b;
+  cudaEventCreate(&a); cudaEventCreate(&b);
+  cudaEventRecord(a, c->stream);
+  c->prof_events.push_back({a, b, c->prof_class + 16 * c->prof_phase});
+}
+static void prof_end(rpo_ctx* c) {
+  if (!c->profile) return;
+  cudaEventRecord(c->prof_events.back().b, c->stream);
+}
+
 #define LAUNCH(ctx, kern, grid, block, smem, ...)                         \
   do {                                                                    \
+    prof_begin(ctx);                                                      \
     kern<<<(grid), (block), (smem), (ctx)->stream>>>(__VA_ARGS__);        \
+    prof_end(ctx);                                                        \
     (ctx)->launches++;                                                    \
     CUDA_TRY(cudaGetLastError());                                         \
   } while (0)
@@ -293,6 +316,7 @@ static KVPool<T> kv_pool(rpo_ctx* c) {
 template <typename T>
 static int gemm(rpo_ctx* c, const T* A, const T* W, void* C, int M, int N, int K, int epi, int impl = 0) {
   if (M <= 0) return RPO_OK;
+  ProfScope ps(c, KC_GEMM);
   if (impl != 1 && tc_gemm_supported<T>(c, M, N, K) && (impl == 2 || c->use_tcgen05))
     return tc_gemm<T>(c, A, W, C, M, N, K, epi);
   if (impl == 2) return RPO_ERR_SHAPE;
@@ -306,6 +330,7 @@ static int gemm(rpo_ctx* c, const T* A, const T* W, void* C, int M, int N, int K
 template <typename T>
 static int rmsnorm(rpo_ctx* c, float* x, const float* g, T* h, int rows) {
   if (rows <= 0) return RPO_OK;
+  ProfScope ps(c, KC_NORM);
   const int d = c->shape.d_model;
   LAUNCH(c, rmsnorm_kernel<T>, rows, 256, (size_t)d * 4, x, g, h, rows, d, c->shape.rms_eps, (const float*)nullptr, 0,
          (int64_t)0);
@@ -317,6 +342,7 @@ static int attention(rpo_ctx* c, int layer, int rows) {
   const rpo_shape& s = c->shape;
   Workspace& w = c->ws;
   const float scale = 1.0f / sqrtf((float)s.head_dim);
+  ProfScope ps(c, KC_ATTN);
   const int grid = ceil_div((int64_t)rows * s.n_q_heads, 4);
   if (s.head_dim == 64)
     LAUNCH(c, (attn_ref_kernel<T, 64>), grid, 128, 0, (const T*)w.qkv, (T*)w.attn, w.row_seq, w.row_t,
@@ -340,9 +366,10 @@ static int run_layers(rpo_ctx* c, int rows) {
     const LayerWeights& L = c->layers[l];
     RPO_TRY(rmsnorm<T>(c, w.x, L.g1, (T*)w.h, rows));
     RPO_TRY(gemm<T>(c, (const T*)w.h, (const T*)L.wqkv, w.qkv, rows, c->qkv_cols, d, EPI_STORE_T));
+    { ProfScope ps(c, KC_ROPE);
     LAUNCH(c, rope_kv_kernel<T>, dim3(rows, s.n_q_heads + 2 * s.n_kv_heads), 64, 0, (T*)w.qkv, w.row_seq, w.row_t,
            (const SeqDesc*)w.seqs, c->d_block_table, (const float2*)c->d_rope, kv_pool<T>(c), l, rows, s.n_q_heads,
-           s.n_kv_heads, c->lim.max_positions, c->d_status);
+           s.n_kv_heads, c->lim.max_positions, c->d_status); }
     RPO_TRY(attention<T>(c, l, rows));
     RPO_TRY(gemm<T>(c, (const T*)w.attn, (const T*)L.wo, w.x, rows, d, qo, EPI_ADD_F32));
     RPO_TRY(rmsnorm<T>(c, w.x, L.g2, (T*)w.h, rows));
@@ -418,6 +445,7 @@ extern "C" int rpo_prefill_prefix(rpo_ctx* c, int32_t n_groups, const int32_t* d
                                   const int32_t* h_group_ids, rpo_group* h_groups_out) {
   if (!c || n_groups < 0 || (n_groups > 0 && (!d_tokens || !h_offsets || !h_groups_out))) return RPO_ERR_INVALID_ARG;
   if (!c->weights_ready) return RPO_ERR_NOT_INITIALISED;
+  c->prof_phase = 0;
   int64_t need_blocks = 0;
   for (int g = 0; g < n_groups; ++g) {
     const int len = h_offsets[g + 1] - h_offsets[g];
@@ -527,7 +555,7 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
          n_groups, d);
   RPO_TRY(head<T>(c, n_groups));
   a.logit_row = w.logit_row; a.step = 0; a.out_col = 0; a.last_step = (S == 1);
-  LAUNCH(c, sampler_kernel, B, 1024, 0, a);
+  { ProfScope ps(c, KC_SAMPLER); LAUNCH(c, sampler_kernel, B, 1024, 0, a); }
   a.logit_row = nullptr;
   for (int j = 1; j < S; ++j) {
     LAUNCH(c, embed_kernel<T>, B, 128, 0, (const int32_t*)w.cur_tok, (const T*)c->embed, w.x, B, d, c->shape.vocab,
@@ -536,7 +564,7 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
     CUDA_TRY(cudaMemcpyAsync(w.xh, w.x, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, st));
     RPO_TRY(head<T>(c, B));
     a.step = j; a.out_col = j; a.last_step = (j == S - 1);
-    LAUNCH(c, sampler_kernel, B, 1024, 0, a);
+    { ProfScope ps(c, KC_SAMPLER); LAUNCH(c, sampler_kernel, B, 1024, 0, a); }
   }
   CUDA_TRY(cudaMemcpyAsync(d_lens_out, w.lens, (size_t)B * 4, cudaMemcpyDeviceToDevice, st));
   return RPO_OK;
@@ -553,6 +581,7 @@ extern "C" int rpo_decode_suffix(rpo_ctx* c, int32_t n_groups, const rpo_group* 
   for (int g = 0; g < n_groups; ++g)
     if (h_groups[g].prefix_len + max_new > c->lim.max_positions) return RPO_ERR_LIMIT;
   std::vector<int32_t> priv;
+  c->prof_phase = 1;
   int rc = c->bf16 ? decode_t<bf16>(c, n_groups, h_groups, G, max_new, sp, d_forced, d_tokens_out, d_lens_out,
                                     d_logprobs_out, d_logits_dbg, priv)
                    : decode_t<float>(c, n_groups, h_groups, G, max_new, sp, d_forced, d_tokens_out, d_lens_out,
@@ -631,6 +660,7 @@ extern "C" int rpo_token_logprobs(rpo_ctx* c, int32_t n_groups, const rpo_group*
   RPO_TRY(check_groups(c, n_groups, h_groups));
   for (int g = 0; g < n_groups; ++g)
     if (h_groups[g].prefix_len + max_new > c->lim.max_positions) return RPO_ERR_LIMIT;
+  c->prof_phase = 2;
   return c->bf16 ? logprobs_t<bf16>(c, n_groups, h_groups, G, max_new, d_tokens, d_lens, inv_temperature,
                                     d_logprobs_out, d_logits_dbg)
                  : logprobs_t<float>(c, n_groups, h_groups, G, max_new, d_tokens, d_lens, inv_temperature,
@@ -721,6 +751,22 @@ extern "C" int rpo_set_option(rpo_ctx* c, const char* name, int32_t value) {
   if (!strcmp(name, "use_tcgen05")) c->use_tcgen05 = value;
   else if (!strcmp(name, "use_tc_attention")) c->use_tc_attention = value;
   else if (!strcmp(name, "use_graph")) c->use_graph = value;
+  else if (!strcmp(name, "profile")) c->profile = value;
   else return RPO_ERR_INVALID_ARG;
+  return RPO_OK;
+}
+
+extern "C" int rpo_profile_read(rpo_ctx* c, double* ms_out, int64_t* count_out, int32_t n) {
+  if (!c || !ms_out || !count_out || n < 3 * KC_COUNT) return RPO_ERR_INVALID_ARG;
+  CUDA_TRY(cudaStreamSynchronize(c->stream));
+  for (int i = 0; i < n; ++i) { ms_out[i] = 0.0; count_out[i] = 0; }
+  for (auto& ev : c->prof_events) {
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, ev.a, ev.b);
+    const int phase = ev.tag / 16, k = ev.tag % 16;
+    if (phase < 3 && k < KC_COUNT) { ms_out[phase * KC_COUNT + k] += ms; count_out[phase * KC_COUNT + k]++; }
+    cudaEventDestroy(ev.a); cudaEventDestroy(ev.b);
+  }
+  c->prof_events.clear();
   return RPO_OK;
 }
