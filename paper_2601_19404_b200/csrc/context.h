@@ -82,6 +82,7 @@ struct rpo_ctx {
   int sm_count = 148;
   // options
   int use_tcgen05 = 1, use_tc_attention = 1, use_graph = 1;
+  int pending_splits = 0, pending_rows = 0;   // split-K partials of ws.x not yet reduced
   // optional per-kernel timing: event pairs around every launch, tagged class + 16*phase
   struct ProfEvent { cudaEvent_t a, b; int tag; };
   int profile = 0, prof_class = 0, prof_phase = 0;

@@ -1,9 +1,418 @@
-// placeholder replaced below
+// bf16 GEMM on the 5th-generation tensor cores: C[M,N] = A[M,K] * W[N,K]^T, float32 accumulation.
+//
+//   * operands: TMA (cp.async.bulk.tensor.2d, no multicast) into 128-byte-swizzled shared memory,
+//     a ring of NS stages of [128 x 64] (A) and [BN x 64] (W) tiles guarded by mbarriers;
+//   * math: tcgen05.mma kind::f16 (bf16 x bf16 -> f32), M = 128, N = BN, K = 16 per instruction,
+//     issued by one thread; accumulators live in tensor memory, two buffers of BN columns so the
+//     epilogue of one tile overlaps the main loop of the next;
+//   * epilogue: four warps read their 32-lane quadrant with tcgen05.ld and apply one of
+//     {store bf16, store f32, add into the f32 residual stream, SwiGLU on interleaved gate/up
+//     columns, store f32 split-K partial};
+//   * persistent CTAs walk work items (tile_m, tile_n, k-split); split-K keeps all SMs streaming
+//     weights when M is a decode batch.  Partials are reduced in fixed order by the next kernel.
+//   * every mbarrier wait is bounded (clock64); on expiry the CTA raises STATUS_TIMEOUT, lets
+//     copies in flight land, frees its tensor memory and returns.
 #pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <map>
+#include <tuple>
+
+#include "common.cuh"
 #include "context.h"
+
 namespace rpo {
-inline int tc_create(rpo_ctx*) { return RPO_OK; }
-inline void tc_destroy(rpo_ctx*) {}
-template <typename T> inline bool tc_gemm_supported(rpo_ctx*, int, int, int) { return false; }
-template <typename T> inline int tc_gemm(rpo_ctx*, const T*, const T*, void*, int, int, int, int) { return RPO_ERR_SHAPE; }
+
+enum TcEpilogue { TC_STORE_BF16 = 0, TC_STORE_F32 = 1, TC_ADD_F32 = 2, TC_SWIGLU = 3, TC_PARTIAL = 4 };
+
+constexpr int TC_BM = 128, TC_BK = 64;
+constexpr long long TC_TIMEOUT_CYCLES = 4000000000LL;   // ~2 s at 2 GHz
+
+struct TcParams {
+  void* C;              // output (type by epilogue)
+  int M, N, K;
+  int ldc;              // elements per output row
+  int tiles_m, tiles_n, splits, kb_per_split, kb_total;
+  int64_t split_stride; // TC_PARTIAL: elements between split planes
+  int* status;
+};
+
+namespace tc {
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: false when the time limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (*abort_flag) return false;
+    if (clock64() - t0 > TC_TIMEOUT_CYCLES) { *abort_flag = 1; return false; }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y) : "memory");
+}
+
+// Shared-memory matrix descriptor, K-major operand, 128-byte swizzle: rows of 128 bytes, groups of
+// 8 rows 1024 bytes apart (SBO), descriptor version 1 (sm_100), layout type 2 (SWIZZLE_128B).
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
+  d |= (uint64_t)1 << 16;                 // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset
+  d |= (uint64_t)1 << 46;                 // version
+  d |= (uint64_t)2 << 61;                 // SWIZZLE_128B
+  return d;
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+}  // namespace tc
+
+template <int BN>
+struct TcCfg {
+  static constexpr int A_BYTES = TC_BM * TC_BK * 2;
+  static constexpr int B_BYTES = BN * TC_BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int NS = (200 * 1024 / STAGE_BYTES) > 8 ? 8 : (200 * 1024 / STAGE_BYTES);
+  static constexpr int TMEM_COLS = (2 * BN < 32) ? 32 : 2 * BN;
+  static constexpr int SMEM_BYTES = NS * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+};
+
+// 192 threads: warp 0 = TMA producer, warp 1 = MMA issuer (+ TMEM owner), warps 2..5 = epilogue.
+template <int BN, int EPI>
+__global__ void __launch_bounds__(192, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, TcParams p) {
+  using Cfg = TcCfg<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = (uint64_t*)(smem + Cfg::NS * Cfg::STAGE_BYTES);
+  uint64_t* full = bars;
+  uint64_t* empty = bars + Cfg::NS;
+  uint64_t* acc_full = bars + 2 * Cfg::NS;
+  uint64_t* acc_empty = bars + 2 * Cfg::NS + 2;
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * Cfg::NS + 4);
+  volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_items = p.tiles_m * p.tiles_n * p.splits;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < Cfg::NS; ++i) { tc::mbar_init(&full[i], 1); tc::mbar_init(&empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { tc::mbar_init(&acc_full[i], 1); tc::mbar_init(&acc_empty[i], 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc::smem_u32(tmem_slot)),
+                 "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc::tmem_fence_before();
+  __syncthreads();
+  tc::tmem_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+        const int split = it % p.splits, t = it / p.splits;
+        const int tn = t % p.tiles_n, tm = t / p.tiles_n;
+        const int kb0 = split * p.kb_per_split, kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!tc::mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+          uint8_t* sa = smem + stage * Cfg::STAGE_BYTES;
+          tc::mbar_expect_tx(&full[stage], Cfg::STAGE_BYTES);
+          tc::tma_load_2d(sa, &map_a, kb * TC_BK, tm * TC_BM, &full[stage]);
+          tc::tma_load_2d(sa + Cfg::A_BYTES, &map_w, kb * TC_BK, tn * BN, &full[stage]);
+          if (++stage == Cfg::NS) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+      int stage = 0; uint32_t phase = 0;
+      int acc = 0; uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+        const int split = it % p.splits;
+        const int kb0 = split * p.kb_per_split, kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+        if (!tc::mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag)) { ok = false; break; }
+        tc::tmem_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!tc::mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+          tc::tmem_fence_after();
+          const uint32_t sa = tc::smem_u32(smem + stage * Cfg::STAGE_BYTES);
+          const uint64_t da = tc::umma_desc_sw128(sa), db = tc::umma_desc_sw128(sa + Cfg::A_BYTES);
+#pragma unroll
+          for (int k = 0; k < TC_BK / 16; ++k)   // +32 bytes per K=16 step inside the 128-byte swizzled row
+            tc::umma_bf16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          tc::umma_commit(&empty[stage]);            // frees the stage once these MMAs have read it
+          if (++stage == Cfg::NS) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        tc::umma_commit(&acc_full[acc]);             // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int quad = warp & 3;                       // TMEM lane quadrant this warp may read
+    int acc = 0; uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+      const int split = it % p.splits, t = it / p.splits;
+      const int tn = t % p.tiles_n, tm = t / p.tiles_n;
+      if (!tc::mbar_wait(&acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+      tc::tmem_fence_after();
+      const int row = tm * TC_BM + quad * 32 + lane;
+      const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN);
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        uint32_t r[32];
+        tc::tmem_ld32(t_row + (uint32_t)c0, r);
+        const int col = tn * BN + c0;
+        if (row < p.M && col < p.N) {
+          const int ncol = min(32, p.N - col);       // multiple of 8 (N % 8 == 0)
+          if (EPI == TC_STORE_BF16) {
+            bf16* dst = (bf16*)p.C + (int64_t)row * p.ldc + col;
+            for (int j = 0; j < ncol; j += 8) {
+              uint4 v;
+              __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+              __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]));
+              __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
+              v.x = *(uint32_t*)&h0; v.y = *(uint32_t*)&h1; v.z = *(uint32_t*)&h2; v.w = *(uint32_t*)&h3;
+              *(uint4*)(dst + j) = v;
+            }
+          } else if (EPI == TC_SWIGLU) {
+            // columns (2j, 2j+1) = (gate_j, up_j)  ->  out[row, col/2 + j]
+            bf16* dst = (bf16*)p.C + (int64_t)row * p.ldc + col / 2;
+            for (int j = 0; j < ncol; j += 16) {
+              uint32_t o[4];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const float g0 = __uint_as_float(r[j + 4 * q]), u0 = __uint_as_float(r[j + 4 * q + 1]);
+                const float g1 = __uint_as_float(r[j + 4 * q + 2]), u1 = __uint_as_float(r[j + 4 * q + 3]);
+                __nv_bfloat162 h = __floats2bfloat162_rn(g0 / (1.0f + __expf(-g0)) * u0, g1 / (1.0f + __expf(-g1)) * u1);
+                o[q] = *(uint32_t*)&h;
+              }
+              *(uint4*)(dst + j / 2) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+          } else {
+            float* dst = (EPI == TC_PARTIAL) ? (float*)p.C + split * p.split_stride + (int64_t)row * p.ldc + col
+                                             : (float*)p.C + (int64_t)row * p.ldc + col;
+            for (int j = 0; j < ncol; j += 4) {
+              float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
+                                     __uint_as_float(r[j + 3]));
+              if (EPI == TC_ADD_F32) {
+                const float4 o = *(float4*)(dst + j);
+                v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+              }
+              *(float4*)(dst + j) = v;
+            }
+          }
+        }
+      }
+      tc::tmem_fence_before();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(&acc_empty[acc]);
+      if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+    }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  __syncwarp();
+  tc::tmem_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) atomicOr(p.status, STATUS_TIMEOUT);
+    for (int i = 0; i < 64; ++i) __nanosleep(1000000);   // let bulk copies in flight land before smem goes away
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc::tmem_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TcState {
+  EncodeTiledFn encode = nullptr;
+  std::map<std::tuple<const void*, int, int, int>, CUtensorMap> maps;   // (ptr, rows, cols, box_rows)
+  bool attrs_set = false;
+};
+
+inline int tc_create(rpo_ctx* c) {
+  TcState* s = new TcState();
+  c->tc_state = s;
+  if (!c->bf16) return RPO_OK;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+      q != cudaDriverEntryPointSuccess || !fn) {
+    cudaGetLastError();
+    fprintf(stderr, "[rpo] cuTensorMapEncodeTiled unavailable: tensor-core GEMM disabled\n");
+    return RPO_OK;
+  }
+  s->encode = (EncodeTiledFn)fn;
+  return RPO_OK;
+}
+inline void tc_destroy(rpo_ctx* c) { delete (TcState*)c->tc_state; c->tc_state = nullptr; }
+
+// Row-major bf16 [rows, cols] with a [box_rows x 64] box, 128-byte swizzle, zero fill out of bounds.
+inline const CUtensorMap* tc_map(rpo_ctx* c, const void* ptr, int rows, int cols, int box_rows) {
+  TcState* s = (TcState*)c->tc_state;
+  auto key = std::make_tuple(ptr, rows, cols, box_rows);
+  auto it = s->maps.find(key);
+  if (it != s->maps.end()) return &it->second;
+  CUtensorMap m;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  CUresult r = s->encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { fprintf(stderr, "[rpo] cuTensorMapEncodeTiled failed (%d)\n", (int)r); return nullptr; }
+  if (s->maps.size() > 4096) s->maps.clear();
+  return &(s->maps[key] = m);
+}
+
+template <typename T>
+inline bool tc_gemm_supported(rpo_ctx* c, int M, int N, int K) { return false; }
+template <>
+inline bool tc_gemm_supported<bf16>(rpo_ctx* c, int M, int N, int K) {
+  TcState* s = (TcState*)c->tc_state;
+  return s && s->encode && M >= 1 && (K % TC_BK) == 0 && (N % 16) == 0;
+}
+
+template <int BN, int EPI>
+inline int tc_launch(rpo_ctx* c, const CUtensorMap* ma, const CUtensorMap* mw, const TcParams& p, int grid) {
+  using Cfg = TcCfg<BN>;
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
+      return RPO_ERR_CUDA;
+    attr_done = true;
+  }
+  gemm_tc_kernel<BN, EPI><<<grid, 192, Cfg::SMEM_BYTES, c->stream>>>(*ma, *mw, p);
+  return cudaGetLastError() == cudaSuccess ? RPO_OK : RPO_ERR_CUDA;
+}
+
+template <int BN>
+inline int tc_launch_epi(rpo_ctx* c, int epi, const CUtensorMap* ma, const CUtensorMap* mw, const TcParams& p, int grid) {
+  switch (epi) {
+    case TC_STORE_BF16: return tc_launch<BN, TC_STORE_BF16>(c, ma, mw, p, grid);
+    case TC_STORE_F32: return tc_launch<BN, TC_STORE_F32>(c, ma, mw, p, grid);
+    case TC_ADD_F32: return tc_launch<BN, TC_ADD_F32>(c, ma, mw, p, grid);
+    case TC_SWIGLU: return tc_launch<BN, TC_SWIGLU>(c, ma, mw, p, grid);
+    default: return tc_launch<BN, TC_PARTIAL>(c, ma, mw, p, grid);
+  }
+}
+
+// Plan and launch.  `splits_out` (optional) receives the number of split-K planes written to
+// ws.partial when the epilogue had to become TC_PARTIAL (only for TC_ADD_F32 requests with
+// allow_split): the caller then owns the reduction.
+inline int tc_gemm_launch(rpo_ctx* c, const bf16* A, const bf16* W, void* C, int M, int N, int K, int epi, int ldc,
+                          bool allow_split, int* splits_out) {
+  if (splits_out) *splits_out = 0;
+  const int tiles_m = (M + TC_BM - 1) / TC_BM;
+  const int kb_total = K / TC_BK;
+  const int sms = c->sm_count;
+  // tile width: widest tile that still yields about one wave of CTAs
+  int bn = 256;
+  if (epi == TC_SWIGLU && bn > 128 && tiles_m * ((N + 255) / 256) < sms) bn = 128;
+  while (bn > 32 && tiles_m * ((N + bn - 1) / bn) < sms) bn >>= 1;
+  if (bn > 64 && tiles_m * ((N + bn - 1) / bn) < 2 * sms && tiles_m * ((N + bn / 2 - 1) / (bn / 2)) <= sms) bn >>= 1;
+  int tiles_n = (N + bn - 1) / bn;
+  int splits = 1;
+  if (allow_split && epi == TC_ADD_F32) {
+    const int tiles = tiles_m * tiles_n;
+    if (tiles < sms) {
+      splits = std::min(std::max(1, sms / tiles), std::max(1, kb_total / 4));
+      while (splits > 1 && (size_t)splits * M * N > c->ws.partial_elems) --splits;
+    }
+  }
+  const int kb_per_split = (kb_total + splits - 1) / splits;
+  splits = (kb_total + kb_per_split - 1) / kb_per_split;
+  TcParams p;
+  p.C = C; p.M = M; p.N = N; p.K = K; p.ldc = ldc;
+  p.tiles_m = tiles_m; p.tiles_n = tiles_n; p.splits = splits; p.kb_per_split = kb_per_split; p.kb_total = kb_total;
+  p.split_stride = (int64_t)M * N; p.status = c->d_status;
+  int use_epi = epi;
+  if (splits > 1) { use_epi = TC_PARTIAL; p.C = c->ws.partial; p.ldc = N; if (splits_out) *splits_out = splits; }
+  const CUtensorMap* ma = tc_map(c, A, M, K, TC_BM);
+  const CUtensorMap* mw = tc_map(c, W, N, K, bn);
+  if (!ma || !mw) return RPO_ERR_CUDA;
+  const int grid = std::min(tiles_m * tiles_n * splits, sms);
+  switch (bn) {
+    case 256: return tc_launch_epi<256>(c, use_epi, ma, mw, p, grid);
+    case 128: return tc_launch_epi<128>(c, use_epi, ma, mw, p, grid);
+    case 64: return tc_launch_epi<64>(c, use_epi, ma, mw, p, grid);
+    default: return tc_launch_epi<32>(c, use_epi, ma, mw, p, grid);
+  }
+}
+
+template <typename T>
+inline int tc_gemm(rpo_ctx*, const T*, const T*, void*, int, int, int, int) { return RPO_ERR_SHAPE; }
+
+}  // namespace rpo

@@ -143,6 +143,19 @@ __global__ void rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ 
   for (int i = threadIdx.x; i < d; i += blockDim.x) hr[i] = from_f32<T>(srow[i] * inv * gain[i]);
 }
 
+// x[i] += sum_s partial[s*stride + i], fixed order (deterministic split-K reduction). n % 4 == 0.
+__global__ void reduce_partials_kernel(float* __restrict__ x, const float* __restrict__ partial, int n_splits, int64_t n,
+                                       int64_t stride) {
+  for (int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4; i < n; i += (int64_t)gridDim.x * blockDim.x * 4) {
+    float4 v = *(const float4*)(x + i);
+    for (int s = 0; s < n_splits; ++s) {
+      const float4 q = *(const float4*)(partial + s * stride + i);
+      v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
+    }
+    *(float4*)(x + i) = v;
+  }
+}
+
 // RoPE (rotate-half) on q and k, then K/V written to the row's slot of its private segment.
 // qkv row layout: [q heads | k heads | v heads] x head_dim.  Grid: (rows, Hq + 2*Hkv).
 template <typename T>

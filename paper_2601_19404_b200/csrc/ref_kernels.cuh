@@ -6,7 +6,7 @@
 
 namespace rpo {
 
-enum GemmEpilogue { EPI_STORE_T = 0, EPI_STORE_F32 = 1, EPI_ADD_F32 = 2 };
+enum GemmEpilogue { EPI_STORE_T = 0, EPI_STORE_F32 = 1, EPI_ADD_F32 = 2, EPI_SWIGLU = 3 };
 
 // C[M,N] (+)= A[M,K] * W[N,K]^T.  64x64 tile, 16-deep K slices, 4x4 outputs per thread.
 template <typename T, int EPI>

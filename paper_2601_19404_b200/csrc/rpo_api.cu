@@ -235,6 +235,8 @@ extern "C" int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limit
   ALLOC(w.logit_row, (size_t)nseq * 4);
   ALLOC(w.slot_idx, (size_t)nseq * 4);
   ALLOC(w.seq_ids, (size_t)nseq * 8);
+  w.partial_elems = (size_t)c->sm_count * 128 * 256;
+  ALLOC(w.partial, w.partial_elems * 4);
   if (rc == RPO_OK) rc = tc_create(c);
 #undef ALLOC
   if (rc != RPO_OK) { rpo_destroy(c); return rc; }
@@ -312,14 +314,37 @@ static KVPool<T> kv_pool(rpo_ctx* c) {
   return p;
 }
 
+// Split-K partial sums of the last residual-add GEMM wait in ws.partial until the next RMSNorm
+// (which folds the reduction in) or an explicit flush.
+static int flush_partials(rpo_ctx* c) {
+  if (c->pending_splits == 0) return RPO_OK;
+  const int64_t n = (int64_t)c->pending_rows * c->shape.d_model;
+  LAUNCH(c, reduce_partials_kernel, grid_for(n / 4, 256), 256, 0, c->ws.x, (const float*)c->ws.partial, c->pending_splits,
+         n, n);
+  c->pending_splits = 0;
+  return RPO_OK;
+}
+
 // C = A W^T with the chosen epilogue.  impl: 0 auto, 1 CUDA cores, 2 tcgen05.
+// EPI_SWIGLU is only valid on the tensor-core path (callers check tc_gemm_supported first).
 template <typename T>
-static int gemm(rpo_ctx* c, const T* A, const T* W, void* C, int M, int N, int K, int epi, int impl = 0) {
+static int gemm(rpo_ctx* c, const T* A, const T* W, void* C, int M, int N, int K, int epi, int impl = 0,
+                bool allow_split = false) {
   if (M <= 0) return RPO_OK;
   ProfScope ps(c, KC_GEMM);
-  if (impl != 1 && tc_gemm_supported<T>(c, M, N, K) && (impl == 2 || c->use_tcgen05))
-    return tc_gemm<T>(c, A, W, C, M, N, K, epi);
-  if (impl == 2) return RPO_ERR_SHAPE;
+  if (impl != 1 && tc_gemm_supported<T>(c, M, N, K) && (impl == 2 || c->use_tcgen05)) {
+    const int tc_epi = epi == EPI_STORE_T ? TC_STORE_BF16 : epi == EPI_STORE_F32 ? TC_STORE_F32
+                     : epi == EPI_ADD_F32 ? TC_ADD_F32 : TC_SWIGLU;
+    int splits = 0;
+    prof_begin(c);
+    const int rc = tc_gemm_launch(c, (const bf16*)A, (const bf16*)W, C, M, N, K, tc_epi, tc_epi == TC_SWIGLU ? N / 2 : N,
+                                  allow_split, &splits);
+    prof_end(c);
+    c->launches++;
+    if (rc == RPO_OK && splits > 1) { c->pending_splits = splits; c->pending_rows = M; }
+    return rc;
+  }
+  if (impl == 2 || epi == EPI_SWIGLU) return RPO_ERR_SHAPE;
   dim3 grid(ceil_div(N, 64), ceil_div(M, 64));
   if (epi == EPI_STORE_T) LAUNCH(c, (gemm_ref_kernel<T, EPI_STORE_T>), grid, 256, 0, A, W, C, M, N, K, (int64_t)N);
   else if (epi == EPI_STORE_F32) LAUNCH(c, (gemm_ref_kernel<T, EPI_STORE_F32>), grid, 256, 0, A, W, C, M, N, K, (int64_t)N);
@@ -332,8 +357,12 @@ static int rmsnorm(rpo_ctx* c, float* x, const float* g, T* h, int rows) {
   if (rows <= 0) return RPO_OK;
   ProfScope ps(c, KC_NORM);
   const int d = c->shape.d_model;
-  LAUNCH(c, rmsnorm_kernel<T>, rows, 256, (size_t)d * 4, x, g, h, rows, d, c->shape.rms_eps, (const float*)nullptr, 0,
-         (int64_t)0);
+  const bool fold = (x == c->ws.x && c->pending_splits > 0 && c->pending_rows == rows);
+  if (!fold && x == c->ws.x) RPO_TRY(flush_partials(c));
+  LAUNCH(c, rmsnorm_kernel<T>, rows, 256, (size_t)d * 4, x, g, h, rows, d, c->shape.rms_eps,
+         fold ? (const float*)c->ws.partial : (const float*)nullptr, fold ? c->pending_splits : 0,
+         (int64_t)rows * d);
+  if (fold) c->pending_splits = 0;
   return RPO_OK;
 }
 
@@ -371,13 +400,17 @@ static int run_layers(rpo_ctx* c, int rows) {
            (const SeqDesc*)w.seqs, c->d_block_table, (const float2*)c->d_rope, kv_pool<T>(c), l, rows, s.n_q_heads,
            s.n_kv_heads, c->lim.max_positions, c->d_status); }
     RPO_TRY(attention<T>(c, l, rows));
-    RPO_TRY(gemm<T>(c, (const T*)w.attn, (const T*)L.wo, w.x, rows, d, qo, EPI_ADD_F32));
+    RPO_TRY(gemm<T>(c, (const T*)w.attn, (const T*)L.wo, w.x, rows, d, qo, EPI_ADD_F32, 0, true));
     RPO_TRY(rmsnorm<T>(c, w.x, L.g2, (T*)w.h, rows));
-    RPO_TRY(gemm<T>(c, (const T*)w.h, (const T*)L.wgu, w.gu, rows, 2 * F, d, EPI_STORE_T));
-    LAUNCH(c, swiglu_kernel<T>, grid_for((int64_t)rows * F, 256), 256, 0, (const T*)w.gu, (T*)w.act, (int64_t)rows * F);
-    RPO_TRY(gemm<T>(c, (const T*)w.act, (const T*)L.wd, w.x, rows, d, F, EPI_ADD_F32));
+    if (c->use_tcgen05 && tc_gemm_supported<T>(c, rows, 2 * F, d) && F % 8 == 0) {
+      RPO_TRY(gemm<T>(c, (const T*)w.h, (const T*)L.wgu, w.act, rows, 2 * F, d, EPI_SWIGLU));   // SwiGLU in the epilogue
+    } else {
+      RPO_TRY(gemm<T>(c, (const T*)w.h, (const T*)L.wgu, w.gu, rows, 2 * F, d, EPI_STORE_T));
+      LAUNCH(c, swiglu_kernel<T>, grid_for((int64_t)rows * F, 256), 256, 0, (const T*)w.gu, (T*)w.act, (int64_t)rows * F);
+    }
+    RPO_TRY(gemm<T>(c, (const T*)w.act, (const T*)L.wd, w.x, rows, d, F, EPI_ADD_F32, 0, true));
   }
-  return RPO_OK;
+  return flush_partials(c);
 }
 
 // logits[n, V] (float32, ws.logits) from n residual rows in ws.xh.

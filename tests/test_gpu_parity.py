@@ -277,3 +277,26 @@ def test_rollout_host_matches_device_calls():
         assert np.array_equal(ht, t) and np.array_equal(hl, l) and np.array_equal(hp, lp)
         assert np.max(np.abs(hq - hp)) < 1e-4
         assert ctx.counters()[1] == ctx.limits.kv_pool_blocks
+
+
+def test_tensor_core_gemm_against_numpy():
+    """tcgen05/TMA GEMM (bf16 in, float32 accumulate) on shapes spanning several tiles, ragged M/N
+    tails, every tile width and a deep K."""
+    rng = np.random.default_rng(3)
+    shape = dict(SMALL_BF16)
+    with make_ctx(shape, 1, 1, 32, 4) as ctx:
+        for (M, N, K) in [(128, 256, 64), (1, 16, 64), (12, 48, 128), (129, 272, 192), (300, 4096, 512),
+                          (128, 2048, 1536), (40, 1536, 8960), (1000, 512, 256), (257, 151936 // 64, 128)]:
+            a = em.round_bf16((rng.standard_normal((M, K))).astype(np.float32))
+            w = em.round_bf16((rng.standard_normal((N, K)) * 0.05).astype(np.float32))
+            dA = torch.from_numpy(a).to(DEV).to(torch.bfloat16); dW = torch.from_numpy(w).to(DEV).to(torch.bfloat16)
+            dC = torch.full((M, N), 777.0, dtype=torch.float32, device=DEV)
+            ctx.gemm(dA, dW, dC, impl=2)
+            torch.cuda.synchronize()
+            assert ctx.device_status() == 0
+            ref = a.astype(np.float64) @ w.astype(np.float64).T
+            err = np.max(np.abs(dC.cpu().numpy() - ref))
+            assert err < 2e-5 * K ** 0.5, (M, N, K, err)
+        with pytest.raises(rpo.RpoError):
+            ctx.gemm(torch.zeros((8, 72), dtype=torch.bfloat16, device=DEV), torch.zeros((16, 72), dtype=torch.bfloat16, device=DEV),
+                     torch.zeros((8, 16), dtype=torch.float32, device=DEV), impl=2)      # K % 64 != 0
