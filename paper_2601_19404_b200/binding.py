@@ -135,9 +135,10 @@ class Context:
         _check(self.lib.rpo_create(C.byref(self.handle), C.byref(self.shape), C.byref(self.limits), stream_ptr), "rpo_create")
 
     def close(self):
-        if getattr(self, "handle", None) is not None and self.handle.value:
-            self.lib.rpo_destroy(self.handle)
-            self.handle = C.c_void_p()
+        h = getattr(self, "handle", None)
+        if h is not None and h.value:
+            self.lib.rpo_destroy(h)
+            h.value = None
 
     __del__ = close
 

@@ -306,11 +306,17 @@ inline int tc_create(rpo_ctx* c) {
   c->tc_state = s;
   if (!c->bf16) return RPO_OK;
   void* fn = nullptr;
-  cudaDriverEntryPointQueryResult q;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
-      q != cudaDriverEntryPointSuccess || !fn) {
+  cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+  cudaError_t e = cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &q);
+  if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn) {
     cudaGetLastError();
-    fprintf(stderr, "[rpo] cuTensorMapEncodeTiled unavailable: tensor-core GEMM disabled\n");
+    fn = nullptr;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+  }
+  if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn) {
+    cudaGetLastError();
+    fprintf(stderr, "[rpo] cuTensorMapEncodeTiled unavailable (%s, query %d): tensor-core GEMM disabled\n",
+            cudaGetErrorName(e), (int)q);
     return RPO_OK;
   }
   s->encode = (EncodeTiledFn)fn;
