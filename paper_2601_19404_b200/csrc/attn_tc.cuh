@@ -1,0 +1,325 @@
+// bf16 attention on tensor cores (mma.sync m16n8k16, float32 softmax and accumulation) over the
+// paged KV cache, flash style: a 64-row query tile stays in registers while 64-key K/V tiles are
+// streamed through a double-buffered, XOR-swizzled shared-memory ring with cp.async.
+//
+// Key space of a query row = [shared segment: the group's prefix blocks, all visible]
+//                         ++ [private segment: the sequence's own blocks, keys 0..t visible].
+// Three uses:
+//   ROWS   (prefill, teacher-forced log-probs): a tile holds 64 consecutive rows of one sequence
+//          for one query head; output is the normalised attention, written as bf16.
+//   SHARED (decode): a tile holds the G * (Hq/Hkv) query rows of one prompt group that share a KV
+//          head, and one split of the group's prefix; the prefix K/V of a group is therefore read
+//          once per group, not once per sample.  Output: (m, l, unnormalised O) partials.
+//   The per-sequence suffix keys and the split merge are handled by attn_decode_merge_kernel.
+#pragma once
+#include "kernels.cuh"
+
+namespace rpo {
+
+constexpr int FA_BM = 64, FA_BN = 64, FA_THREADS = 128;
+enum FlashMode { FA_ROWS = 0, FA_SHARED = 1 };
+
+struct FlashArgs {
+  const bf16* qkv; int qkv_cols;
+  bf16* out; int out_cols;
+  float* part_ml; float* part_o; int n_splits; int split_chunk;   // SHARED
+  const int32_t* row_seq; const int32_t* row_t; const SeqDesc* seqs; const int32_t* block_table;
+  KVPool<bf16> pool; int layer, hq, hkv; float scale_log2;
+  const int2* tiles;      // ROWS: (first row, number of rows)
+  int G;                  // SHARED: samples per group
+  int* status;
+};
+
+namespace fa {
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void st_zero16(uint32_t dst) {
+  asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *(uint32_t*)&h;
+}
+}  // namespace fa
+
+template <int DH, int MODE>
+__global__ void __launch_bounds__(FA_THREADS) flash_attn_kernel(FlashArgs a) {
+  constexpr int CH = DH / 8;                 // 16-byte chunks per row
+  constexpr int ROW_BYTES = DH * 2;
+  constexpr int TILE_BYTES = FA_BN * ROW_BYTES;
+  constexpr int KSTEPS = DH / 16, ONT = DH / 8;
+  extern __shared__ __align__(128) uint8_t fsm[];
+  const uint32_t sQ = (uint32_t)__cvta_generic_to_shared(fsm);
+  const uint32_t sK = sQ + FA_BM * ROW_BYTES;          // 2 buffers
+  const uint32_t sV = sK + 2 * TILE_BYTES;             // 2 buffers
+  __shared__ int s_qrow[FA_BM];     // qkv row of each tile row (-1: padding)
+  __shared__ int s_head[FA_BM];
+  __shared__ int s_t[FA_BM];        // private causal limit (-1: nothing visible / inactive)
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
+  const int rep = a.hq / a.hkv;
+  int kvh, n_rows, split = 0;
+  SeqDesc sd;
+  if (MODE == FA_ROWS) {
+    const int2 tile = a.tiles[blockIdx.x];
+    const int head = blockIdx.y;
+    kvh = head / rep; n_rows = tile.y;
+    sd = a.seqs[a.row_seq[tile.x]];
+    if (tid < FA_BM) {
+      const bool v = tid < n_rows;
+      s_qrow[tid] = v ? tile.x + tid : -1;
+      s_head[tid] = head;
+      s_t[tid] = v ? a.row_t[tile.x + tid] : -1;
+    }
+  } else {
+    const int rows_per_group = a.G * rep;
+    const int tiles_per_group = (rows_per_group + FA_BM - 1) / FA_BM;
+    const int grp = blockIdx.x / tiles_per_group, r0 = (blockIdx.x % tiles_per_group) * FA_BM;
+    kvh = blockIdx.y; split = blockIdx.z;
+    n_rows = min(FA_BM, rows_per_group - r0);
+    sd = a.seqs[grp * a.G];
+    if (tid < FA_BM) {
+      const bool v = tid < n_rows;
+      const int i = r0 + tid;
+      s_qrow[tid] = v ? grp * a.G + i / rep : -1;
+      s_head[tid] = kvh * rep + (v ? i % rep : 0);
+      s_t[tid] = -1;
+    }
+  }
+  __syncthreads();
+
+  // ---- key ranges
+  int sh_begin = 0, sh_end = 0, pr_end = 0;
+  if (MODE == FA_ROWS) {
+    sh_end = (sd.shared_tbl >= 0) ? sd.shared_len : 0;
+    int mt = -1;
+    for (int i = 0; i < n_rows; ++i) mt = max(mt, s_t[i]);
+    pr_end = mt + 1;
+  } else {
+    sh_begin = min(sd.shared_len, split * a.split_chunk);
+    sh_end = min(sd.shared_len, sh_begin + a.split_chunk);
+  }
+  const int n_sh_tiles = (sh_end - sh_begin + FA_BN - 1) / FA_BN;
+  const int n_pr_tiles = (pr_end + FA_BN - 1) / FA_BN;
+  const int n_tiles = n_sh_tiles + n_pr_tiles;
+
+  // ---- loaders: thread pair per row, interleaved 16-byte chunks (32 contiguous bytes per pair)
+  const int lrow = tid >> 1, lpar = tid & 1;
+  auto sw = [&](int row, int chunk) -> uint32_t { return (uint32_t)(row * ROW_BYTES + ((chunk ^ (row & 7)) << 4)); };
+  auto load_kv = [&](int it, int buf) {
+    int tbl, key0, limit;
+    if (it < n_sh_tiles) { tbl = sd.shared_tbl; key0 = sh_begin + it * FA_BN; limit = sh_end; }
+    else { tbl = sd.priv_tbl; key0 = (it - n_sh_tiles) * FA_BN; limit = pr_end; }
+    const int u = key0 + lrow;
+    const bf16 *kp = nullptr, *vp = nullptr;
+    if (u < limit) {
+      const int blk = a.block_table[tbl + u / KV_BLOCK];
+      if (blk >= 0 && blk < a.pool.n_blocks) {
+        kp = a.pool.at(a.layer, 0, kvh, blk, u % KV_BLOCK);
+        vp = a.pool.at(a.layer, 1, kvh, blk, u % KV_BLOCK);
+      } else {
+        atomicOr(a.status, STATUS_BAD_BLOCK);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < CH / 2; ++j) {
+      const int ch = 2 * j + lpar;
+      const uint32_t off = sw(lrow, ch);
+      if (kp) { fa::cp_async16(sK + buf * TILE_BYTES + off, kp + ch * 8); fa::cp_async16(sV + buf * TILE_BYTES + off, vp + ch * 8); }
+      else { fa::st_zero16(sK + buf * TILE_BYTES + off); fa::st_zero16(sV + buf * TILE_BYTES + off); }
+    }
+  };
+  {
+    const int qr = s_qrow[lrow];
+    const bf16* qp = (qr >= 0) ? a.qkv + (int64_t)qr * a.qkv_cols + s_head[lrow] * DH : nullptr;
+#pragma unroll
+    for (int j = 0; j < CH / 2; ++j) {
+      const int ch = 2 * j + lpar;
+      if (qp) fa::cp_async16(sQ + sw(lrow, ch), qp + ch * 8); else fa::st_zero16(sQ + sw(lrow, ch));
+    }
+  }
+  if (n_tiles > 0) load_kv(0, 0);
+  fa::cp_commit();
+
+  float o[ONT][4];
+#pragma unroll
+  for (int i = 0; i < ONT; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+  float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+  uint32_t qf[KSTEPS][4];
+  const int r_lo = warp * 16 + g, r_hi = r_lo + 8;
+  const int t_lo = s_t[r_lo], t_hi = s_t[r_hi];
+
+  for (int it = 0; it < n_tiles; ++it) {
+    const int buf = it & 1;
+    if (it + 1 < n_tiles) { load_kv(it + 1, buf ^ 1); fa::cp_commit(); fa::cp_wait<1>(); } else { fa::cp_wait<0>(); }
+    __syncthreads();
+    if (it == 0) {
+#pragma unroll
+      for (int kk = 0; kk < KSTEPS; ++kk)
+        fa::ldsm_x4(sQ + sw(warp * 16 + (lane & 15), kk * 2 + (lane >> 4)), qf[kk][0], qf[kk][1], qf[kk][2], qf[kk][3]);
+    }
+    // ---- S = Q K^T
+    float s[FA_BN / 8][4];
+#pragma unroll
+    for (int j = 0; j < FA_BN / 8; ++j) { s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f; }
+    const uint32_t kb = sK + buf * TILE_BYTES, vb = sV + buf * TILE_BYTES;
+#pragma unroll
+    for (int kk = 0; kk < KSTEPS; ++kk) {
+#pragma unroll
+      for (int jp = 0; jp < FA_BN / 16; ++jp) {
+        uint32_t b0, b1, b2, b3;
+        fa::ldsm_x4(kb + sw(jp * 16 + (lane & 7) + ((lane >> 4) << 3), kk * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
+        fa::mma_bf16(s[2 * jp], qf[kk], b0, b1);
+        fa::mma_bf16(s[2 * jp + 1], qf[kk], b2, b3);
+      }
+    }
+    // ---- mask + online softmax (base-2 exponent domain)
+    const bool shared_tile = it < n_sh_tiles;
+    const int key0 = shared_tile ? sh_begin + it * FA_BN : (it - n_sh_tiles) * FA_BN;
+    float mx_lo = -INFINITY, mx_hi = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < FA_BN / 8; ++j) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const int key = key0 + j * 8 + tq * 2 + (c & 1);
+        const bool vis = shared_tile ? (key < sh_end) : (key <= ((c & 2) ? t_hi : t_lo));
+        const float v = vis ? s[j][c] * a.scale_log2 : -INFINITY;
+        s[j][c] = v;
+        if (c & 2) mx_hi = fmaxf(mx_hi, v); else mx_lo = fmaxf(mx_lo, v);
+      }
+    }
+    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1)); mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1)); mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+    const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
+    const float mu_lo = (mn_lo == -INFINITY) ? 0.f : mn_lo, mu_hi = (mn_hi == -INFINITY) ? 0.f : mn_hi;
+    const float c_lo = exp2f(m_lo - mu_lo), c_hi = exp2f(m_hi - mu_hi);
+    m_lo = mn_lo; m_hi = mn_hi;
+    float ps_lo = 0.f, ps_hi = 0.f;
+    uint32_t pf[FA_BN / 16][4];
+#pragma unroll
+    for (int j = 0; j < FA_BN / 8; ++j) {
+      const float p0 = exp2f(s[j][0] - mu_lo), p1 = exp2f(s[j][1] - mu_lo);
+      const float p2 = exp2f(s[j][2] - mu_hi), p3 = exp2f(s[j][3] - mu_hi);
+      ps_lo += p0 + p1; ps_hi += p2 + p3;
+      pf[j >> 1][(j & 1) * 2] = fa::pack_bf16(p0, p1);
+      pf[j >> 1][(j & 1) * 2 + 1] = fa::pack_bf16(p2, p3);
+    }
+    l_lo = l_lo * c_lo + ps_lo; l_hi = l_hi * c_hi + ps_hi;
+#pragma unroll
+    for (int i = 0; i < ONT; ++i) { o[i][0] *= c_lo; o[i][1] *= c_lo; o[i][2] *= c_hi; o[i][3] *= c_hi; }
+    // ---- O += P V
+#pragma unroll
+    for (int kk = 0; kk < FA_BN / 16; ++kk) {
+#pragma unroll
+      for (int np = 0; np < ONT / 2; ++np) {
+        uint32_t b0, b1, b2, b3;
+        fa::ldsm_x4_t(vb + sw(kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), np * 2 + (lane >> 4)), b0, b1, b2, b3);
+        fa::mma_bf16(o[2 * np], pf[kk], b0, b1);
+        fa::mma_bf16(o[2 * np + 1], pf[kk], b2, b3);
+      }
+    }
+    __syncthreads();
+  }
+  fa::cp_wait<0>();
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1); l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1); l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+
+  // ---- write
+#pragma unroll
+  for (int half = 0; half < 2; ++half) {
+    const int r = half ? r_hi : r_lo;
+    const int qr = s_qrow[r];
+    if (qr < 0) continue;
+    const float l = half ? l_hi : l_lo, m = half ? m_hi : m_lo;
+    if (MODE == FA_ROWS) {
+      const float inv = (l > 0.f) ? 1.0f / l : 0.f;
+      bf16* dst = a.out + (int64_t)qr * a.out_cols + s_head[r] * DH;
+#pragma unroll
+      for (int i = 0; i < ONT; ++i)
+        *(uint32_t*)(dst + i * 8 + tq * 2) = fa::pack_bf16(o[i][half * 2] * inv, o[i][half * 2 + 1] * inv);
+    } else {
+      const int64_t slot = ((int64_t)qr * a.hq + s_head[r]) * a.n_splits + split;
+      if (tq == 0) { a.part_ml[slot * 2] = m; a.part_ml[slot * 2 + 1] = l; }
+      float* dst = a.part_o + slot * DH;
+#pragma unroll
+      for (int i = 0; i < ONT; ++i) *(float2*)(dst + i * 8 + tq * 2) = make_float2(o[i][half * 2], o[i][half * 2 + 1]);
+    }
+  }
+}
+
+// Decode: merge the shared-prefix partials of (sequence, query head) with attention over the
+// sequence's own suffix keys 0..t (private blocks), one warp each; lanes own DH/32 dimensions.
+template <int DH>
+__global__ void __launch_bounds__(128) attn_decode_merge_kernel(const bf16* __restrict__ qkv, int qkv_cols,
+                                                                bf16* __restrict__ out, const float* __restrict__ part_ml,
+                                                                const float* __restrict__ part_o, int n_splits,
+                                                                const int32_t* __restrict__ row_seq,
+                                                                const int32_t* __restrict__ row_t,
+                                                                const SeqDesc* __restrict__ seqs,
+                                                                const int32_t* __restrict__ block_table,
+                                                                KVPool<bf16> pool, int layer, int rows, int hq, int hkv,
+                                                                float scale_log2, int* status) {
+  constexpr int DPL = DH / 32;
+  const int w = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (w >= rows * hq) return;
+  const int r = w / hq, head = w % hq;
+  bf16* o = out + (int64_t)r * hq * DH + head * DH + lane * DPL;
+  const int t = row_t[r];
+  if (t < 0) {
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) o[i] = __float2bfloat16_rn(0.f);
+    return;
+  }
+  const SeqDesc sd = seqs[row_seq[r]];
+  const int kvh = head / (hq / hkv);
+  float m = -INFINITY, l = 0.f, acc[DPL];
+#pragma unroll
+  for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
+  for (int s = 0; s < n_splits; ++s) {
+    const int64_t slot = ((int64_t)r * hq + head) * n_splits + s;
+    const float ms = part_ml[slot * 2], ls = part_ml[slot * 2 + 1];
+    if (ls <= 0.f) continue;
+    const float mn = fmaxf(m, ms), c0 = exp2f(m - mn), c1 = exp2f(ms - mn);
+    l = l * c0 + ls * c1;
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) acc[i] = acc[i] * c0 + part_o[slot * DH + lane * DPL + i] * c1;
+    m = mn;
+  }
+  const bf16* qp = qkv + (int64_t)r * qkv_cols + head * DH + lane * DPL;
+  float q[DPL];
+#pragma unroll
+  for (int i = 0; i < DPL; ++i) q[i] = __bfloat162float(qp[i]) * scale_log2;
+  for (int u = 0; u <= t; ++u) {
+    const int blk = block_table[sd.priv_tbl + u / KV_BLOCK];
+    if (blk < 0 || blk >= pool.n_blocks) { if (lane == 0) atomicOr(status, STATUS_BAD_BLOCK); continue; }
+    const bf16* kp = pool.at(layer, 0, kvh, blk, u % KV_BLOCK) + lane * DPL;
+    const bf16* vp = pool.at(layer, 1, kvh, blk, u % KV_BLOCK) + lane * DPL;
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) s = fmaf(q[i], __bfloat162float(kp[i]), s);
+    s = warp_sum(s);
+    const float mn = fmaxf(m, s), c0 = exp2f(m - mn), p = exp2f(s - mn);
+    l = l * c0 + p;
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) acc[i] = acc[i] * c0 + p * __bfloat162float(vp[i]);
+    m = mn;
+  }
+  const float inv = 1.0f / l;
+#pragma unroll
+  for (int i = 0; i < DPL; ++i) o[i] = __float2bfloat16_rn(acc[i] * inv);
+}
+
+}  // namespace rpo

@@ -43,6 +43,7 @@ struct Workspace {
   size_t partial_elems = 0;
   float* attn_part = nullptr;    // decode attention partials
   size_t attn_part_elems = 0;
+  void* tiles = nullptr;   // int2 (first row, rows) per 64-row attention tile
   int32_t *row_seq = nullptr, *row_t = nullptr, *row_tok = nullptr;
   void* seqs = nullptr;    // SeqDesc[]
   int32_t *done = nullptr, *lens = nullptr, *cur_tok = nullptr, *logit_row = nullptr, *slot_idx = nullptr;
@@ -82,6 +83,8 @@ struct rpo_ctx {
   int sm_count = 148;
   // options
   int use_tcgen05 = 1, use_tc_attention = 1, use_graph = 1;
+  // attention plan of the pass being enqueued: 0 = row tiles (prefill / teacher), 1 = decode
+  int attn_mode = 0, attn_tiles = 0, attn_G = 1, attn_groups = 0, attn_splits = 1, attn_split_chunk = 64;
   int pending_splits = 0, pending_rows = 0;   // split-K partials of ws.x not yet reduced
   // optional per-kernel timing: event pairs around every launch, tagged class + 16*phase
   struct ProfEvent { cudaEvent_t a, b; int tag; };

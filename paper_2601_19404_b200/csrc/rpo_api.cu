@@ -7,6 +7,9 @@
 #include <cstring>
 #include <new>
 
+#include <type_traits>
+
+#include "attn_tc.cuh"
 #include "context.h"
 #include "gemm_tc.cuh"
 #include "kernels.cuh"
@@ -235,6 +238,9 @@ extern "C" int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limit
   ALLOC(w.logit_row, (size_t)nseq * 4);
   ALLOC(w.slot_idx, (size_t)nseq * 4);
   ALLOC(w.seq_ids, (size_t)nseq * 8);
+  ALLOC(w.tiles, ((size_t)w.R / FA_BM + nseq + 2) * sizeof(int2));
+  w.attn_part_elems = (size_t)lim->max_seqs * s.n_q_heads * 32 * (dh + 2);
+  ALLOC(w.attn_part, w.attn_part_elems * 4);
   w.partial_elems = (size_t)c->sm_count * 128 * 256;
   ALLOC(w.partial, w.partial_elems * 4);
   if (rc == RPO_OK) rc = tc_create(c);
@@ -366,12 +372,51 @@ static int rmsnorm(rpo_ctx* c, float* x, const float* g, T* h, int rows) {
   return RPO_OK;
 }
 
+template <int DH, int MODE>
+static int launch_flash(rpo_ctx* c, const FlashArgs& a, dim3 grid) {
+  constexpr int smem = (FA_BM + 4 * FA_BN) * DH * 2;
+  static bool attr_done = false;
+  if (!attr_done) {
+    CUDA_TRY(cudaFuncSetAttribute(flash_attn_kernel<DH, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    attr_done = true;
+  }
+  LAUNCH(c, (flash_attn_kernel<DH, MODE>), grid, FA_THREADS, smem, a);
+  return RPO_OK;
+}
+
 template <typename T>
 static int attention(rpo_ctx* c, int layer, int rows) {
   const rpo_shape& s = c->shape;
   Workspace& w = c->ws;
   const float scale = 1.0f / sqrtf((float)s.head_dim);
   ProfScope ps(c, KC_ATTN);
+  if constexpr (std::is_same<T, bf16>::value) {
+    if (c->use_tc_attention) {
+      FlashArgs a;
+      memset(&a, 0, sizeof(a));
+      a.qkv = (const bf16*)w.qkv; a.qkv_cols = c->qkv_cols; a.out = (bf16*)w.attn; a.out_cols = s.n_q_heads * s.head_dim;
+      a.part_ml = w.attn_part; a.part_o = w.attn_part + (size_t)2 * c->lim.max_seqs * s.n_q_heads * 32;
+      a.row_seq = w.row_seq; a.row_t = w.row_t; a.seqs = (const SeqDesc*)w.seqs; a.block_table = c->d_block_table;
+      a.pool = kv_pool<bf16>(c); a.layer = layer; a.hq = s.n_q_heads; a.hkv = s.n_kv_heads;
+      a.scale_log2 = scale * 1.4426950408889634f; a.tiles = (const int2*)w.tiles; a.G = c->attn_G; a.status = c->d_status;
+      a.n_splits = c->attn_splits; a.split_chunk = c->attn_split_chunk;
+      if (c->attn_mode == 0) {
+        dim3 grid(c->attn_tiles, s.n_q_heads);
+        return s.head_dim == 128 ? launch_flash<128, FA_ROWS>(c, a, grid) : launch_flash<64, FA_ROWS>(c, a, grid);
+      }
+      const int rep = s.n_q_heads / s.n_kv_heads;
+      dim3 grid(c->attn_groups * ceil_div(c->attn_G * rep, FA_BM), s.n_kv_heads, c->attn_splits);
+      RPO_TRY((s.head_dim == 128 ? launch_flash<128, FA_SHARED>(c, a, grid) : launch_flash<64, FA_SHARED>(c, a, grid)));
+      const int mgrid = ceil_div((int64_t)rows * s.n_q_heads, 4);
+      if (s.head_dim == 128)
+        LAUNCH(c, (attn_decode_merge_kernel<128>), mgrid, 128, 0, a.qkv, a.qkv_cols, a.out, a.part_ml, a.part_o, a.n_splits,
+               w.row_seq, w.row_t, a.seqs, a.block_table, a.pool, layer, rows, a.hq, a.hkv, a.scale_log2, c->d_status);
+      else
+        LAUNCH(c, (attn_decode_merge_kernel<64>), mgrid, 128, 0, a.qkv, a.qkv_cols, a.out, a.part_ml, a.part_o, a.n_splits,
+               w.row_seq, w.row_t, a.seqs, a.block_table, a.pool, layer, rows, a.hq, a.hkv, a.scale_log2, c->d_status);
+      return RPO_OK;
+    }
+  }
   const int grid = ceil_div((int64_t)rows * s.n_q_heads, 4);
   if (s.head_dim == 64)
     LAUNCH(c, (attn_ref_kernel<T, 64>), grid, 128, 0, (const T*)w.qkv, (T*)w.attn, w.row_seq, w.row_t,
@@ -381,6 +426,20 @@ static int attention(rpo_ctx* c, int layer, int rows) {
     LAUNCH(c, (attn_ref_kernel<T, 128>), grid, 128, 0, (const T*)w.qkv, (T*)w.attn, w.row_seq, w.row_t,
            (const SeqDesc*)w.seqs, c->d_block_table, kv_pool<T>(c), layer, rows, s.n_q_heads, s.n_kv_heads, scale,
            c->d_status);
+  return RPO_OK;
+}
+
+// 64-row query tiles of a pass whose sequences own consecutive row ranges.
+static int upload_row_tiles(rpo_ctx* c, const std::vector<int>& rows_per_seq) {
+  std::vector<int2> tiles;
+  int r = 0;
+  for (int n : rows_per_seq) {
+    for (int r0 = 0; r0 < n; r0 += FA_BM) tiles.push_back(make_int2(r + r0, std::min(FA_BM, n - r0)));
+    r += n;
+  }
+  c->attn_mode = 0; c->attn_tiles = (int)tiles.size();
+  if (!tiles.empty())
+    CUDA_TRY(cudaMemcpyAsync(c->ws.tiles, tiles.data(), tiles.size() * sizeof(int2), cudaMemcpyHostToDevice, c->stream));
   return RPO_OK;
 }
 
@@ -464,6 +523,7 @@ static int prefill_chunk(rpo_ctx* c, const int32_t* d_tokens, int tok0, const st
   CUDA_TRY(cudaMemcpyAsync(w.row_seq, row_seq.data(), (size_t)rows * 4, cudaMemcpyHostToDevice, c->stream));
   CUDA_TRY(cudaMemcpyAsync(w.row_t, row_t.data(), (size_t)rows * 4, cudaMemcpyHostToDevice, c->stream));
   CUDA_TRY(cudaMemcpyAsync(w.seqs, sd.data(), (size_t)n * sizeof(SeqDesc), cudaMemcpyHostToDevice, c->stream));
+  RPO_TRY(upload_row_tiles(c, lens));
   LAUNCH(c, embed_kernel<T>, rows, 128, 0, d_tokens + tok0, (const T*)c->embed, w.x, rows, c->shape.d_model,
          c->shape.vocab, c->d_status);
   RPO_TRY(run_layers<T>(c, rows));
@@ -578,6 +638,16 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
   CUDA_TRY(cudaMemsetAsync(w.lens, 0, (size_t)B * 4, st));
   CUDA_TRY(cudaMemsetAsync(w.row_t, 0xFF, (size_t)B * 4, st));
 
+  {
+    int max_p = 1;
+    for (int g = 0; g < n_groups; ++g) max_p = std::max(max_p, groups[g].prefix_len);
+    const int rep = c->shape.n_q_heads / c->shape.n_kv_heads;
+    const int pairs = n_groups * c->shape.n_kv_heads * ceil_div(G * rep, FA_BM);
+    const int want = std::max(1, std::min(32, ceil_div(2 * c->sm_count, pairs)));
+    c->attn_split_chunk = std::max(FA_BN, ceil_div(ceil_div(max_p, want), FA_BN) * FA_BN);
+    c->attn_splits = ceil_div(max_p, c->attn_split_chunk);
+    c->attn_mode = 1; c->attn_G = G; c->attn_groups = n_groups;
+  }
   SamplerArgs a = sampler_args(c, sp);
   a.seq_ids = w.seq_ids; a.out_stride = S; a.forced = d_forced; a.tokens_out = d_tokens_out;
   a.logprobs_out = d_logprobs_out; a.done = w.done; a.lens = w.lens; a.cur_tok = w.cur_tok; a.row_t = w.row_t;
@@ -659,6 +729,7 @@ static int logprobs_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, 
       }
       const int rows = ns * (S - 1);
       if (rows > 0) {
+        if ((rc = upload_row_tiles(c, std::vector<int>(ns, S - 1))) != RPO_OK) break;
         build_teacher_rows_kernel<<<grid_for(rows, 256), 256, 0, st>>>(d_tokens, d_lens, s0, ns, S, w.row_seq, w.row_t,
                                                                       w.row_tok);
         c->launches++;
