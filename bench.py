@@ -167,6 +167,10 @@ def main():
     ap.add_argument("--ref-prefix", type=int, default=128)
     ap.add_argument("--ref-suffix", type=int, default=4)
     ap.add_argument("--options", default="", help="comma list name=value passed to rpo_set_option")
+    ap.add_argument("--layers", type=int, default=0, help="override n_layers (reduced case for profiler captures)")
+    ap.add_argument("--suffix", type=int, default=0, help="override the suffix length (reduced case for profiler captures)")
+    ap.add_argument("--groups", type=int, default=0, help="override the number of prompt groups (reduced case)")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -187,8 +191,15 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=dev)
 
-    cfg = workloads.CONFIGS[args.config]
-    shape = workloads.SHAPES[cfg["shape"]]
+    cfg = dict(workloads.CONFIGS[args.config])
+    shape = dict(workloads.SHAPES[cfg["shape"]])
+    reduced = []
+    if args.layers:
+        shape["n_layers"] = args.layers; reduced.append(f"layers={args.layers}")
+    if args.suffix:
+        cfg["suffix"] = args.suffix; reduced.append(f"suffix={args.suffix}")
+    if args.groups:
+        cfg["n_groups"] = args.groups; reduced.append(f"groups={args.groups}")
     n_g, G, S = cfg["n_groups"], cfg["G"], cfg["suffix"]
     B = n_g * G
     lens = workloads.prefix_lengths(cfg, seed=rank)
@@ -266,33 +277,36 @@ def main():
     value = emitted_all / (ms_per_step / 1e3)
 
     # ---- end to end through the host-buffer call (pinned host memory, copies inside the timed region)
-    h_toks = torch.from_numpy(toks).pin_memory()
-    h_out = torch.zeros((B, S), dtype=torch.int32).pin_memory()
-    h_lens = torch.zeros(B, dtype=torch.int32).pin_memory()
-    h_lp = torch.zeros((B, S), dtype=torch.float32).pin_memory()
-    h_pol = torch.zeros((B, S), dtype=torch.float32).pin_memory() if want_lp else None
+    e2e = None
+    if not args.no_e2e:
+        h_toks = torch.from_numpy(toks).pin_memory()
+        h_out = torch.zeros((B, S), dtype=torch.int32).pin_memory()
+        h_lens = torch.zeros(B, dtype=torch.int32).pin_memory()
+        h_lp = torch.zeros((B, S), dtype=torch.float32).pin_memory()
+        h_pol = torch.zeros((B, S), dtype=torch.float32).pin_memory() if want_lp else None
 
-    def e2e_step():
-        ctx.rollout_host(h_toks.numpy(), off, G, S, smp, h_out.numpy(), h_lens.numpy(), h_lp.numpy(),
-                         None if h_pol is None else h_pol.numpy(), group_ids=group_ids)
+        def e2e_step():
+            ctx.rollout_host(h_toks.numpy(), off, G, S, smp, h_out.numpy(), h_lens.numpy(), h_lp.numpy(),
+                             None if h_pol is None else h_pol.numpy(), group_ids=group_ids)
 
-    e2e_step()
-    barrier()
-    e_begin = torch.cuda.Event(enable_timing=True); e_end = torch.cuda.Event(enable_timing=True)
-    n_e2e = max(1, min(args.steps, 3))
-    e_begin.record(stream)
-    for _ in range(n_e2e):
         e2e_step()
-    e_end.record(stream)
-    barrier()
-    e2e_ms = e_begin.elapsed_time(e_end) / n_e2e
-    e2e_tokens = int(h_lens.sum().item())
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64); dist.all_reduce(t, op=dist.ReduceOp.MAX); e2e_ms = t.item()
-        em = torch.tensor([e2e_tokens], device=dev, dtype=torch.int64); dist.all_reduce(em, op=dist.ReduceOp.SUM); e2e_tokens = int(em.item())
-    e2e_value = e2e_tokens / (e2e_ms / 1e3)
-    h2d = int(toks.nbytes)
-    d2h = int(h_out.numel() * 4 + h_lens.numel() * 4 + h_lp.numel() * 4 + (h_pol.numel() * 4 if want_lp else 0))
+        barrier()
+        e_begin = torch.cuda.Event(enable_timing=True); e_end = torch.cuda.Event(enable_timing=True)
+        n_e2e = max(1, min(args.steps, 3))
+        e_begin.record(stream)
+        for _ in range(n_e2e):
+            e2e_step()
+        e_end.record(stream)
+        barrier()
+        e2e_ms = e_begin.elapsed_time(e_end) / n_e2e
+        e2e_tokens = int(h_lens.sum().item())
+        if world > 1:
+            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64); dist.all_reduce(t, op=dist.ReduceOp.MAX); e2e_ms = t.item()
+            em = torch.tensor([e2e_tokens], device=dev, dtype=torch.int64); dist.all_reduce(em, op=dist.ReduceOp.SUM); e2e_tokens = int(em.item())
+        h2d = int(toks.nbytes)
+        d2h = int(h_out.numel() * 4 + h_lens.numel() * 4 + h_lp.numel() * 4 + (h_pol.numel() * 4 if want_lp else 0))
+        e2e = {"value": e2e_tokens / (e2e_ms / 1e3), "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h}
 
     # ---- roofline: per-kernel event timing in one extra profiled step (graphs off, same kernels)
     peaks = measured_peaks()
@@ -323,7 +337,7 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if shape["dtype"] == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": args.config, "shape": cfg["shape"], "n_groups": n_g, "G": G, "prefix_tokens": int(lens.sum()),
+        "config": {"workload": args.config + ("" if not reduced else " REDUCED(" + ",".join(reduced) + ")"), "shape": cfg["shape"], "n_groups": n_g, "G": G, "prefix_tokens": int(lens.sum()),
                    "suffix": S, "l2": "inputs larger than L2 (weights %.2f GB + KV)" % (ab["weights"] / 1e9),
                    "parallelism": f"groups sharded over {world} rank(s), no collective in the step"},
         "phases_ms": {"prefill": pre_ms, "decode": dec_ms, "logprobs": lp_ms, "decode_per_step": dec_step_ms},
@@ -332,7 +346,7 @@ def main():
         "prefill_tensor": {"flops": pf, "achieved_tflops": prefill_tfs, "frac_of_measured_burst": prefill_tfs / peaks["bf16_tflops"],
                            "frac_of_2250": prefill_tfs / 2250.0},
         "roofline": roofline, "kernel_classes": phases,
-        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "e2e": e2e,
         "gpu_launches": int(launches), "clocks": clk, "device_status": ctx.device_status(),
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
