@@ -204,7 +204,7 @@ def main():
     B = n_g * G
     lens = workloads.prefix_lengths(cfg, seed=rank)
     toks, off = workloads.prefix_tokens(lens, shape["vocab"], seed=rank)
-    group_ids = np.arange(n_g, dtype=np.int32) + rank * n_g          # weak scaling: every rank its own groups
+    group_ids = workloads.rank_group_ids(n_g, rank)                  # weak scaling: every rank its own groups
     sc = cfg["sampler"]
     smp = rpo.Sampler(sc["temperature"], sc["top_p"], sc["greedy"], sc["eos_id"], seed=0)
     want_lp = bool(cfg.get("logprobs"))

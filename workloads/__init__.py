@@ -54,6 +54,12 @@ def prefix_lengths(cfg, seed=0, n_groups=None):
     return rng.integers(spec[1], spec[2] + 1, size=n).astype(np.int32)
 
 
+def rank_group_ids(n_groups, rank):
+    """Group ids of a rank when prompt groups are sharded over ranks (each rank its own groups,
+    ids disjoint so that the samples' random streams differ)."""
+    return np.arange(n_groups, dtype=np.int32) + np.int32(rank * n_groups)
+
+
 def prefix_tokens(lengths, vocab, seed=0):
     """Concatenated uniform token ids and the offsets array [n_groups + 1]."""
     rng = np.random.Generator(np.random.PCG64([seed, 202]))
