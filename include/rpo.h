@@ -17,7 +17,9 @@
  *    keeps caller memory beyond the call, except that work reading/writing d_ buffers is
  *    *enqueued* on the stream given to rpo_create and may still be running on return;
  *    synchronise that stream before reading outputs or reusing inputs.
- *  - All kernels run on the one CUDA stream passed at creation (0 = legacy default).
+ *  - All kernels run on the one CUDA stream passed at creation.  With NULL the library creates a
+ *    blocking stream of its own, which keeps the implicit ordering with work on the legacy
+ *    default stream (that stream itself cannot be captured into the CUDA graphs decode uses).
  *  - There is no CPU fallback: without a CUDA device every compute call fails with
  *    RPO_ERR_CUDA.
  *  - Matrices are stored [out_features, in_features]; y = x W^T.

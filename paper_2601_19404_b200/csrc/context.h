@@ -47,6 +47,7 @@ struct Workspace {
   int32_t *row_seq = nullptr, *row_t = nullptr, *row_tok = nullptr;
   void* seqs = nullptr;    // SeqDesc[]
   int32_t *done = nullptr, *lens = nullptr, *cur_tok = nullptr, *logit_row = nullptr, *slot_idx = nullptr;
+  int32_t* step_ctr = nullptr;   // device counter of the decode step being computed
   int64_t* seq_ids = nullptr;
   int R = 0, HR = 0;
 };
@@ -57,6 +58,7 @@ struct rpo_ctx {
   rpo_shape shape;
   rpo_limits lim;
   cudaStream_t stream = nullptr;
+  bool own_stream = false;   // created by rpo_create because the caller passed NULL
   bool bf16 = false;
   size_t esz = 4;
   int qkv_cols = 0;
@@ -90,6 +92,9 @@ struct rpo_ctx {
   struct ProfEvent { cudaEvent_t a, b; int tag; };
   int profile = 0, prof_class = 0, prof_phase = 0;
   std::vector<ProfEvent> prof_events;
+  // instantiated CUDA graphs of one decode step, keyed by everything the step's launches depend on
+  struct StepGraph { std::vector<uint64_t> key; cudaGraphExec_t exec; int64_t launches; };
+  std::vector<StepGraph> step_graphs;
   // tcgen05 GEMM state (tensor maps are built per call; see gemm_tc.cuh)
   void* tc_state = nullptr;
 };

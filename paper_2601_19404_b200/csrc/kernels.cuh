@@ -79,10 +79,13 @@ __global__ void rope_table_kernel(float2* __restrict__ tab, int max_pos, int hal
 }
 
 // x[r,:] = E[tok[r],:]  (float32 residual stream).
+// step_ctr (decode only): the first kernel of a decode forward advances the device step counter
+// that the sampler at the end of the forward reads, so that every step is the same launch sequence.
 template <typename T>
 __global__ void embed_kernel(const int32_t* __restrict__ tokens, const T* __restrict__ E, float* __restrict__ x,
-                             int rows, int d, int vocab, int* status) {
+                             int rows, int d, int vocab, int* status, int32_t* step_ctr = nullptr) {
   const int r = blockIdx.x;
+  if (step_ctr && r == 0 && threadIdx.x == 0) *step_ctr += 1;
   if (r >= rows) return;
   int tok = tokens[r];
   if (tok < 0 || tok >= vocab) {

@@ -131,8 +131,11 @@ static void add_tensor(rpo_ctx* c, const std::string& name, void* ptr, int rows,
 extern "C" int rpo_destroy(rpo_ctx* ctx) {
   if (!ctx) return RPO_ERR_INVALID_ARG;
   cudaStreamSynchronize(ctx->stream);
+  for (auto& g : ctx->step_graphs) cudaGraphExecDestroy(g.exec);
+  ctx->step_graphs.clear();
   tc_destroy(ctx);
   for (void* p : ctx->allocations) cudaFree(p);
+  if (ctx->own_stream) cudaStreamDestroy(ctx->stream);
   delete ctx;
   return RPO_OK;
 }
@@ -158,6 +161,12 @@ extern "C" int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limit
   rpo_ctx* c = new (std::nothrow) rpo_ctx();
   if (!c) return RPO_ERR_CUDA;
   c->shape = s; c->lim = *lim; c->stream = (cudaStream_t)cuda_stream;
+  if (!c->stream) {
+    // The legacy default stream cannot be captured into a CUDA graph.  A blocking stream of our own
+    // keeps the implicit ordering with the caller's default-stream work and can be captured.
+    if (cudaStreamCreateWithFlags(&c->stream, cudaStreamDefault) != cudaSuccess) { cudaGetLastError(); delete c; return RPO_ERR_CUDA; }
+    c->own_stream = true;
+  }
   c->bf16 = s.dtype == RPO_DTYPE_BF16; c->esz = c->bf16 ? 2 : 4;
   c->qkv_cols = (s.n_q_heads + 2 * s.n_kv_heads) * s.head_dim;
   int dev = 0;
@@ -237,6 +246,7 @@ extern "C" int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limit
   ALLOC(w.cur_tok, (size_t)nseq * 4);
   ALLOC(w.logit_row, (size_t)nseq * 4);
   ALLOC(w.slot_idx, (size_t)nseq * 4);
+  ALLOC(w.step_ctr, 16);
   ALLOC(w.seq_ids, (size_t)nseq * 8);
   ALLOC(w.tiles, ((size_t)w.R / FA_BM + nseq + 2) * sizeof(int2));
   w.attn_part_elems = (size_t)lim->max_seqs * s.n_q_heads * 32 * (dh + 2);
@@ -654,21 +664,61 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
   a.logits_dbg = d_logits_dbg; a.logits = w.logits;
 
   // step 0: the G samples of a group draw from the logits of the group's last prefix token
+  CUDA_TRY(cudaMemsetAsync(w.step_ctr, 0, 4, st));
+  a.step_ptr = w.step_ctr; a.n_steps = S;
   LAUNCH(c, gather_rows_f32_kernel, n_groups, 128, 0, (const float*)c->d_x_last, (const int32_t*)w.slot_idx, w.xh,
          n_groups, d);
   RPO_TRY(head<T>(c, n_groups));
-  a.logit_row = w.logit_row; a.step = 0; a.out_col = 0; a.last_step = (S == 1);
+  a.logit_row = w.logit_row;
   { ProfScope ps(c, KC_SAMPLER); LAUNCH(c, sampler_kernel, B, 1024, 0, a); }
   a.logit_row = nullptr;
-  for (int j = 1; j < S; ++j) {
+  // steps 1..S-1 are one and the same launch sequence (the step number lives on the device):
+  // the first runs eagerly, the others replay a CUDA graph of it.
+  auto enqueue_step = [&]() -> int {
     LAUNCH(c, embed_kernel<T>, B, 128, 0, (const int32_t*)w.cur_tok, (const T*)c->embed, w.x, B, d, c->shape.vocab,
-           c->d_status);
+           c->d_status, w.step_ctr);
     RPO_TRY(run_layers<T>(c, B));
     CUDA_TRY(cudaMemcpyAsync(w.xh, w.x, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, st));
     RPO_TRY(head<T>(c, B));
-    a.step = j; a.out_col = j; a.last_step = (j == S - 1);
     { ProfScope ps(c, KC_SAMPLER); LAUNCH(c, sampler_kernel, B, 1024, 0, a); }
+    return RPO_OK;
+  };
+  int j = 1;
+  if (j < S) { RPO_TRY(enqueue_step()); ++j; }
+  if (j < S && c->use_graph && !c->profile && S - j >= 2) {
+    uint32_t temp_bits; memcpy(&temp_bits, &a.temperature, 4);
+    std::vector<uint64_t> key = {(uint64_t)B, (uint64_t)n_groups, (uint64_t)G, (uint64_t)S, (uint64_t)c->attn_splits,
+                                 (uint64_t)c->attn_split_chunk, (uint64_t)(uintptr_t)d_forced, (uint64_t)(uintptr_t)d_tokens_out,
+                                 (uint64_t)(uintptr_t)d_logprobs_out, (uint64_t)(uintptr_t)d_logits_dbg,
+                                 (uint64_t)a.top_p24, (uint64_t)temp_bits,
+                                 (uint64_t)a.greedy, (uint64_t)(uint32_t)a.eos_id, a.seed,
+                                 (uint64_t)c->use_tcgen05, (uint64_t)c->use_tc_attention};
+    rpo_ctx::StepGraph* sg = nullptr;
+    for (auto& g : c->step_graphs) if (g.key == key) sg = &g;
+    if (!sg) {
+      if (c->step_graphs.size() >= 8) {            // drop the oldest; nothing may still be running from it
+        CUDA_TRY(cudaStreamSynchronize(st));
+        cudaGraphExecDestroy(c->step_graphs.front().exec);
+        c->step_graphs.erase(c->step_graphs.begin());
+      }
+      const int64_t l0 = c->launches;
+      cudaGraph_t graph = nullptr;
+      CUDA_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+      const int rc = enqueue_step();
+      const cudaError_t ce = cudaStreamEndCapture(st, &graph);
+      const int64_t per_step = c->launches - l0;
+      c->launches = l0;
+      if (rc != RPO_OK || ce != cudaSuccess || !graph) { if (graph) cudaGraphDestroy(graph); cudaGetLastError(); return rc != RPO_OK ? rc : RPO_ERR_CUDA; }
+      cudaGraphExec_t exec = nullptr;
+      const cudaError_t ie = cudaGraphInstantiate(&exec, graph, 0);
+      cudaGraphDestroy(graph);
+      if (ie != cudaSuccess) { cudaGetLastError(); return RPO_ERR_CUDA; }
+      c->step_graphs.push_back({key, exec, per_step});
+      sg = &c->step_graphs.back();
+    }
+    for (; j < S; ++j) { CUDA_TRY(cudaGraphLaunch(sg->exec, st)); c->launches += sg->launches; }
   }
+  for (; j < S; ++j) RPO_TRY(enqueue_step());
   CUDA_TRY(cudaMemcpyAsync(d_lens_out, w.lens, (size_t)B * 4, cudaMemcpyDeviceToDevice, st));
   return RPO_OK;
 }

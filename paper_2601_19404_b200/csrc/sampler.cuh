@@ -24,6 +24,8 @@ struct SamplerArgs {
   uint64_t seed;
   const int64_t* seq_ids;     // sequence number per row
   int step;                   // draw number (suffix position)
+  const int32_t* step_ptr;    // non-NULL (decode): step, out_col and last_step come from this device counter
+  int n_steps;                // with step_ptr: the call's number of suffix positions
   int out_stride, out_col;    // outputs land at [r*out_stride + out_col]
   const int32_t* forced;      // NULL or forced tokens, same indexing as outputs
   int32_t* tokens_out;
@@ -107,6 +109,7 @@ __device__ __forceinline__ int select_bucket(const uint64_t* hist, uint64_t targ
 }
 
 __global__ void __launch_bounds__(1024) sampler_kernel(SamplerArgs a) {
+  if (a.step_ptr) { a.step = *a.step_ptr; a.out_col = a.step; a.last_step = (a.step == a.n_steps - 1); }
   __shared__ uint64_t hist[2048];
   __shared__ uint64_t sh[48];
   __shared__ float fred[32];
