@@ -170,6 +170,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override n_layers (reduced case for profiler captures)")
     ap.add_argument("--suffix", type=int, default=0, help="override the suffix length (reduced case for profiler captures)")
     ap.add_argument("--groups", type=int, default=0, help="override the number of prompt groups (reduced case)")
+    ap.add_argument("--kernel-table", action="store_true", help="print per-kernel event timings of one profiled step on stderr")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     args = ap.parse_args()
 
@@ -315,7 +316,7 @@ def main():
     roofline = None
     phases = None
     if not args.no_profile and rank == 0:
-        ctx.set_option("profile", 1)
+        ctx.set_option("profile", 2 if args.kernel_table else 1)
         step()
         prof = ctx.profile_read()
         ctx.set_option("profile", 0)

@@ -7,10 +7,11 @@
 // Three uses:
 //   ROWS   (prefill, teacher-forced log-probs): a tile holds 64 consecutive rows of one sequence
 //          for one query head; output is the normalised attention, written as bf16.
-//   SHARED (decode): a tile holds the G * (Hq/Hkv) query rows of one prompt group that share a KV
-//          head, and one split of the group's prefix; the prefix K/V of a group is therefore read
-//          once per group, not once per sample.  Output: (m, l, unnormalised O) partials.
-//   The per-sequence suffix keys and the split merge are handled by attn_decode_merge_kernel.
+//   SHARED (decode): two kinds of work item in one grid.  A shared item holds the G * (Hq/Hkv) query
+//          rows of one prompt group that share a KV head, and one split of the group's prefix; the
+//          prefix K/V of a group is therefore read once per group, not once per sample.  A private
+//          item holds the Hq/Hkv query rows of one sequence and that sequence's own suffix keys.
+//          Output of both: (m, l, unnormalised O) partials, merged by attn_decode_merge_kernel.
 #pragma once
 #include "kernels.cuh"
 
@@ -22,7 +23,8 @@ enum FlashMode { FA_ROWS = 0, FA_SHARED = 1 };
 struct FlashArgs {
   const bf16* qkv; int qkv_cols;
   bf16* out; int out_cols;
-  float* part_ml; float* part_o; int n_splits; int split_chunk;   // SHARED
+  float* part_ml; float* part_o; int n_splits; int split_chunk;   // SHARED: partial slots 0..n_splits-1 = prefix splits,
+  int n_shared_items; int n_seqs;                                 //         slot n_splits = the sequence's own suffix
   const int32_t* row_seq; const int32_t* row_t; const SeqDesc* seqs; const int32_t* block_table;
   KVPool<bf16> pool; int layer, hq, hkv; float scale_log2;
   const int2* tiles;      // ROWS: (first row, number of rows)
@@ -57,14 +59,15 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 template <int DH, int MODE>
 __global__ void __launch_bounds__(FA_THREADS) flash_attn_kernel(FlashArgs a) {
+  constexpr int NST = (MODE == FA_SHARED) ? 3 : 2;   // K/V ring depth: decode is latency-bound, prefill is not
   constexpr int CH = DH / 8;                 // 16-byte chunks per row
   constexpr int ROW_BYTES = DH * 2;
   constexpr int TILE_BYTES = FA_BN * ROW_BYTES;
   constexpr int KSTEPS = DH / 16, ONT = DH / 8;
   extern __shared__ __align__(128) uint8_t fsm[];
   const uint32_t sQ = (uint32_t)__cvta_generic_to_shared(fsm);
-  const uint32_t sK = sQ + FA_BM * ROW_BYTES;          // 2 buffers
-  const uint32_t sV = sK + 2 * TILE_BYTES;             // 2 buffers
+  const uint32_t sK = sQ + FA_BM * ROW_BYTES;          // NST buffers
+  const uint32_t sV = sK + NST * TILE_BYTES;           // NST buffers
   __shared__ int s_qrow[FA_BM];     // qkv row of each tile row (-1: padding)
   __shared__ int s_head[FA_BM];
   __shared__ int s_t[FA_BM];        // private causal limit (-1: nothing visible / inactive)
@@ -72,6 +75,7 @@ __global__ void __launch_bounds__(FA_THREADS) flash_attn_kernel(FlashArgs a) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
   const int rep = a.hq / a.hkv;
   int kvh, n_rows, split = 0;
+  bool private_item = false;
   SeqDesc sd;
   if (MODE == FA_ROWS) {
     const int2 tile = a.tiles[blockIdx.x];
@@ -84,11 +88,13 @@ __global__ void __launch_bounds__(FA_THREADS) flash_attn_kernel(FlashArgs a) {
       s_head[tid] = head;
       s_t[tid] = v ? a.row_t[tile.x + tid] : -1;
     }
-  } else {
+  } else if ((int)blockIdx.x < a.n_shared_items) {
     const int rows_per_group = a.G * rep;
     const int tiles_per_group = (rows_per_group + FA_BM - 1) / FA_BM;
-    const int grp = blockIdx.x / tiles_per_group, r0 = (blockIdx.x % tiles_per_group) * FA_BM;
-    kvh = blockIdx.y; split = blockIdx.z;
+    const int item = blockIdx.x / a.n_splits;
+    split = blockIdx.x % a.n_splits;
+    const int grp = item / tiles_per_group, r0 = (item % tiles_per_group) * FA_BM;
+    kvh = blockIdx.y;
     n_rows = min(FA_BM, rows_per_group - r0);
     sd = a.seqs[grp * a.G];
     if (tid < FA_BM) {
@@ -98,13 +104,27 @@ __global__ void __launch_bounds__(FA_THREADS) flash_attn_kernel(FlashArgs a) {
       s_head[tid] = kvh * rep + (v ? i % rep : 0);
       s_t[tid] = -1;
     }
+  } else {
+    // private item: the rep query heads of one sequence against its own suffix keys 0..t
+    private_item = true;
+    const int seq = blockIdx.x - a.n_shared_items;
+    kvh = blockIdx.y; split = a.n_splits;
+    n_rows = min(rep, FA_BM);
+    sd = a.seqs[a.row_seq[seq]];
+    const int t = a.row_t[seq];
+    if (tid < FA_BM) {
+      const bool v = tid < n_rows;
+      s_qrow[tid] = v ? seq : -1;
+      s_head[tid] = kvh * rep + (v ? tid : 0);
+      s_t[tid] = v ? t : -1;
+    }
   }
   __syncthreads();
 
   // ---- key ranges
   int sh_begin = 0, sh_end = 0, pr_end = 0;
-  if (MODE == FA_ROWS) {
-    sh_end = (sd.shared_tbl >= 0) ? sd.shared_len : 0;
+  if (MODE == FA_ROWS || private_item) {
+    sh_end = (MODE == FA_ROWS && sd.shared_tbl >= 0) ? sd.shared_len : 0;
     int mt = -1;
     for (int i = 0; i < n_rows; ++i) mt = max(mt, s_t[i]);
     pr_end = mt + 1;
@@ -151,8 +171,11 @@ __global__ void __launch_bounds__(FA_THREADS) flash_attn_kernel(FlashArgs a) {
       if (qp) fa::cp_async16(sQ + sw(lrow, ch), qp + ch * 8); else fa::st_zero16(sQ + sw(lrow, ch));
     }
   }
-  if (n_tiles > 0) load_kv(0, 0);
-  fa::cp_commit();
+#pragma unroll
+  for (int st = 0; st < NST - 1; ++st) {      // prologue: tiles 0..NST-2 (the first group also carries Q)
+    if (st < n_tiles) load_kv(st, st);
+    fa::cp_commit();
+  }
 
   float o[ONT][4];
 #pragma unroll
@@ -163,8 +186,11 @@ __global__ void __launch_bounds__(FA_THREADS) flash_attn_kernel(FlashArgs a) {
   const int t_lo = s_t[r_lo], t_hi = s_t[r_hi];
 
   for (int it = 0; it < n_tiles; ++it) {
-    const int buf = it & 1;
-    if (it + 1 < n_tiles) { load_kv(it + 1, buf ^ 1); fa::cp_commit(); fa::cp_wait<1>(); } else { fa::cp_wait<0>(); }
+    const int buf = it % NST;
+    // tile it+NST-1 goes into the buffer that iteration it-1 finished reading (its trailing barrier)
+    if (it + NST - 1 < n_tiles) load_kv(it + NST - 1, (it + NST - 1) % NST);
+    fa::cp_commit();
+    fa::cp_wait<NST - 1>();                   // all but the newest NST-1 groups have landed: tile `it` is in
     __syncthreads();
     if (it == 0) {
 #pragma unroll
@@ -251,7 +277,7 @@ __global__ void __launch_bounds__(FA_THREADS) flash_attn_kernel(FlashArgs a) {
       for (int i = 0; i < ONT; ++i)
         *(uint32_t*)(dst + i * 8 + tq * 2) = fa::pack_bf16(o[i][half * 2] * inv, o[i][half * 2 + 1] * inv);
     } else {
-      const int64_t slot = ((int64_t)qr * a.hq + s_head[r]) * a.n_splits + split;
+      const int64_t slot = ((int64_t)qr * a.hq + s_head[r]) * (a.n_splits + 1) + split;
       if (tq == 0) { a.part_ml[slot * 2] = m; a.part_ml[slot * 2 + 1] = l; }
       float* dst = a.part_o + slot * DH;
 #pragma unroll
@@ -260,64 +286,34 @@ __global__ void __launch_bounds__(FA_THREADS) flash_attn_kernel(FlashArgs a) {
   }
 }
 
-// Decode: merge the shared-prefix partials of (sequence, query head) with attention over the
-// sequence's own suffix keys 0..t (private blocks), one warp each; lanes own DH/32 dimensions.
+// Decode: log-sum-exp merge of the partials of (sequence, query head) -- slots 0..n_splits-1 from the
+// splits of the shared prefix, slot n_splits from the sequence's own suffix keys -- one warp each;
+// lanes own DH/32 dimensions.  Fixed slot order, hence reproducible.
 template <int DH>
-__global__ void __launch_bounds__(128) attn_decode_merge_kernel(const bf16* __restrict__ qkv, int qkv_cols,
-                                                                bf16* __restrict__ out, const float* __restrict__ part_ml,
-                                                                const float* __restrict__ part_o, int n_splits,
-                                                                const int32_t* __restrict__ row_seq,
-                                                                const int32_t* __restrict__ row_t,
-                                                                const SeqDesc* __restrict__ seqs,
-                                                                const int32_t* __restrict__ block_table,
-                                                                KVPool<bf16> pool, int layer, int rows, int hq, int hkv,
-                                                                float scale_log2, int* status) {
+__global__ void __launch_bounds__(128) attn_decode_merge_kernel(bf16* __restrict__ out, const float* __restrict__ part_ml,
+                                                                const float* __restrict__ part_o, int n_slots,
+                                                                const int32_t* __restrict__ row_t, int rows, int hq) {
   constexpr int DPL = DH / 32;
   const int w = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (w >= rows * hq) return;
   const int r = w / hq, head = w % hq;
   bf16* o = out + (int64_t)r * hq * DH + head * DH + lane * DPL;
-  const int t = row_t[r];
-  if (t < 0) {
-#pragma unroll
-    for (int i = 0; i < DPL; ++i) o[i] = __float2bfloat16_rn(0.f);
-    return;
-  }
-  const SeqDesc sd = seqs[row_seq[r]];
-  const int kvh = head / (hq / hkv);
   float m = -INFINITY, l = 0.f, acc[DPL];
 #pragma unroll
   for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
-  for (int s = 0; s < n_splits; ++s) {
-    const int64_t slot = ((int64_t)r * hq + head) * n_splits + s;
-    const float ms = part_ml[slot * 2], ls = part_ml[slot * 2 + 1];
-    if (ls <= 0.f) continue;
-    const float mn = fmaxf(m, ms), c0 = exp2f(m - mn), c1 = exp2f(ms - mn);
-    l = l * c0 + ls * c1;
+  if (row_t[r] >= 0) {
+    for (int s = 0; s < n_slots; ++s) {
+      const int64_t slot = ((int64_t)r * hq + head) * n_slots + s;
+      const float ms = part_ml[slot * 2], ls = part_ml[slot * 2 + 1];
+      if (!(ls > 0.f)) continue;
+      const float mn = fmaxf(m, ms), c0 = exp2f(m - mn), c1 = exp2f(ms - mn);
+      l = l * c0 + ls * c1;
 #pragma unroll
-    for (int i = 0; i < DPL; ++i) acc[i] = acc[i] * c0 + part_o[slot * DH + lane * DPL + i] * c1;
-    m = mn;
+      for (int i = 0; i < DPL; ++i) acc[i] = acc[i] * c0 + part_o[slot * DH + lane * DPL + i] * c1;
+      m = mn;
+    }
   }
-  const bf16* qp = qkv + (int64_t)r * qkv_cols + head * DH + lane * DPL;
-  float q[DPL];
-#pragma unroll
-  for (int i = 0; i < DPL; ++i) q[i] = __bfloat162float(qp[i]) * scale_log2;
-  for (int u = 0; u <= t; ++u) {
-    const int blk = block_table[sd.priv_tbl + u / KV_BLOCK];
-    if (blk < 0 || blk >= pool.n_blocks) { if (lane == 0) atomicOr(status, STATUS_BAD_BLOCK); continue; }
-    const bf16* kp = pool.at(layer, 0, kvh, blk, u % KV_BLOCK) + lane * DPL;
-    const bf16* vp = pool.at(layer, 1, kvh, blk, u % KV_BLOCK) + lane * DPL;
-    float s = 0.f;
-#pragma unroll
-    for (int i = 0; i < DPL; ++i) s = fmaf(q[i], __bfloat162float(kp[i]), s);
-    s = warp_sum(s);
-    const float mn = fmaxf(m, s), c0 = exp2f(m - mn), p = exp2f(s - mn);
-    l = l * c0 + p;
-#pragma unroll
-    for (int i = 0; i < DPL; ++i) acc[i] = acc[i] * c0 + p * __bfloat162float(vp[i]);
-    m = mn;
-  }
-  const float inv = 1.0f / l;
+  const float inv = (l > 0.f) ? 1.0f / l : 0.f;
 #pragma unroll
   for (int i = 0; i < DPL; ++i) o[i] = __float2bfloat16_rn(acc[i] * inv);
 }

@@ -89,7 +89,7 @@ struct rpo_ctx {
   int attn_mode = 0, attn_tiles = 0, attn_G = 1, attn_groups = 0, attn_splits = 1, attn_split_chunk = 64;
   int pending_splits = 0, pending_rows = 0;   // split-K partials of ws.x not yet reduced
   // optional per-kernel timing: event pairs around every launch, tagged class + 16*phase
-  struct ProfEvent { cudaEvent_t a, b; int tag; };
+  struct ProfEvent { cudaEvent_t a, b; int tag; const char* label; };
   int profile = 0, prof_class = 0, prof_phase = 0;
   std::vector<ProfEvent> prof_events;
   // instantiated CUDA graphs of one decode step, keyed by everything the step's launches depend on

@@ -43,12 +43,12 @@ struct ProfScope {
   ~ProfScope() { c->prof_class = prev; }
 };
 
-static void prof_begin(rpo_ctx* c) {
+static void prof_begin(rpo_ctx* c, const char* label = "gemm_tc_kernel") {
   if (!c->profile) return;
   cudaEvent_t a, b;
   cudaEventCreate(&a); cudaEventCreate(&b);
   cudaEventRecord(a, c->stream);
-  c->prof_events.push_back({a, b, c->prof_class + 16 * c->prof_phase});
+  c->prof_events.push_back({a, b, c->prof_class + 16 * c->prof_phase, label});
 }
 static void prof_end(rpo_ctx* c) {
   if (!c->profile) return;
@@ -57,7 +57,7 @@ static void prof_end(rpo_ctx* c) {
 
 #define LAUNCH(ctx, kern, grid, block, smem, ...)                         \
   do {                                                                    \
-    prof_begin(ctx);                                                      \
+    prof_begin(ctx, #kern);                                               \
     kern<<<(grid), (block), (smem), (ctx)->stream>>>(__VA_ARGS__);        \
     prof_end(ctx);                                                        \
     (ctx)->launches++;                                                    \
@@ -249,7 +249,7 @@ extern "C" int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limit
   ALLOC(w.step_ctr, 16);
   ALLOC(w.seq_ids, (size_t)nseq * 8);
   ALLOC(w.tiles, ((size_t)w.R / FA_BM + nseq + 2) * sizeof(int2));
-  w.attn_part_elems = (size_t)lim->max_seqs * s.n_q_heads * 32 * (dh + 2);
+  w.attn_part_elems = (size_t)lim->max_seqs * s.n_q_heads * 33 * (dh + 2);
   ALLOC(w.attn_part, w.attn_part_elems * 4);
   w.partial_elems = (size_t)c->sm_count * 128 * 256;
   ALLOC(w.partial, w.partial_elems * 4);
@@ -384,7 +384,7 @@ static int rmsnorm(rpo_ctx* c, float* x, const float* g, T* h, int rows) {
 
 template <int DH, int MODE>
 static int launch_flash(rpo_ctx* c, const FlashArgs& a, dim3 grid) {
-  constexpr int smem = (FA_BM + 4 * FA_BN) * DH * 2;
+  constexpr int smem = (FA_BM + 2 * (MODE == FA_SHARED ? 3 : 2) * FA_BN) * DH * 2;
   static bool attr_done = false;
   if (!attr_done) {
     CUDA_TRY(cudaFuncSetAttribute(flash_attn_kernel<DH, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
@@ -405,7 +405,7 @@ static int attention(rpo_ctx* c, int layer, int rows) {
       FlashArgs a;
       memset(&a, 0, sizeof(a));
       a.qkv = (const bf16*)w.qkv; a.qkv_cols = c->qkv_cols; a.out = (bf16*)w.attn; a.out_cols = s.n_q_heads * s.head_dim;
-      a.part_ml = w.attn_part; a.part_o = w.attn_part + (size_t)2 * c->lim.max_seqs * s.n_q_heads * 32;
+      a.part_ml = w.attn_part; a.part_o = w.attn_part + (size_t)2 * c->lim.max_seqs * s.n_q_heads * 33;
       a.row_seq = w.row_seq; a.row_t = w.row_t; a.seqs = (const SeqDesc*)w.seqs; a.block_table = c->d_block_table;
       a.pool = kv_pool<bf16>(c); a.layer = layer; a.hq = s.n_q_heads; a.hkv = s.n_kv_heads;
       a.scale_log2 = scale * 1.4426950408889634f; a.tiles = (const int2*)w.tiles; a.G = c->attn_G; a.status = c->d_status;
@@ -415,15 +415,14 @@ static int attention(rpo_ctx* c, int layer, int rows) {
         return s.head_dim == 128 ? launch_flash<128, FA_ROWS>(c, a, grid) : launch_flash<64, FA_ROWS>(c, a, grid);
       }
       const int rep = s.n_q_heads / s.n_kv_heads;
-      dim3 grid(c->attn_groups * ceil_div(c->attn_G * rep, FA_BM), s.n_kv_heads, c->attn_splits);
+      a.n_shared_items = c->attn_groups * ceil_div(c->attn_G * rep, FA_BM) * c->attn_splits; a.n_seqs = rows;
+      dim3 grid(a.n_shared_items + rows, s.n_kv_heads);
       RPO_TRY((s.head_dim == 128 ? launch_flash<128, FA_SHARED>(c, a, grid) : launch_flash<64, FA_SHARED>(c, a, grid)));
       const int mgrid = ceil_div((int64_t)rows * s.n_q_heads, 4);
       if (s.head_dim == 128)
-        LAUNCH(c, (attn_decode_merge_kernel<128>), mgrid, 128, 0, a.qkv, a.qkv_cols, a.out, a.part_ml, a.part_o, a.n_splits,
-               w.row_seq, w.row_t, a.seqs, a.block_table, a.pool, layer, rows, a.hq, a.hkv, a.scale_log2, c->d_status);
+        LAUNCH(c, (attn_decode_merge_kernel<128>), mgrid, 128, 0, a.out, a.part_ml, a.part_o, a.n_splits + 1, w.row_t, rows, a.hq);
       else
-        LAUNCH(c, (attn_decode_merge_kernel<64>), mgrid, 128, 0, a.qkv, a.qkv_cols, a.out, a.part_ml, a.part_o, a.n_splits,
-               w.row_seq, w.row_t, a.seqs, a.block_table, a.pool, layer, rows, a.hq, a.hkv, a.scale_log2, c->d_status);
+        LAUNCH(c, (attn_decode_merge_kernel<64>), mgrid, 128, 0, a.out, a.part_ml, a.part_o, a.n_splits + 1, w.row_t, rows, a.hq);
       return RPO_OK;
     }
   }
@@ -914,13 +913,22 @@ extern "C" int rpo_profile_read(rpo_ctx* c, double* ms_out, int64_t* count_out, 
   if (!c || !ms_out || !count_out || n < 3 * KC_COUNT) return RPO_ERR_INVALID_ARG;
   CUDA_TRY(cudaStreamSynchronize(c->stream));
   for (int i = 0; i < n; ++i) { ms_out[i] = 0.0; count_out[i] = 0; }
+  std::map<std::string, std::pair<double, int64_t>> by_label;   // option profile = 2: table on stderr
   for (auto& ev : c->prof_events) {
     float ms = 0.f;
     cudaEventElapsedTime(&ms, ev.a, ev.b);
+    if (c->profile >= 2) {
+      static const char* ph[] = {"prefill", "decode", "logprobs", "?"};
+      auto& e = by_label[std::string(ph[std::min(ev.tag / 16, 3)]) + " " + ev.label];
+      e.first += ms; e.second++;
+    }
     const int phase = ev.tag / 16, k = ev.tag % 16;
     if (phase < 3 && k < KC_COUNT) { ms_out[phase * KC_COUNT + k] += ms; count_out[phase * KC_COUNT + k]++; }
     cudaEventDestroy(ev.a); cudaEventDestroy(ev.b);
   }
   c->prof_events.clear();
+  for (auto& kv : by_label)
+    fprintf(stderr, "[rpo profile] %-60s %8lld launches %10.3f ms  %8.2f us/launch\n", kv.first.c_str(),
+            (long long)kv.second.second, kv.second.first, 1e3 * kv.second.first / kv.second.second);
   return RPO_OK;
 }
