@@ -95,7 +95,7 @@ int rpo_shape_preset(const char* name, rpo_shape* out);
 /* Create a context on the current CUDA device: allocates the weight arena, the paged KV
  * pool ([layer][K|V][kv_head][block][16][head_dim]), block tables and workspaces.
  * cuda_stream is a cudaStream_t (may be NULL).  *out is owned by the caller until
- * rpo_destroy.  Errors: RPO_ERR_SHAPE (head_dim not 64/128, d_model or d_ffn not a
+ * rpo_destroy.  Errors: RPO_ERR_SHAPE (vocab >= 2^18, head_dim not 64/128, d_model or d_ffn not a
  * multiple of 8, n_q_heads not a multiple of n_kv_heads, kv_block_tokens != 16),
  * RPO_ERR_CUDA (allocation failed). */
 int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limits* limits, void* cuda_stream);
@@ -176,7 +176,8 @@ int rpo_rollout_host(rpo_ctx* ctx, int32_t n_groups, const int32_t* h_tokens, co
 
 /* The sampler alone, on caller-supplied float32 logits [n_rows, vocab] (row r belongs to
  * sequence d_seq_ids[r], draw number `step`): used to test the sampler in isolation.
- * d_tokens_out int32 [n_rows]; d_logprobs_out NULL or float [n_rows]. */
+ * d_tokens_out int32 [n_rows]; d_logprobs_out NULL or float [n_rows].  Takes n_rows*vocab*4
+ * bytes of stream-ordered temporary device memory for the call. */
 int rpo_sample_rows(rpo_ctx* ctx, int32_t n_rows, int32_t vocab, const float* d_logits, const rpo_sampler* sampler,
                     const int64_t* d_seq_ids, int32_t step, int32_t* d_tokens_out, float* d_logprobs_out);
 

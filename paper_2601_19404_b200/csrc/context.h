@@ -39,6 +39,8 @@ struct Workspace {
   float* xh = nullptr;     // [HR, d] head input rows
   void* hh = nullptr;      // [HR, d]
   float* logits = nullptr; // [HR, V]
+  uint32_t* sampler_w = nullptr;  // [max(max_seqs, max_groups), V] quantised sampler weights
+  size_t sampler_w_rows = 0;
   float* partial = nullptr;      // split-K partial sums
   size_t partial_elems = 0;
   float* attn_part = nullptr;    // decode attention partials

@@ -146,6 +146,7 @@ extern "C" int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limit
   const rpo_shape& s = *shape;
   if (s.n_layers < 0 || s.d_model <= 0 || s.n_q_heads <= 0 || s.n_kv_heads <= 0 || s.d_ffn <= 0 || s.vocab <= 0)
     return RPO_ERR_SHAPE;
+  if (s.vocab >= (1 << 18)) return RPO_ERR_SHAPE;   // sampler mass histograms: 14-bit pieces summed in 32 bits
   if ((s.head_dim != 64 && s.head_dim != 128) || s.n_q_heads % s.n_kv_heads || s.kv_block_tokens != KV_BLOCK ||
       s.d_model % 8 || s.d_ffn % 8 || (s.dtype != RPO_DTYPE_FP32 && s.dtype != RPO_DTYPE_BF16) || s.rms_eps < 0)
     return RPO_ERR_SHAPE;
@@ -241,6 +242,8 @@ extern "C" int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limit
   ALLOC(w.row_tok, (size_t)w.R * 4);
   const int nseq = std::max(lim->max_seqs, lim->max_groups);
   ALLOC(w.seqs, (size_t)nseq * sizeof(SeqDesc));
+  w.sampler_w_rows = nseq;
+  ALLOC(w.sampler_w, (size_t)nseq * V * 4);
   ALLOC(w.done, (size_t)nseq * 4);
   ALLOC(w.lens, (size_t)nseq * 4);
   ALLOC(w.cur_tok, (size_t)nseq * 4);
@@ -598,6 +601,17 @@ extern "C" int rpo_release_groups(rpo_ctx* c, int32_t n_groups, const rpo_group*
 // ---------------------------------------------------------------------------------------------
 // decode
 // ---------------------------------------------------------------------------------------------
+static int launch_sampler(rpo_ctx* c, int n_rows, const SamplerArgs& a) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    CUDA_TRY(cudaFuncSetAttribute(sampler_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SAMPLER_SMEM));
+    attr_done = true;
+  }
+  ProfScope ps(c, KC_SAMPLER);
+  LAUNCH(c, sampler_kernel, n_rows, 1024, SAMPLER_SMEM, a);
+  return RPO_OK;
+}
+
 static SamplerArgs sampler_args(rpo_ctx* c, const rpo_sampler* sp) {
   SamplerArgs a;
   memset(&a, 0, sizeof(a));
@@ -605,6 +619,7 @@ static SamplerArgs sampler_args(rpo_ctx* c, const rpo_sampler* sp) {
   a.temperature = sp->temperature;
   a.top_p24 = (uint32_t)floorf(sp->top_p * 16777216.0f);
   a.greedy = sp->greedy; a.eos_id = sp->eos_id; a.seed = sp->seed;
+  a.weights = c->ws.sampler_w;
   return a;
 }
 
@@ -669,7 +684,7 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
          n_groups, d);
   RPO_TRY(head<T>(c, n_groups));
   a.logit_row = w.logit_row;
-  { ProfScope ps(c, KC_SAMPLER); LAUNCH(c, sampler_kernel, B, 1024, 0, a); }
+  RPO_TRY(launch_sampler(c, B, a));
   a.logit_row = nullptr;
   // steps 1..S-1 are one and the same launch sequence (the step number lives on the device):
   // the first runs eagerly, the others replay a CUDA graph of it.
@@ -679,7 +694,7 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
     RPO_TRY(run_layers<T>(c, B));
     CUDA_TRY(cudaMemcpyAsync(w.xh, w.x, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, st));
     RPO_TRY(head<T>(c, B));
-    { ProfScope ps(c, KC_SAMPLER); LAUNCH(c, sampler_kernel, B, 1024, 0, a); }
+    RPO_TRY(launch_sampler(c, B, a));
     return RPO_OK;
   };
   int j = 1;
@@ -865,14 +880,19 @@ extern "C" int rpo_rollout_host(rpo_ctx* c, int32_t n_groups, const int32_t* h_t
 // ---------------------------------------------------------------------------------------------
 extern "C" int rpo_sample_rows(rpo_ctx* c, int32_t n_rows, int32_t vocab, const float* d_logits, const rpo_sampler* sp,
                                const int64_t* d_seq_ids, int32_t step, int32_t* d_tokens_out, float* d_logprobs_out) {
-  if (!c || n_rows < 0 || vocab <= 0 || !d_logits || !d_seq_ids || !d_tokens_out || step < 0) return RPO_ERR_INVALID_ARG;
+  if (!c || n_rows < 0 || vocab <= 0 || vocab >= (1 << 18) || !d_logits || !d_seq_ids || !d_tokens_out || step < 0) return RPO_ERR_INVALID_ARG;
   RPO_TRY(check_sampler(sp));
   if (n_rows == 0) return RPO_OK;
   SamplerArgs a = sampler_args(c, sp);
   a.V = vocab; a.logits = d_logits; a.seq_ids = d_seq_ids; a.step = step; a.out_stride = 1; a.out_col = 0;
   a.tokens_out = d_tokens_out; a.logprobs_out = d_logprobs_out; a.eos_id = -1;
-  LAUNCH(c, sampler_kernel, n_rows, 1024, 0, a);
-  return RPO_OK;
+  // This test entry takes any vocabulary: its weight scratch is a stream-ordered temporary.
+  void* tmp = nullptr;
+  CUDA_TRY(cudaMallocAsync(&tmp, (size_t)n_rows * vocab * 4, c->stream));
+  a.weights = (uint32_t*)tmp;
+  const int rc = launch_sampler(c, n_rows, a);
+  CUDA_TRY(cudaFreeAsync(tmp, c->stream));
+  return rc;
 }
 
 extern "C" int rpo_gemm(rpo_ctx* c, int32_t impl, int32_t M, int32_t N, int32_t K, const void* d_A, const void* d_W,
