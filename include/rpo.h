@@ -188,6 +188,15 @@ int rpo_sample_rows(rpo_ctx* ctx, int32_t n_rows, int32_t vocab, const float* d_
 int rpo_gemm(rpo_ctx* ctx, int32_t impl, int32_t M, int32_t N, int32_t K, const void* d_A, const void* d_W,
              float* d_C);
 
+/* Kernel micro-benchmark (bf16 contexts): the tensor-core GEMM of C[M,N] = A[M,K] W^T as the layers
+ * launch it (planner or its "gemm_bn"/"gemm_splits" override; split-K planes are left unreduced),
+ * `iters` launches cycling through the n_w weight matrices of h_W_list (host array of device
+ * pointers; use enough matrices to exceed the L2 capacity), replayed as one CUDA graph.  The output
+ * goes to an internal buffer.  *h_ms_out = mean device time per launch in milliseconds.
+ * Synchronises the stream.  RPO_ERR_LIMIT if M*N exceeds the internal logits buffer. */
+int rpo_gemm_bench(rpo_ctx* ctx, int32_t M, int32_t N, int32_t K, const void* d_A, const void* const* h_W_list,
+                   int32_t n_w, int32_t iters, float* h_ms_out);
+
 /* Device status word, sticky until read: 0 = clean; bit 0 = a bounded wait expired
  * (TMA / MMA pipeline), bit 1 = token id out of range (clamped), bit 2 = block-table
  * index out of range (access skipped).  Synchronises the stream; *out receives the word
@@ -199,7 +208,9 @@ int rpo_counters(rpo_ctx* ctx, int64_t* kernel_launches, int64_t* free_kv_blocks
 
 /* Runtime switches (tests/benchmarks): name = "use_tcgen05" (bf16 GEMMs on the tensor-core
  * kernel, default 1), "use_tc_attention" (tensor-core attention kernels, default 1),
- * "use_graph" (CUDA graph per decode step, default 1), "profile" (see rpo_profile_read). */
+ * "use_graph" (CUDA graph per decode step, default 1), "profile" (see rpo_profile_read),
+ * "gemm_bn" (0 = planner, else force the tensor-core tile width: 32/64/96/128/256) and
+ * "gemm_splits" (with gemm_bn: force the split-K factor where the caller can reduce planes). */
 int rpo_set_option(rpo_ctx* ctx, const char* name, int32_t value);
 
 /* Per-kernel timing.  With option "profile" = 1 every kernel launch is bracketed by a pair of

@@ -14,7 +14,7 @@ _LIB = None
 EXPORTED_SYMBOLS = [
     "rpo_strerror", "rpo_shape_preset", "rpo_create", "rpo_destroy", "rpo_init_weights", "rpo_read_tensor",
     "rpo_write_tensor", "rpo_prefill_prefix", "rpo_decode_suffix", "rpo_token_logprobs", "rpo_release_groups",
-    "rpo_rollout_host", "rpo_sample_rows", "rpo_gemm", "rpo_device_status", "rpo_counters", "rpo_set_option", "rpo_profile_read",
+    "rpo_rollout_host", "rpo_sample_rows", "rpo_gemm", "rpo_gemm_bench", "rpo_device_status", "rpo_counters", "rpo_set_option", "rpo_profile_read",
 ]
 
 
@@ -72,6 +72,7 @@ def load_library(path=None):
     lib.rpo_rollout_host.argtypes = [vp, i32, vp, vp, vp, i32, i32, C.POINTER(Sampler), vp, vp, vp, i32, vp]
     lib.rpo_sample_rows.argtypes = [vp, i32, i32, vp, C.POINTER(Sampler), vp, i32, vp, vp]
     lib.rpo_gemm.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp]
+    lib.rpo_gemm_bench.argtypes = [vp, i32, i32, i32, vp, C.POINTER(vp), i32, i32, C.POINTER(f32)]
     lib.rpo_device_status.argtypes = [vp, C.POINTER(i32)]
     lib.rpo_counters.argtypes = [vp, C.POINTER(i64), C.POINTER(i64)]
     lib.rpo_set_option.argtypes = [vp, C.c_char_p, i32]
@@ -220,6 +221,16 @@ class Context:
         M, K = d_A.shape
         N = d_W.shape[0]
         _check(self.lib.rpo_gemm(self.handle, int(impl), M, N, K, _ptr(d_A), _ptr(d_W), _ptr(d_C)), "rpo_gemm")
+
+    def gemm_bench(self, d_A, d_W_list, iters):
+        """Mean device milliseconds per launch of the tensor-core GEMM A W^T, cycling through d_W_list."""
+        M, K = d_A.shape
+        N = d_W_list[0].shape[0]
+        ptrs = (C.c_void_p * len(d_W_list))(*[w.data_ptr() for w in d_W_list])
+        ms = C.c_float()
+        _check(self.lib.rpo_gemm_bench(self.handle, M, N, K, _ptr(d_A), ptrs, len(d_W_list), int(iters), C.byref(ms)),
+               "rpo_gemm_bench")
+        return ms.value
 
     def device_status(self):
         v = C.c_int32()

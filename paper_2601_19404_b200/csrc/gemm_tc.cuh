@@ -119,7 +119,7 @@ struct TcCfg {
   static constexpr int B_BYTES = BN * TC_BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int NS = (200 * 1024 / STAGE_BYTES) > 8 ? 8 : (200 * 1024 / STAGE_BYTES);
-  static constexpr int TMEM_COLS = (2 * BN < 32) ? 32 : 2 * BN;
+  static constexpr int TMEM_COLS = (2 * BN <= 32) ? 32 : (2 * BN <= 64) ? 64 : (2 * BN <= 128) ? 128 : (2 * BN <= 256) ? 256 : 512;   // power of two
   static constexpr int SMEM_BYTES = NS * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
 };
 
@@ -375,31 +375,62 @@ inline int tc_launch_epi(rpo_ctx* c, int epi, const CUtensorMap* ma, const CUten
   }
 }
 
-// Plan and launch.  `splits_out` (optional) receives the number of split-K planes written to
-// ws.partial when the epilogue had to become TC_PARTIAL (only for TC_ADD_F32 requests with
-// allow_split): the caller then owns the reduction.
+// Tile width and split-K factor.  Two regimes:
+//   * many row tiles (prefill, log-probs): tensor-bound; 256-wide tiles.
+//   * few row tiles (decode): the launch streams the weight matrix once from HBM, so every SM must
+//     be pulling weights all the time.  If 128-wide tiles alone give about one item per SM, use
+//     them unsplit; otherwise (tile_n, k-split) items are sized by a small cost model fitted to
+//     measurements: cost of an item ~ k-blocks x (W rows + a share for the A tile re-read from L2)
+//     + a pipeline-fill term, cost of the launch = rounds x item cost + a term per split plane
+//     (partials written and re-read by the reducing kernel).
+struct TcPlan { int bn, splits, kb_per_split; };
+
+inline TcPlan tc_plan(rpo_ctx* c, int M, int N, int K, int epi, bool allow_split) {
+  const int sms = c->sm_count, tiles_m = (M + TC_BM - 1) / TC_BM, kb_total = K / TC_BK;
+  TcPlan best{256, 1, kb_total};
+  if (c->gemm_bn > 0) {                                  // test / sweep override
+    best.bn = c->gemm_bn;
+    best.splits = (allow_split && c->gemm_splits > 0) ? std::min(c->gemm_splits, kb_total) : 1;
+  } else if (tiles_m * ((N + 255) / 256) >= sms && tiles_m >= 4) {
+    best.bn = 256;
+  } else if (tiles_m * ((N + 127) / 128) * 20 >= sms * 17) {
+    best.bn = 128;                                       // enough 128-wide tiles for every SM: no split
+  } else {
+    static const int widths[] = {128, 96, 64, 32};
+    double best_cost = 1e30;
+    for (int bn : widths) {
+      if (epi == TC_SWIGLU && bn % 32) continue;
+      const int tiles = tiles_m * ((N + bn - 1) / bn);
+      int max_splits = 1;
+      if (allow_split && tiles < sms) max_splits = std::max(1, std::min(sms / tiles, kb_total / 2));
+      for (int sp = 1; sp <= max_splits; ++sp) {
+        const int kbs = (kb_total + sp - 1) / sp;
+        const int real = (kb_total + kbs - 1) / kbs;
+        if (real > 1 && (size_t)real * M * N > c->ws.partial_elems) continue;
+        const int rounds = (tiles * real + sms - 1) / sms;
+        const double cost = (double)rounds * (kbs * (bn + 40.0) + 600.0) + (real > 1 ? 60.0 * real : 0.0);
+        if (cost < best_cost) { best_cost = cost; best.bn = bn; best.splits = real; }
+      }
+    }
+  }
+  best.kb_per_split = (kb_total + best.splits - 1) / best.splits;
+  best.splits = (kb_total + best.kb_per_split - 1) / best.kb_per_split;
+  if (best.splits > 1 && (size_t)best.splits * M * N > c->ws.partial_elems) { best.splits = 1; best.kb_per_split = kb_total; }
+  return best;
+}
+
+// Plan and launch.  With allow_split the launch may write split-K partial planes [splits][M][N]
+// (float32) to ws.partial instead of applying `epi`; `splits_out` then receives the number of
+// planes (> 1) and the caller owns the reduction and the epilogue.
 inline int tc_gemm_launch(rpo_ctx* c, const bf16* A, const bf16* W, void* C, int M, int N, int K, int epi, int ldc,
                           bool allow_split, int* splits_out) {
   if (splits_out) *splits_out = 0;
   const int tiles_m = (M + TC_BM - 1) / TC_BM;
   const int kb_total = K / TC_BK;
   const int sms = c->sm_count;
-  // tile width: widest tile that still yields about one wave of CTAs
-  int bn = 256;
-  if (epi == TC_SWIGLU && bn > 128 && tiles_m * ((N + 255) / 256) < sms) bn = 128;
-  while (bn > 32 && tiles_m * ((N + bn - 1) / bn) < sms) bn >>= 1;
-  if (bn > 64 && tiles_m * ((N + bn - 1) / bn) < 2 * sms && tiles_m * ((N + bn / 2 - 1) / (bn / 2)) <= sms) bn >>= 1;
-  int tiles_n = (N + bn - 1) / bn;
-  int splits = 1;
-  if (allow_split && epi == TC_ADD_F32) {
-    const int tiles = tiles_m * tiles_n;
-    if (tiles < sms) {
-      splits = std::min(std::max(1, sms / tiles), std::max(1, kb_total / 4));
-      while (splits > 1 && (size_t)splits * M * N > c->ws.partial_elems) --splits;
-    }
-  }
-  const int kb_per_split = (kb_total + splits - 1) / splits;
-  splits = (kb_total + kb_per_split - 1) / kb_per_split;
+  const TcPlan plan = tc_plan(c, M, N, K, epi, allow_split);
+  const int bn = plan.bn, splits = plan.splits, kb_per_split = plan.kb_per_split;
+  const int tiles_n = (N + bn - 1) / bn;
   TcParams p;
   p.C = C; p.M = M; p.N = N; p.K = K; p.ldc = ldc;
   p.tiles_m = tiles_m; p.tiles_n = tiles_n; p.splits = splits; p.kb_per_split = kb_per_split; p.kb_total = kb_total;
@@ -413,8 +444,10 @@ inline int tc_gemm_launch(rpo_ctx* c, const bf16* A, const bf16* W, void* C, int
   switch (bn) {
     case 256: return tc_launch_epi<256>(c, use_epi, ma, mw, p, grid);
     case 128: return tc_launch_epi<128>(c, use_epi, ma, mw, p, grid);
+    case 96: return tc_launch_epi<96>(c, use_epi, ma, mw, p, grid);
     case 64: return tc_launch_epi<64>(c, use_epi, ma, mw, p, grid);
-    default: return tc_launch_epi<32>(c, use_epi, ma, mw, p, grid);
+    case 32: return tc_launch_epi<32>(c, use_epi, ma, mw, p, grid);
+    default: return RPO_ERR_INVALID_ARG;
   }
 }
 

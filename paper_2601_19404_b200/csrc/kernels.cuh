@@ -161,11 +161,15 @@ __global__ void reduce_partials_kernel(float* __restrict__ x, const float* __res
 
 // RoPE (rotate-half) on q and k, then K/V written to the row's slot of its private segment.
 // qkv row layout: [q heads | k heads | v heads] x head_dim.  Grid: (rows, Hq + 2*Hkv).
+// With `partial` the projection arrives as n_splits split-K planes [rows, qkv_cols] of float32:
+// they are summed in plane order and rounded to the storage type first, exactly what the
+// unsplit GEMM epilogue would have stored.
 template <typename T>
 __global__ void rope_kv_kernel(T* __restrict__ qkv, const int32_t* __restrict__ row_seq,
                                const int32_t* __restrict__ row_t, const SeqDesc* __restrict__ seqs,
                                const int32_t* __restrict__ block_table, const float2* __restrict__ rope_tab,
-                               KVPool<T> pool, int layer, int rows, int hq, int hkv, int max_pos, int* status) {
+                               KVPool<T> pool, int layer, int rows, int hq, int hkv, int max_pos, int* status,
+                               const float* __restrict__ partial, int n_splits, int64_t split_stride) {
   const int r = blockIdx.x, head = blockIdx.y;
   if (r >= rows) return;
   const int t = row_t[r];
@@ -174,7 +178,14 @@ __global__ void rope_kv_kernel(T* __restrict__ qkv, const int32_t* __restrict__ 
   const SeqDesc sd = seqs[row_seq[r]];
   const int pos = sd.shared_len + t;
   if (pos >= max_pos) { if (threadIdx.x == 0) atomicOr(status, STATUS_BAD_BLOCK); return; }
-  T* src = qkv + (int64_t)r * (hq + 2 * hkv) * dh + (int64_t)head * dh;
+  const int64_t off = (int64_t)r * (hq + 2 * hkv) * dh + (int64_t)head * dh;
+  T* src = qkv + off;
+  auto ld = [&](int i) -> float {
+    if (!partial) return to_f32(src[i]);
+    float v = 0.f;
+    for (int s = 0; s < n_splits; ++s) v += partial[s * split_stride + off + i];
+    return to_f32(from_f32<T>(v));
+  };
   T* dst = nullptr;
   if (head >= hq) {
     const int kv = (head - hq) / hkv, kh = (head - hq) % hkv;
@@ -185,12 +196,12 @@ __global__ void rope_kv_kernel(T* __restrict__ qkv, const int32_t* __restrict__ 
   if (head < hq + hkv) {  // q or k: rotate
     for (int i = threadIdx.x; i < half; i += blockDim.x) {
       const float2 cs = rope_tab[(int64_t)pos * half + i];
-      const float a = to_f32(src[i]), b = to_f32(src[i + half]);
+      const float a = ld(i), b = ld(i + half);
       const T o1 = from_f32<T>(a * cs.x - b * cs.y), o2 = from_f32<T>(b * cs.x + a * cs.y);
       if (dst) { dst[i] = o1; dst[i + half] = o2; } else { src[i] = o1; src[i + half] = o2; }
     }
   } else {
-    for (int i = threadIdx.x; i < dh; i += blockDim.x) dst[i] = src[i];
+    for (int i = threadIdx.x; i < dh; i += blockDim.x) dst[i] = from_f32<T>(ld(i));
   }
 }
 

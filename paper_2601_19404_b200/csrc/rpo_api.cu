@@ -346,9 +346,13 @@ static int flush_partials(rpo_ctx* c) {
 
 // C = A W^T with the chosen epilogue.  impl: 0 auto, 1 CUDA cores, 2 tcgen05.
 // EPI_SWIGLU is only valid on the tensor-core path (callers check tc_gemm_supported first).
+// allow_split: the tensor-core kernel may leave split-K partial planes in ws.partial instead of
+// applying the epilogue.  For EPI_ADD_F32 on ws.x the next RMSNorm (or flush_partials) folds them
+// in; for other epilogues the caller must pass splits_out and reduce the planes itself.
 template <typename T>
 static int gemm(rpo_ctx* c, const T* A, const T* W, void* C, int M, int N, int K, int epi, int impl = 0,
-                bool allow_split = false) {
+                bool allow_split = false, int* splits_out = nullptr) {
+  if (splits_out) *splits_out = 0;
   if (M <= 0) return RPO_OK;
   ProfScope ps(c, KC_GEMM);
   if (impl != 1 && tc_gemm_supported<T>(c, M, N, K) && (impl == 2 || c->use_tcgen05)) {
@@ -357,10 +361,13 @@ static int gemm(rpo_ctx* c, const T* A, const T* W, void* C, int M, int N, int K
     int splits = 0;
     prof_begin(c);
     const int rc = tc_gemm_launch(c, (const bf16*)A, (const bf16*)W, C, M, N, K, tc_epi, tc_epi == TC_SWIGLU ? N / 2 : N,
-                                  allow_split, &splits);
+                                  allow_split && (epi == EPI_ADD_F32 || splits_out), &splits);
     prof_end(c);
     c->launches++;
-    if (rc == RPO_OK && splits > 1) { c->pending_splits = splits; c->pending_rows = M; }
+    if (rc == RPO_OK && splits > 1) {
+      if (epi == EPI_ADD_F32) { c->pending_splits = splits; c->pending_rows = M; }
+      else *splits_out = splits;
+    }
     return rc;
   }
   if (impl == 2 || epi == EPI_SWIGLU) return RPO_ERR_SHAPE;
@@ -465,11 +472,13 @@ static int run_layers(rpo_ctx* c, int rows) {
   for (int l = 0; l < s.n_layers; ++l) {
     const LayerWeights& L = c->layers[l];
     RPO_TRY(rmsnorm<T>(c, w.x, L.g1, (T*)w.h, rows));
-    RPO_TRY(gemm<T>(c, (const T*)w.h, (const T*)L.wqkv, w.qkv, rows, c->qkv_cols, d, EPI_STORE_T));
+    int qkv_splits = 0;
+    RPO_TRY(gemm<T>(c, (const T*)w.h, (const T*)L.wqkv, w.qkv, rows, c->qkv_cols, d, EPI_STORE_T, 0, true, &qkv_splits));
     { ProfScope ps(c, KC_ROPE);
     LAUNCH(c, rope_kv_kernel<T>, dim3(rows, s.n_q_heads + 2 * s.n_kv_heads), 64, 0, (T*)w.qkv, w.row_seq, w.row_t,
            (const SeqDesc*)w.seqs, c->d_block_table, (const float2*)c->d_rope, kv_pool<T>(c), l, rows, s.n_q_heads,
-           s.n_kv_heads, c->lim.max_positions, c->d_status); }
+           s.n_kv_heads, c->lim.max_positions, c->d_status, qkv_splits > 1 ? (const float*)w.partial : (const float*)nullptr,
+           qkv_splits, (int64_t)rows * c->qkv_cols); }
     RPO_TRY(attention<T>(c, l, rows));
     RPO_TRY(gemm<T>(c, (const T*)w.attn, (const T*)L.wo, w.x, rows, d, qo, EPI_ADD_F32, 0, true));
     RPO_TRY(rmsnorm<T>(c, w.x, L.g2, (T*)w.h, rows));
@@ -898,8 +907,54 @@ extern "C" int rpo_sample_rows(rpo_ctx* c, int32_t n_rows, int32_t vocab, const 
 extern "C" int rpo_gemm(rpo_ctx* c, int32_t impl, int32_t M, int32_t N, int32_t K, const void* d_A, const void* d_W,
                         float* d_C) {
   if (!c || M < 0 || N <= 0 || K <= 0 || !d_A || !d_W || !d_C || impl < 0 || impl > 2) return RPO_ERR_INVALID_ARG;
-  return c->bf16 ? gemm<bf16>(c, (const bf16*)d_A, (const bf16*)d_W, d_C, M, N, K, EPI_STORE_F32, impl)
-                 : gemm<float>(c, (const float*)d_A, (const float*)d_W, d_C, M, N, K, EPI_STORE_F32, impl);
+  int splits = 0;
+  RPO_TRY(c->bf16 ? gemm<bf16>(c, (const bf16*)d_A, (const bf16*)d_W, d_C, M, N, K, EPI_STORE_F32, impl, true, &splits)
+                  : gemm<float>(c, (const float*)d_A, (const float*)d_W, d_C, M, N, K, EPI_STORE_F32, impl));
+  if (splits > 1) {                       // the planner (or its override) split K: reduce the planes into C
+    const int64_t n = (int64_t)M * N;     // N % 16 == 0 on this path
+    CUDA_TRY(cudaMemsetAsync(d_C, 0, (size_t)n * 4, c->stream));
+    LAUNCH(c, reduce_partials_kernel, grid_for(n / 4, 256), 256, 0, d_C, (const float*)c->ws.partial, splits, n, n);
+  }
+  return RPO_OK;
+}
+
+extern "C" int rpo_gemm_bench(rpo_ctx* c, int32_t M, int32_t N, int32_t K, const void* d_A, const void* const* h_W_list,
+                              int32_t n_w, int32_t iters, float* h_ms_out) {
+  if (!c || !c->bf16 || M <= 0 || N <= 0 || K <= 0 || !d_A || !h_W_list || n_w <= 0 || iters <= 0 || !h_ms_out)
+    return RPO_ERR_INVALID_ARG;
+  if (!tc_gemm_supported<bf16>(c, M, N, K)) return RPO_ERR_SHAPE;
+  if ((size_t)M * N > (size_t)c->ws.HR * c->shape.vocab) return RPO_ERR_LIMIT;   // output lands in ws.logits
+  cudaStream_t st = c->stream;
+  auto enqueue = [&]() -> int {
+    for (int i = 0; i < iters; ++i) {
+      int splits = 0;
+      RPO_TRY(tc_gemm_launch(c, (const bf16*)d_A, (const bf16*)h_W_list[i % n_w], c->ws.logits, M, N, K, TC_STORE_F32, N,
+                             true, &splits));
+    }
+    return RPO_OK;
+  };
+  RPO_TRY(enqueue());                                   // warm-up: attributes, tensor maps
+  cudaGraph_t graph = nullptr; cudaGraphExec_t exec = nullptr;
+  CUDA_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+  const int rc = enqueue();
+  const cudaError_t ce = cudaStreamEndCapture(st, &graph);
+  if (rc != RPO_OK || ce != cudaSuccess) { if (graph) cudaGraphDestroy(graph); cudaGetLastError(); return rc != RPO_OK ? rc : RPO_ERR_CUDA; }
+  const cudaError_t ie = cudaGraphInstantiate(&exec, graph, 0);
+  cudaGraphDestroy(graph);
+  if (ie != cudaSuccess) { cudaGetLastError(); return RPO_ERR_CUDA; }
+  cudaEvent_t e0, e1;
+  cudaEventCreate(&e0); cudaEventCreate(&e1);
+  cudaGraphLaunch(exec, st);
+  cudaEventRecord(e0, st);
+  cudaGraphLaunch(exec, st);
+  cudaEventRecord(e1, st);
+  const cudaError_t se = cudaStreamSynchronize(st);
+  float ms = 0.f;
+  cudaEventElapsedTime(&ms, e0, e1);
+  cudaEventDestroy(e0); cudaEventDestroy(e1); cudaGraphExecDestroy(exec);
+  if (se != cudaSuccess) return RPO_ERR_CUDA;
+  *h_ms_out = ms / iters;
+  return RPO_OK;
 }
 
 extern "C" int rpo_device_status(rpo_ctx* c, int32_t* out) {
@@ -924,6 +979,8 @@ extern "C" int rpo_set_option(rpo_ctx* c, const char* name, int32_t value) {
   if (!strcmp(name, "use_tcgen05")) c->use_tcgen05 = value;
   else if (!strcmp(name, "use_tc_attention")) c->use_tc_attention = value;
   else if (!strcmp(name, "use_graph")) c->use_graph = value;
+  else if (!strcmp(name, "gemm_bn")) { if (value != 0 && value != 32 && value != 64 && value != 96 && value != 128 && value != 256) return RPO_ERR_INVALID_ARG; c->gemm_bn = value; }
+  else if (!strcmp(name, "gemm_splits")) c->gemm_splits = value;
   else if (!strcmp(name, "profile")) c->profile = value;
   else return RPO_ERR_INVALID_ARG;
   return RPO_OK;

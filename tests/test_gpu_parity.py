@@ -300,3 +300,40 @@ def test_tensor_core_gemm_against_numpy():
         with pytest.raises(rpo.RpoError):
             ctx.gemm(torch.zeros((8, 72), dtype=torch.bfloat16, device=DEV), torch.zeros((16, 72), dtype=torch.bfloat16, device=DEV),
                      torch.zeros((8, 16), dtype=torch.float32, device=DEV), impl=2)      # K % 64 != 0
+
+
+def _sampled_gemm_error(dA, dW, dC, n_samples, rng):
+    """max |C - A W^T| over randomly sampled outputs, the reference dot products in float64 on the host."""
+    M, K = dA.shape
+    N = dW.shape[0]
+    mi = rng.integers(0, M, n_samples); ni = rng.integers(0, N, n_samples)
+    a = dA[torch.from_numpy(mi).to(DEV)].float().cpu().numpy().astype(np.float64)
+    w = dW[torch.from_numpy(ni).to(DEV)].float().cpu().numpy().astype(np.float64)
+    ref = np.einsum("ik,ik->i", a, w)
+    got = dC[torch.from_numpy(mi).to(DEV), torch.from_numpy(ni).to(DEV)].cpu().numpy()
+    return float(np.max(np.abs(got - ref)))
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 17920, 1536), (256, 152064, 3584), (512, 1536, 8960), (4096, 4608, 3584)],
+                         ids=["decode_gate_up_1p5b", "decode_lm_head_7b", "decode_down_1p5b_B512", "prefill_qkv_7b"])
+def test_tensor_core_gemm_full_size_every_tile_width_and_split(M, N, K):
+    """The GEMM at the sizes the benchmark configurations launch it with, for every tile width and
+    several split-K factors the planner may choose (many work items per persistent CTA), checked on
+    sampled outputs, plus the planner's own choice."""
+    rng = np.random.default_rng(11)
+    shape = dict(SMALL_BF16)
+    gen = torch.Generator(device=DEV); gen.manual_seed(5)
+    dA = torch.randn((M, K), device=DEV, generator=gen).to(torch.bfloat16)
+    dW = (torch.randn((N, K), device=DEV, generator=gen) * 0.05).to(torch.bfloat16)
+    with make_ctx(shape, 1, 1, 32, 4) as ctx:
+        for bn, splits in [(0, 0), (256, 1), (128, 1), (96, 1), (64, 1), (32, 1), (128, 4), (64, 3), (256, 2)]:
+            ctx.set_option("gemm_bn", bn); ctx.set_option("gemm_splits", splits)
+            dC = torch.full((M, N), 777.0, dtype=torch.float32, device=DEV)
+            ctx.gemm(dA, dW, dC, impl=2)
+            torch.cuda.synchronize()
+            assert ctx.device_status() == 0
+            err = _sampled_gemm_error(dA, dW, dC, 4000, rng)
+            assert err < 2e-5 * K ** 0.5, (bn, splits, err)
+            # edges of the output: first/last rows and columns are written
+            assert float(dC[0, 0]) != 777.0 and float(dC[M - 1, N - 1]) != 777.0 and float(dC[M - 1, 0]) != 777.0
+            del dC
