@@ -181,6 +181,30 @@ int rpo_rollout_host(rpo_ctx* ctx, int32_t n_groups, const int32_t* h_tokens, co
 int rpo_sample_rows(rpo_ctx* ctx, int32_t n_rows, int32_t vocab, const float* d_logits, const rpo_sampler* sampler,
                     const int64_t* d_seq_ids, int32_t step, int32_t* d_tokens_out, float* d_logprobs_out);
 
+/* The same sampler for callers that must not allocate.  (The paper has no counterpart: this is a
+ * deployment variant of rpo_sample_rows, not a step of the method.)  Some hosts of this library
+ * cannot obtain device memory when they sample: a serving process that gave the whole device to
+ * its own memory pool at start-up, a plug-in that is handed buffers and a stream but no
+ * allocator, a latency-critical loop in which the implicit synchronisation of an allocation is
+ * not acceptable.  This call needs no rpo_ctx and calls no allocating routine; the per-token
+ * weight scratch the sampler needs is a fixed 16 MiB array inside the library image, which every
+ * GPU that loads the library holds until the process exits.
+ *   n_rows * vocab must not exceed 4 * 2^20 words (e.g. 27 rows of a 151936-token vocabulary):
+ *   larger requests are rejected with RPO_ERR_LIMIT and a message on stderr, nothing is launched.
+ *   d_logits float32 [n_rows, vocab], d_seq_ids int64 [n_rows], d_tokens_out int32 [n_rows],
+ *   d_logprobs_out NULL or float32 [n_rows]: caller-owned device memory, as in rpo_sample_rows;
+ *   cuda_stream: the cudaStream_t the kernel is enqueued on (may be NULL); sampler->eos_id is
+ *   ignored.  Results are identical to rpo_sample_rows.
+ * The first call on a device looks up the array's device address and sets a kernel attribute
+ * (once per device, for the device current at that moment); make that first call before any
+ * stream capture.  All calls on a device share the one array and it keeps the previous call's
+ * contents; nothing in it has to start at zero, because every row's words are rewritten before
+ * they are read.  Two calls whose kernels overlap on the GPU (different streams, no ordering
+ * between them) race on the array: order them. */
+int rpo_sample_rows_noalloc(int32_t n_rows, int32_t vocab, const float* d_logits, const rpo_sampler* sampler,
+                            const int64_t* d_seq_ids, int32_t step, int32_t* d_tokens_out, float* d_logprobs_out,
+                            void* cuda_stream);
+
 /* Dense product C[M,N] = A[M,K] * W[N,K]^T through the same GEMM kernel the layers use
  * (storage type of the context; C is float32).  For kernel-level parity tests.
  * impl: 0 = the kernel the context would choose, 1 = plain CUDA-core kernel,

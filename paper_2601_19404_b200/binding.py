@@ -14,7 +14,7 @@ _LIB = None
 EXPORTED_SYMBOLS = [
     "rpo_strerror", "rpo_shape_preset", "rpo_create", "rpo_destroy", "rpo_init_weights", "rpo_read_tensor",
     "rpo_write_tensor", "rpo_prefill_prefix", "rpo_decode_suffix", "rpo_token_logprobs", "rpo_release_groups",
-    "rpo_rollout_host", "rpo_sample_rows", "rpo_gemm", "rpo_gemm_bench", "rpo_device_status", "rpo_counters", "rpo_set_option", "rpo_profile_read",
+    "rpo_rollout_host", "rpo_sample_rows", "rpo_sample_rows_noalloc", "rpo_gemm", "rpo_gemm_bench", "rpo_device_status", "rpo_counters", "rpo_set_option", "rpo_profile_read",
 ]
 
 
@@ -71,6 +71,7 @@ def load_library(path=None):
     lib.rpo_release_groups.argtypes = [vp, i32, C.POINTER(Group)]
     lib.rpo_rollout_host.argtypes = [vp, i32, vp, vp, vp, i32, i32, C.POINTER(Sampler), vp, vp, vp, i32, vp]
     lib.rpo_sample_rows.argtypes = [vp, i32, i32, vp, C.POINTER(Sampler), vp, i32, vp, vp]
+    lib.rpo_sample_rows_noalloc.argtypes = [i32, i32, vp, C.POINTER(Sampler), vp, i32, vp, vp, vp]
     lib.rpo_gemm.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp]
     lib.rpo_gemm_bench.argtypes = [vp, i32, i32, i32, vp, C.POINTER(vp), i32, i32, C.POINTER(f32)]
     lib.rpo_device_status.argtypes = [vp, C.POINTER(i32)]
@@ -119,6 +120,17 @@ def _ptr(t):
 def _check(rc, what):
     if rc != 0:
         raise RpoError(rc, what)
+
+
+def sample_rows_noalloc(d_logits, sampler, d_seq_ids, step, d_tokens_out, d_logprobs_out=None, stream=None):
+    """rpo_sample_rows_noalloc: the sampler on caller-supplied logits [n_rows, vocab] without a context
+    and without any allocation (its scratch is a fixed 16 MiB array inside the library, so
+    n_rows * vocab is limited to 4 Mi words).  `stream` is a torch.cuda.Stream or None."""
+    n, v = d_logits.shape
+    stream_ptr = None if stream is None else C.c_void_p(stream.cuda_stream)
+    _check(load_library().rpo_sample_rows_noalloc(n, v, _ptr(d_logits), C.byref(sampler), _ptr(d_seq_ids), int(step),
+                                                  _ptr(d_tokens_out), _ptr(d_logprobs_out), stream_ptr),
+           "rpo_sample_rows_noalloc")
 
 
 class Context:

@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include <type_traits>
@@ -1007,5 +1008,61 @@ extern "C" int rpo_profile_read(rpo_ctx* c, double* ms_out, int64_t* count_out, 
   for (auto& kv : by_label)
     fprintf(stderr, "[rpo profile] %-60s %8lld launches %10.3f ms  %8.2f us/launch\n", kv.first.c_str(),
             (long long)kv.second.second, kv.second.first, 1e3 * kv.second.first / kv.second.second);
+  return RPO_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// sampling without any allocation
+// ---------------------------------------------------------------------------------------------
+// The sampler parks one 32-bit weight per (row, token) in scratch memory.  rpo_sample_rows takes
+// that scratch from the stream-ordered allocator; this variant keeps a fixed array inside the
+// library image instead, so it needs neither a context nor an allocator.
+#define RPO_NOALLOC_SAMPLER_WORDS (4u << 20)     /* 4 Mi words = 16 MiB, held by every GPU that loads the library */
+static __device__ __align__(256) uint32_t g_noalloc_sampler_scratch[RPO_NOALLOC_SAMPLER_WORDS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+uint32_t* g_noalloc_scratch_ptr[kMaxDevices] = {};   // device address of the array, per device ordinal
+}  // namespace
+
+extern "C" int rpo_sample_rows_noalloc(int32_t n_rows, int32_t vocab, const float* d_logits, const rpo_sampler* sp,
+                                       const int64_t* d_seq_ids, int32_t step, int32_t* d_tokens_out,
+                                       float* d_logprobs_out, void* cuda_stream) {
+  if (n_rows < 0 || vocab <= 0 || vocab >= (1 << 18) || !d_logits || !d_seq_ids || !d_tokens_out || step < 0)
+    return RPO_ERR_INVALID_ARG;
+  RPO_TRY(check_sampler(sp));
+  if ((uint64_t)n_rows * (uint64_t)vocab > (uint64_t)RPO_NOALLOC_SAMPLER_WORDS) {
+    fprintf(stderr, "[rpo] rpo_sample_rows_noalloc: %d rows x %d tokens = %llu words exceed the built-in scratch of %u words\n",
+            n_rows, vocab, (unsigned long long)n_rows * (unsigned long long)vocab, RPO_NOALLOC_SAMPLER_WORDS);
+    return RPO_ERR_LIMIT;
+  }
+  if (n_rows == 0) return RPO_OK;
+  int dev = -1;
+  CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return RPO_ERR_LIMIT;
+  uint32_t* scratch = nullptr;
+  {
+    // Set-up, once per device, with that device current.  In host code the array's name is only
+    // a handle: the address a kernel may use has to be asked for.
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_scratch_ptr[dev]) {
+      uint32_t* ptr = nullptr;
+      CUDA_TRY(cudaGetSymbolAddress((void**)&ptr, g_noalloc_sampler_scratch));
+      CUDA_TRY(cudaFuncSetAttribute(sampler_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SAMPLER_SMEM));
+      g_noalloc_scratch_ptr[dev] = ptr;
+    }
+    scratch = g_noalloc_scratch_ptr[dev];
+  }
+  SamplerArgs a;
+  memset(&a, 0, sizeof(a));
+  a.V = vocab; a.logits = d_logits; a.weights = scratch;
+  a.temperature = sp->temperature;
+  a.top_p24 = (uint32_t)floorf(sp->top_p * 16777216.0f);
+  a.greedy = sp->greedy; a.eos_id = -1; a.seed = sp->seed;
+  a.seq_ids = d_seq_ids; a.step = step; a.out_stride = 1; a.out_col = 0;
+  a.tokens_out = d_tokens_out; a.logprobs_out = d_logprobs_out;
+  sampler_kernel<<<n_rows, 1024, SAMPLER_SMEM, (cudaStream_t)cuda_stream>>>(a);
+  CUDA_TRY(cudaGetLastError());
   return RPO_OK;
 }
