@@ -57,12 +57,25 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 }  // namespace fa
 
+// Tile shape per mode.  Prefill (ROWS) is compute-bound: 64-key tiles, Q fragments kept in registers,
+// two K/V buffers.  Decode (SHARED) is latency-bound: 32-key tiles, Q fragments re-read from shared
+// memory and a register cap so that four CTAs (16 warps) share an SM and hide each other's waits.
+template <int MODE> struct FaCfg {
+  static constexpr int BN = (MODE == FA_SHARED) ? 32 : 64;     // keys per tile
+  static constexpr int NST = (MODE == FA_SHARED) ? 2 : 2;      // K/V ring depth
+  static constexpr int MIN_CTAS = (MODE == FA_SHARED) ? 4 : 1;
+  static constexpr bool Q_IN_REGS = (MODE != FA_SHARED);
+  template <int DH> static constexpr int smem_bytes() { return (FA_BM + 2 * NST * BN) * DH * 2; }
+};
+
 template <int DH, int MODE>
-__global__ void __launch_bounds__(FA_THREADS) flash_attn_kernel(FlashArgs a) {
-  constexpr int NST = (MODE == FA_SHARED) ? 3 : 2;   // K/V ring depth: decode is latency-bound, prefill is not
+__global__ void __launch_bounds__(FA_THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_kernel(FlashArgs a) {
+  constexpr int NST = FaCfg<MODE>::NST;
+  constexpr int BN = FaCfg<MODE>::BN;
+  constexpr bool Q_IN_REGS = FaCfg<MODE>::Q_IN_REGS;
   constexpr int CH = DH / 8;                 // 16-byte chunks per row
   constexpr int ROW_BYTES = DH * 2;
-  constexpr int TILE_BYTES = FA_BN * ROW_BYTES;
+  constexpr int TILE_BYTES = BN * ROW_BYTES;
   constexpr int KSTEPS = DH / 16, ONT = DH / 8;
   extern __shared__ __align__(128) uint8_t fsm[];
   const uint32_t sQ = (uint32_t)__cvta_generic_to_shared(fsm);
@@ -132,17 +145,18 @@ __global__ void __launch_bounds__(FA_THREADS) flash_attn_kernel(FlashArgs a) {
     sh_begin = min(sd.shared_len, split * a.split_chunk);
     sh_end = min(sd.shared_len, sh_begin + a.split_chunk);
   }
-  const int n_sh_tiles = (sh_end - sh_begin + FA_BN - 1) / FA_BN;
-  const int n_pr_tiles = (pr_end + FA_BN - 1) / FA_BN;
+  const int n_sh_tiles = (sh_end - sh_begin + BN - 1) / BN;
+  const int n_pr_tiles = (pr_end + BN - 1) / BN;
   const int n_tiles = n_sh_tiles + n_pr_tiles;
 
-  // ---- loaders: thread pair per row, interleaved 16-byte chunks (32 contiguous bytes per pair)
-  const int lrow = tid >> 1, lpar = tid & 1;
+  // ---- loaders: TPR threads per K/V row (a thread pair per Q row), interleaved 16-byte chunks
+  constexpr int TPR = FA_THREADS / BN;
+  const int lrow = tid / TPR, lpar = tid % TPR;
   auto sw = [&](int row, int chunk) -> uint32_t { return (uint32_t)(row * ROW_BYTES + ((chunk ^ (row & 7)) << 4)); };
   auto load_kv = [&](int it, int buf) {
     int tbl, key0, limit;
-    if (it < n_sh_tiles) { tbl = sd.shared_tbl; key0 = sh_begin + it * FA_BN; limit = sh_end; }
-    else { tbl = sd.priv_tbl; key0 = (it - n_sh_tiles) * FA_BN; limit = pr_end; }
+    if (it < n_sh_tiles) { tbl = sd.shared_tbl; key0 = sh_begin + it * BN; limit = sh_end; }
+    else { tbl = sd.priv_tbl; key0 = (it - n_sh_tiles) * BN; limit = pr_end; }
     const int u = key0 + lrow;
     const bf16 *kp = nullptr, *vp = nullptr;
     if (u < limit) {
@@ -155,20 +169,21 @@ __global__ void __launch_bounds__(FA_THREADS) flash_attn_kernel(FlashArgs a) {
       }
     }
 #pragma unroll
-    for (int j = 0; j < CH / 2; ++j) {
-      const int ch = 2 * j + lpar;
+    for (int j = 0; j < CH / TPR; ++j) {
+      const int ch = TPR * j + lpar;
       const uint32_t off = sw(lrow, ch);
       if (kp) { fa::cp_async16(sK + buf * TILE_BYTES + off, kp + ch * 8); fa::cp_async16(sV + buf * TILE_BYTES + off, vp + ch * 8); }
       else { fa::st_zero16(sK + buf * TILE_BYTES + off); fa::st_zero16(sV + buf * TILE_BYTES + off); }
     }
   };
   {
-    const int qr = s_qrow[lrow];
-    const bf16* qp = (qr >= 0) ? a.qkv + (int64_t)qr * a.qkv_cols + s_head[lrow] * DH : nullptr;
+    const int qrow = tid >> 1, qpar = tid & 1;
+    const int qr = s_qrow[qrow];
+    const bf16* qp = (qr >= 0) ? a.qkv + (int64_t)qr * a.qkv_cols + s_head[qrow] * DH : nullptr;
 #pragma unroll
     for (int j = 0; j < CH / 2; ++j) {
-      const int ch = 2 * j + lpar;
-      if (qp) fa::cp_async16(sQ + sw(lrow, ch), qp + ch * 8); else fa::st_zero16(sQ + sw(lrow, ch));
+      const int ch = 2 * j + qpar;
+      if (qp) fa::cp_async16(sQ + sw(qrow, ch), qp + ch * 8); else fa::st_zero16(sQ + sw(qrow, ch));
     }
   }
 #pragma unroll
@@ -181,7 +196,7 @@ __global__ void __launch_bounds__(FA_THREADS) flash_attn_kernel(FlashArgs a) {
 #pragma unroll
   for (int i = 0; i < ONT; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
   float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
-  uint32_t qf[KSTEPS][4];
+  uint32_t qf[Q_IN_REGS ? KSTEPS : 1][4];
   const int r_lo = warp * 16 + g, r_hi = r_lo + 8;
   const int t_lo = s_t[r_lo], t_hi = s_t[r_hi];
 
@@ -192,32 +207,36 @@ __global__ void __launch_bounds__(FA_THREADS) flash_attn_kernel(FlashArgs a) {
     fa::cp_commit();
     fa::cp_wait<NST - 1>();                   // all but the newest NST-1 groups have landed: tile `it` is in
     __syncthreads();
-    if (it == 0) {
+    if (Q_IN_REGS && it == 0) {
 #pragma unroll
       for (int kk = 0; kk < KSTEPS; ++kk)
         fa::ldsm_x4(sQ + sw(warp * 16 + (lane & 15), kk * 2 + (lane >> 4)), qf[kk][0], qf[kk][1], qf[kk][2], qf[kk][3]);
     }
+    if (warp * 16 < n_rows) {        // warps whose 16 rows are all padding only help with the loads
     // ---- S = Q K^T
-    float s[FA_BN / 8][4];
+    float s[BN / 8][4];
 #pragma unroll
-    for (int j = 0; j < FA_BN / 8; ++j) { s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f; }
+    for (int j = 0; j < BN / 8; ++j) { s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f; }
     const uint32_t kb = sK + buf * TILE_BYTES, vb = sV + buf * TILE_BYTES;
 #pragma unroll
     for (int kk = 0; kk < KSTEPS; ++kk) {
+      const int qi = Q_IN_REGS ? kk : 0;
+      if (!Q_IN_REGS)
+        fa::ldsm_x4(sQ + sw(warp * 16 + (lane & 15), kk * 2 + (lane >> 4)), qf[0][0], qf[0][1], qf[0][2], qf[0][3]);
 #pragma unroll
-      for (int jp = 0; jp < FA_BN / 16; ++jp) {
+      for (int jp = 0; jp < BN / 16; ++jp) {
         uint32_t b0, b1, b2, b3;
         fa::ldsm_x4(kb + sw(jp * 16 + (lane & 7) + ((lane >> 4) << 3), kk * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
-        fa::mma_bf16(s[2 * jp], qf[kk], b0, b1);
-        fa::mma_bf16(s[2 * jp + 1], qf[kk], b2, b3);
+        fa::mma_bf16(s[2 * jp], qf[qi], b0, b1);
+        fa::mma_bf16(s[2 * jp + 1], qf[qi], b2, b3);
       }
     }
     // ---- mask + online softmax (base-2 exponent domain)
     const bool shared_tile = it < n_sh_tiles;
-    const int key0 = shared_tile ? sh_begin + it * FA_BN : (it - n_sh_tiles) * FA_BN;
+    const int key0 = shared_tile ? sh_begin + it * BN : (it - n_sh_tiles) * BN;
     float mx_lo = -INFINITY, mx_hi = -INFINITY;
 #pragma unroll
-    for (int j = 0; j < FA_BN / 8; ++j) {
+    for (int j = 0; j < BN / 8; ++j) {
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         const int key = key0 + j * 8 + tq * 2 + (c & 1);
@@ -234,9 +253,9 @@ __global__ void __launch_bounds__(FA_THREADS) flash_attn_kernel(FlashArgs a) {
     const float c_lo = exp2f(m_lo - mu_lo), c_hi = exp2f(m_hi - mu_hi);
     m_lo = mn_lo; m_hi = mn_hi;
     float ps_lo = 0.f, ps_hi = 0.f;
-    uint32_t pf[FA_BN / 16][4];
+    uint32_t pf[BN / 16][4];
 #pragma unroll
-    for (int j = 0; j < FA_BN / 8; ++j) {
+    for (int j = 0; j < BN / 8; ++j) {
       const float p0 = exp2f(s[j][0] - mu_lo), p1 = exp2f(s[j][1] - mu_lo);
       const float p2 = exp2f(s[j][2] - mu_hi), p3 = exp2f(s[j][3] - mu_hi);
       ps_lo += p0 + p1; ps_hi += p2 + p3;
@@ -248,7 +267,7 @@ __global__ void __launch_bounds__(FA_THREADS) flash_attn_kernel(FlashArgs a) {
     for (int i = 0; i < ONT; ++i) { o[i][0] *= c_lo; o[i][1] *= c_lo; o[i][2] *= c_hi; o[i][3] *= c_hi; }
     // ---- O += P V
 #pragma unroll
-    for (int kk = 0; kk < FA_BN / 16; ++kk) {
+    for (int kk = 0; kk < BN / 16; ++kk) {
 #pragma unroll
       for (int np = 0; np < ONT / 2; ++np) {
         uint32_t b0, b1, b2, b3;
@@ -256,6 +275,7 @@ __global__ void __launch_bounds__(FA_THREADS) flash_attn_kernel(FlashArgs a) {
         fa::mma_bf16(o[2 * np], pf[kk], b0, b1);
         fa::mma_bf16(o[2 * np + 1], pf[kk], b2, b3);
       }
+    }
     }
     __syncthreads();
   }

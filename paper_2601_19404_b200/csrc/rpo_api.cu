@@ -395,7 +395,7 @@ static int rmsnorm(rpo_ctx* c, float* x, const float* g, T* h, int rows) {
 
 template <int DH, int MODE>
 static int launch_flash(rpo_ctx* c, const FlashArgs& a, dim3 grid) {
-  constexpr int smem = (FA_BM + 2 * (MODE == FA_SHARED ? 3 : 2) * FA_BN) * DH * 2;
+  constexpr int smem = FaCfg<MODE>::template smem_bytes<DH>();
   static bool attr_done = false;
   if (!attr_done) {
     CUDA_TRY(cudaFuncSetAttribute(flash_attn_kernel<DH, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
