@@ -70,6 +70,7 @@ template <int MODE> struct FaCfg {
 
 template <int DH, int MODE>
 __global__ void __launch_bounds__(FA_THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_kernel(FlashArgs a) {
+  pdl_prologue();
   constexpr int NST = FaCfg<MODE>::NST;
   constexpr int BN = FaCfg<MODE>::BN;
   constexpr bool Q_IN_REGS = FaCfg<MODE>::Q_IN_REGS;
@@ -307,33 +308,50 @@ __global__ void __launch_bounds__(FA_THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_
 }
 
 // Decode: log-sum-exp merge of the partials of (sequence, query head) -- slots 0..n_splits-1 from the
-// splits of the shared prefix, slot n_splits from the sequence's own suffix keys -- one warp each;
-// lanes own DH/32 dimensions.  Fixed slot order, hence reproducible.
+// splits of the shared prefix, slot n_splits from the sequence's own suffix keys (n_slots <= 33) -- one
+// warp each.  Lane s first reads (m, l) of slot s, the warp agrees on the maximum and on each
+// slot's weight, then all slots' O rows are accumulated with independent loads in slot order
+// (reproducible); lanes own DH/32 dimensions.
 template <int DH>
 __global__ void __launch_bounds__(128) attn_decode_merge_kernel(bf16* __restrict__ out, const float* __restrict__ part_ml,
                                                                 const float* __restrict__ part_o, int n_slots,
                                                                 const int32_t* __restrict__ row_t, int rows, int hq) {
+  pdl_prologue();
   constexpr int DPL = DH / 32;
   const int w = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (w >= rows * hq) return;
   const int r = w / hq, head = w % hq;
   bf16* o = out + (int64_t)r * hq * DH + head * DH + lane * DPL;
-  float m = -INFINITY, l = 0.f, acc[DPL];
+  float acc[DPL];
 #pragma unroll
   for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
+  float l_tot = 0.f, m_run = -INFINITY;        // warp-uniform
   if (row_t[r] >= 0) {
-    for (int s = 0; s < n_slots; ++s) {
-      const int64_t slot = ((int64_t)r * hq + head) * n_slots + s;
-      const float ms = part_ml[slot * 2], ls = part_ml[slot * 2 + 1];
-      if (!(ls > 0.f)) continue;
-      const float mn = fmaxf(m, ms), c0 = exp2f(m - mn), c1 = exp2f(ms - mn);
-      l = l * c0 + ls * c1;
+    const int64_t slot0 = ((int64_t)r * hq + head) * n_slots;
+    for (int s0 = 0; s0 < n_slots; s0 += 32) {         // one pass for n_slots <= 32, a second for the 33rd
+      const int s = s0 + lane;
+      float ms = -INFINITY, ls = 0.f;
+      if (s < n_slots) { const float2 ml = *reinterpret_cast<const float2*>(part_ml + (slot0 + s) * 2); ms = ml.x; ls = ml.y; }
+      if (!(ls > 0.f)) ms = -INFINITY;
+      // running maximum over passes: rescale what has been accumulated so far
+      const float m_new = fmaxf(m_run, warp_max(ms));
+      const float rescale = (m_run == -INFINITY) ? 0.f : exp2f(m_run - m_new);
+      const float wgt = (ls > 0.f) ? exp2f(ms - m_new) : 0.f;
+      l_tot = l_tot * rescale + warp_sum(ls * wgt);
 #pragma unroll
-      for (int i = 0; i < DPL; ++i) acc[i] = acc[i] * c0 + part_o[slot * DH + lane * DPL + i] * c1;
-      m = mn;
+      for (int i = 0; i < DPL; ++i) acc[i] *= rescale;
+      const int n_here = min(32, n_slots - s0);
+#pragma unroll 4
+      for (int k = 0; k < n_here; ++k) {
+        const float c = __shfl_sync(0xffffffffu, wgt, k);
+        const float* po = part_o + (slot0 + s0 + k) * DH + lane * DPL;
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) { const float v = po[i]; acc[i] += (c != 0.f) ? c * v : 0.f; }
+      }
+      m_run = m_new;
     }
   }
-  const float inv = (l > 0.f) ? 1.0f / l : 0.f;
+  const float inv = (l_tot > 0.f) ? 1.0f / l_tot : 0.f;
 #pragma unroll
   for (int i = 0; i < DPL; ++i) o[i] = __float2bfloat16_rn(acc[i] * inv);
 }

@@ -140,6 +140,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_items = p.tiles_m * p.tiles_n * p.splits;
+  pdl_launch_dependents();
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < Cfg::NS; ++i) { tc::mbar_init(&full[i], 1); tc::mbar_init(&empty[i], 1); }
@@ -162,13 +163,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (lane == 0) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
-      int stage = 0; uint32_t phase = 0;
+      // The weight matrix does not depend on the kernel running before this one: the W tiles of
+      // this CTA's first work item go into the (still empty) ring first, then the producer waits
+      // for the predecessor and sends the matching A tiles after them.
+      int pre = 0;
+      if ((int)blockIdx.x < n_items) {
+        const int split = blockIdx.x % p.splits, t = blockIdx.x / p.splits;
+        const int tn = t % p.tiles_n, tm = t / p.tiles_n;
+        const int kb0 = split * p.kb_per_split, kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+        pre = min(Cfg::NS, kb1 - kb0);
+        for (int i = 0; i < pre; ++i) {
+          tc::mbar_expect_tx(&full[i], Cfg::STAGE_BYTES);
+          tc::tma_load_2d(smem + i * Cfg::STAGE_BYTES + Cfg::A_BYTES, &map_w, (kb0 + i) * TC_BK, tn * BN, &full[i]);
+        }
+        pdl_wait();
+        for (int i = 0; i < pre; ++i)
+          tc::tma_load_2d(smem + i * Cfg::STAGE_BYTES, &map_a, (kb0 + i) * TC_BK, tm * TC_BM, &full[i]);
+      } else {
+        pdl_wait();
+      }
+      int stage = pre % Cfg::NS; uint32_t phase = (pre == Cfg::NS) ? 1u : 0u;
       bool ok = true;
       for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
         const int split = it % p.splits, t = it / p.splits;
         const int tn = t % p.tiles_n, tm = t / p.tiles_n;
         const int kb0 = split * p.kb_per_split, kb1 = min(p.kb_total, kb0 + p.kb_per_split);
-        for (int kb = kb0; kb < kb1; ++kb) {
+        for (int kb = kb0 + (it == (int)blockIdx.x ? pre : 0); kb < kb1; ++kb) {
           if (!tc::mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
           uint8_t* sa = smem + stage * Cfg::STAGE_BYTES;
           tc::mbar_expect_tx(&full[stage], Cfg::STAGE_BYTES);
@@ -210,6 +230,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..5)
     const int quad = warp & 3;                       // TMEM lane quadrant this warp may read
+    pdl_wait();                                      // the epilogue reads / overwrites what earlier kernels produced
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
     for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
@@ -360,8 +381,13 @@ inline int tc_launch(rpo_ctx* c, const CUtensorMap* ma, const CUtensorMap* mw, c
       return RPO_ERR_CUDA;
     attr_done = true;
   }
-  gemm_tc_kernel<BN, EPI><<<grid, 192, Cfg::SMEM_BYTES, c->stream>>>(*ma, *mw, p);
-  return cudaGetLastError() == cudaSuccess ? RPO_OK : RPO_ERR_CUDA;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = Cfg::SMEM_BYTES; cfg.stream = c->stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = c->use_pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, EPI>, *ma, *mw, p) == cudaSuccess ? RPO_OK : RPO_ERR_CUDA;
 }
 
 template <int BN>

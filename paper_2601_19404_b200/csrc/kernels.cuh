@@ -34,6 +34,7 @@ struct KVPool {
 template <typename T>
 __global__ void init_normal_kernel(T* __restrict__ dst, int64_t n_elems, int cols, int row_mul, int row_add,
                                    uint32_t k0, uint32_t k1, uint32_t tensor_id, float stdv) {
+  pdl_prologue();
   const int64_t n_blocks = (n_elems + 3) / 4;
   for (int64_t blk = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; blk < n_blocks;
        blk += (int64_t)gridDim.x * blockDim.x) {
@@ -62,12 +63,14 @@ __global__ void init_normal_kernel(T* __restrict__ dst, int64_t n_elems, int col
 
 template <typename T>
 __global__ void fill_kernel(T* dst, int64_t n, float v) {
+  pdl_prologue();
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
     dst[i] = from_f32<T>(v);
 }
 
 // cos/sin table [max_positions][head_dim/2], angles in float64.
 __global__ void rope_table_kernel(float2* __restrict__ tab, int max_pos, int half, double base) {
+  pdl_prologue();
   const int64_t n = (int64_t)max_pos * half;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
     const int pos = (int)(i / half), j = (int)(i % half);
@@ -83,7 +86,8 @@ __global__ void rope_table_kernel(float2* __restrict__ tab, int max_pos, int hal
 // that the sampler at the end of the forward reads, so that every step is the same launch sequence.
 template <typename T>
 __global__ void embed_kernel(const int32_t* __restrict__ tokens, const T* __restrict__ E, float* __restrict__ x,
-                             int rows, int d, int vocab, int* status, int32_t* step_ctr = nullptr) {
+                             int rows, int d, int vocab, int* status, int32_t* step_ctr) {
+  pdl_prologue();
   const int r = blockIdx.x;
   if (step_ctr && r == 0 && threadIdx.x == 0) *step_ctr += 1;
   if (r >= rows) return;
@@ -100,6 +104,7 @@ __global__ void embed_kernel(const int32_t* __restrict__ tokens, const T* __rest
 // dst[r,:] = src[idx[r],:]  (float32 rows; idx may be NULL = identity)
 __global__ void gather_rows_f32_kernel(const float* __restrict__ src, const int32_t* __restrict__ idx,
                                        float* __restrict__ dst, int rows, int d) {
+  pdl_prologue();
   const int r = blockIdx.x;
   if (r >= rows) return;
   const int s = idx ? idx[r] : r;
@@ -110,27 +115,38 @@ __global__ void gather_rows_f32_kernel(const float* __restrict__ src, const int3
   for (int i = threadIdx.x; i < d; i += blockDim.x) dst[(int64_t)r * d + i] = src[(int64_t)s * d + i];
 }
 
-// RMSNorm of the float32 residual stream, one CTA per row:
-//   x[r,:] += sum_s partial[s][r,:]   (optional split-K partial sums of the previous GEMM)
+// RMSNorm of the float32 residual stream, one CTA per row, 128-bit accesses (d % 4 == 0):
+//   x[r,:] += sum_s partial[s][r,:]   (optional split-K partial planes of the previous GEMM, summed
+//                                      in plane order; the loads of all planes are independent)
 //   h[r,:]  = x[r,:] / sqrt(mean(x^2) + eps) * g
+// Dynamic shared memory: d floats (the row, kept between the two passes).
 template <typename T>
 __global__ void rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ gain, T* __restrict__ h, int rows,
                                int d, float eps, const float* __restrict__ partial, int n_splits,
                                int64_t split_stride) {
-  extern __shared__ float srow[];
+  pdl_prologue();
+  extern __shared__ __align__(16) float srow[];
   __shared__ float red[32];
   const int r = blockIdx.x;
   if (r >= rows) return;
-  float* xr = x + (int64_t)r * d;
+  const int d4 = d >> 2;
+  float4* xr = reinterpret_cast<float4*>(x + (int64_t)r * d);
+  float4* s4 = reinterpret_cast<float4*>(srow);
   float ss = 0.f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    float v = xr[i];
+  for (int i = threadIdx.x; i < d4; i += blockDim.x) {
+    float4 v = xr[i];
     if (partial) {
-      for (int s = 0; s < n_splits; ++s) v += partial[s * split_stride + (int64_t)r * d + i];
+      const float4* p4 = reinterpret_cast<const float4*>(partial + (int64_t)r * d) + i;
+      const int64_t st4 = split_stride >> 2;
+#pragma unroll 4
+      for (int s = 0; s < n_splits; ++s) {
+        const float4 q = p4[s * st4];
+        v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
+      }
       xr[i] = v;
     }
-    srow[i] = v;
-    ss += v * v;
+    s4[i] = v;
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   ss = warp_sum(ss);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
@@ -142,13 +158,19 @@ __global__ void rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ 
   }
   __syncthreads();
   const float inv = 1.0f / sqrtf(red[0] / (float)d + eps);
+  const float4* g4 = reinterpret_cast<const float4*>(gain);
   T* hr = h + (int64_t)r * d;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) hr[i] = from_f32<T>(srow[i] * inv * gain[i]);
+  for (int i = threadIdx.x; i < d4; i += blockDim.x) {
+    const float4 v = s4[i], g = g4[i];
+    hr[4 * i] = from_f32<T>(v.x * inv * g.x); hr[4 * i + 1] = from_f32<T>(v.y * inv * g.y);
+    hr[4 * i + 2] = from_f32<T>(v.z * inv * g.z); hr[4 * i + 3] = from_f32<T>(v.w * inv * g.w);
+  }
 }
 
 // x[i] += sum_s partial[s*stride + i], fixed order (deterministic split-K reduction). n % 4 == 0.
 __global__ void reduce_partials_kernel(float* __restrict__ x, const float* __restrict__ partial, int n_splits, int64_t n,
                                        int64_t stride) {
+  pdl_prologue();
   for (int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4; i < n; i += (int64_t)gridDim.x * blockDim.x * 4) {
     float4 v = *(const float4*)(x + i);
     for (int s = 0; s < n_splits; ++s) {
@@ -170,6 +192,7 @@ __global__ void rope_kv_kernel(T* __restrict__ qkv, const int32_t* __restrict__ 
                                const int32_t* __restrict__ block_table, const float2* __restrict__ rope_tab,
                                KVPool<T> pool, int layer, int rows, int hq, int hkv, int max_pos, int* status,
                                const float* __restrict__ partial, int n_splits, int64_t split_stride) {
+  pdl_prologue();
   const int r = blockIdx.x, head = blockIdx.y;
   if (r >= rows) return;
   const int t = row_t[r];
@@ -183,6 +206,7 @@ __global__ void rope_kv_kernel(T* __restrict__ qkv, const int32_t* __restrict__ 
   auto ld = [&](int i) -> float {
     if (!partial) return to_f32(src[i]);
     float v = 0.f;
+#pragma unroll 4
     for (int s = 0; s < n_splits; ++s) v += partial[s * split_stride + off + i];
     return to_f32(from_f32<T>(v));
   };
@@ -208,6 +232,7 @@ __global__ void rope_kv_kernel(T* __restrict__ qkv, const int32_t* __restrict__ 
 // act[r, j] = silu(gu[r, 2j]) * gu[r, 2j+1]   (gate/up interleaved by the fused weight layout)
 template <typename T>
 __global__ void swiglu_kernel(const T* __restrict__ gu, T* __restrict__ act, int64_t n_out) {
+  pdl_prologue();
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_out; i += (int64_t)gridDim.x * blockDim.x) {
     const float g = to_f32(gu[2 * i]), u = to_f32(gu[2 * i + 1]);
     act[i] = from_f32<T>(g / (1.0f + __expf(-g)) * u);
@@ -219,6 +244,7 @@ __global__ void swiglu_kernel(const T* __restrict__ gu, T* __restrict__ act, int
 __global__ void build_teacher_rows_kernel(const int32_t* __restrict__ tokens, const int32_t* __restrict__ lens,
                                           int seq0, int n_seq, int S, int32_t* __restrict__ row_seq,
                                           int32_t* __restrict__ row_t, int32_t* __restrict__ row_tok) {
+  pdl_prologue();
   const int n = n_seq * (S - 1);
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
     const int s = i / (S - 1), j = i % (S - 1);
@@ -235,6 +261,7 @@ __global__ void build_teacher_rows_kernel(const int32_t* __restrict__ tokens, co
 __global__ void gather_head_rows_kernel(const float* __restrict__ x, const float* __restrict__ x_last,
                                         const int32_t* __restrict__ seq_slot, int row0, int n_rows, int S, int d,
                                         float* __restrict__ dst) {
+  pdl_prologue();
   const int i = blockIdx.x;
   if (i >= n_rows) return;
   const int hr = row0 + i, s = hr / S, j = hr % S;
@@ -276,6 +303,7 @@ __device__ __forceinline__ float block_reduce_sum(float v, float* red) {
 __global__ void logprob_rows_kernel(const float* __restrict__ logits, int row0, int n_rows, int V, int S,
                                     const int32_t* __restrict__ tokens, const int32_t* __restrict__ lens, int seq0,
                                     float inv_T, float* __restrict__ out, float* __restrict__ logits_dbg) {
+  pdl_prologue();
   __shared__ float red[32];
   const int i = blockIdx.x;
   if (i >= n_rows) return;

@@ -12,6 +12,7 @@ enum GemmEpilogue { EPI_STORE_T = 0, EPI_STORE_F32 = 1, EPI_ADD_F32 = 2, EPI_SWI
 template <typename T, int EPI>
 __global__ void __launch_bounds__(256) gemm_ref_kernel(const T* __restrict__ A, const T* __restrict__ W,
                                                        void* __restrict__ Cv, int M, int N, int K, int64_t ldc) {
+  pdl_prologue();
   __shared__ float sA[16][64 + 4];
   __shared__ float sW[16][64 + 4];
   const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
@@ -68,6 +69,7 @@ __global__ void __launch_bounds__(128) attn_ref_kernel(const T* __restrict__ qkv
                                                        const int32_t* __restrict__ block_table, KVPool<T> pool,
                                                        int layer, int rows, int hq, int hkv, float scale,
                                                        int* status) {
+  pdl_prologue();
   constexpr int DPL = DH / 32;
   const int w = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (w >= rows * hq) return;

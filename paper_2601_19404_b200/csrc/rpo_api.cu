@@ -9,6 +9,7 @@
 #include <new>
 
 #include <type_traits>
+#include <utility>
 
 #include "attn_tc.cuh"
 #include "context.h"
@@ -56,13 +57,28 @@ static void prof_end(rpo_ctx* c) {
   cudaEventRecord(c->prof_events.back().b, c->stream);
 }
 
-#define LAUNCH(ctx, kern, grid, block, smem, ...)                         \
-  do {                                                                    \
-    prof_begin(ctx, #kern);                                               \
-    kern<<<(grid), (block), (smem), (ctx)->stream>>>(__VA_ARGS__);        \
-    prof_end(ctx);                                                        \
-    (ctx)->launches++;                                                    \
-    CUDA_TRY(cudaGetLastError());                                         \
+// Every kernel of the library starts with pdl_prologue() (or places pdl_wait() itself), so it may be
+// launched with programmatic stream serialization: its CTAs are scheduled while the previous
+// kernel drains, which hides launch latency between the many short kernels of a decode step.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_kernel(rpo_ctx* c, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = c->use_pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
+#define LAUNCH(ctx, kern, grid, block, smem, ...)                                            \
+  do {                                                                                       \
+    prof_begin(ctx, #kern);                                                                  \
+    const cudaError_t le_ = launch_kernel(ctx, kern, dim3(grid), dim3(block), (size_t)(smem), __VA_ARGS__); \
+    prof_end(ctx);                                                                           \
+    (ctx)->launches++;                                                                       \
+    CUDA_TRY(le_);                                                                           \
+    CUDA_TRY(cudaGetLastError());                                                            \
   } while (0)
 
 static inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
@@ -386,7 +402,8 @@ static int rmsnorm(rpo_ctx* c, float* x, const float* g, T* h, int rows) {
   const int d = c->shape.d_model;
   const bool fold = (x == c->ws.x && c->pending_splits > 0 && c->pending_rows == rows);
   if (!fold && x == c->ws.x) RPO_TRY(flush_partials(c));
-  LAUNCH(c, rmsnorm_kernel<T>, rows, 256, (size_t)d * 4, x, g, h, rows, d, c->shape.rms_eps,
+  const int threads = std::min(1024, ((d / 4 + 31) / 32) * 32);
+  LAUNCH(c, rmsnorm_kernel<T>, rows, threads, (size_t)d * 4, x, g, h, rows, d, c->shape.rms_eps,
          fold ? (const float*)c->ws.partial : (const float*)nullptr, fold ? c->pending_splits : 0,
          (int64_t)rows * d);
   if (fold) c->pending_splits = 0;
@@ -547,7 +564,7 @@ static int prefill_chunk(rpo_ctx* c, const int32_t* d_tokens, int tok0, const st
   CUDA_TRY(cudaMemcpyAsync(w.seqs, sd.data(), (size_t)n * sizeof(SeqDesc), cudaMemcpyHostToDevice, c->stream));
   RPO_TRY(upload_row_tiles(c, lens));
   LAUNCH(c, embed_kernel<T>, rows, 128, 0, d_tokens + tok0, (const T*)c->embed, w.x, rows, c->shape.d_model,
-         c->shape.vocab, c->d_status);
+         c->shape.vocab, c->d_status, (int32_t*)nullptr);
   RPO_TRY(run_layers<T>(c, rows));
   // keep the residual stream of every group's last prefix token: step-0 logits come from it
   for (int i = 0; i < n; ++i)
@@ -716,7 +733,8 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
                                  (uint64_t)(uintptr_t)d_logprobs_out, (uint64_t)(uintptr_t)d_logits_dbg,
                                  (uint64_t)a.top_p24, (uint64_t)temp_bits,
                                  (uint64_t)a.greedy, (uint64_t)(uint32_t)a.eos_id, a.seed,
-                                 (uint64_t)c->use_tcgen05, (uint64_t)c->use_tc_attention};
+                                 (uint64_t)c->use_tcgen05, (uint64_t)c->use_tc_attention, (uint64_t)c->use_pdl,
+                                 (uint64_t)c->gemm_bn, (uint64_t)c->gemm_splits};
     rpo_ctx::StepGraph* sg = nullptr;
     for (auto& g : c->step_graphs) if (g.key == key) sg = &g;
     if (!sg) {
@@ -807,7 +825,7 @@ static int logprobs_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, 
         build_teacher_rows_kernel<<<grid_for(rows, 256), 256, 0, st>>>(d_tokens, d_lens, s0, ns, S, w.row_seq, w.row_t,
                                                                       w.row_tok);
         c->launches++;
-        embed_kernel<T><<<rows, 128, 0, st>>>((const int32_t*)w.row_tok, (const T*)c->embed, w.x, rows, d, V, c->d_status);
+        embed_kernel<T><<<rows, 128, 0, st>>>((const int32_t*)w.row_tok, (const T*)c->embed, w.x, rows, d, V, c->d_status, nullptr);
         c->launches++;
         if ((rc = run_layers<T>(c, rows)) != RPO_OK) break;
       }
@@ -980,6 +998,7 @@ extern "C" int rpo_set_option(rpo_ctx* c, const char* name, int32_t value) {
   if (!strcmp(name, "use_tcgen05")) c->use_tcgen05 = value;
   else if (!strcmp(name, "use_tc_attention")) c->use_tc_attention = value;
   else if (!strcmp(name, "use_graph")) c->use_graph = value;
+  else if (!strcmp(name, "use_pdl")) c->use_pdl = value;
   else if (!strcmp(name, "gemm_bn")) { if (value != 0 && value != 32 && value != 64 && value != 96 && value != 128 && value != 256) return RPO_ERR_INVALID_ARG; c->gemm_bn = value; }
   else if (!strcmp(name, "gemm_splits")) c->gemm_splits = value;
   else if (!strcmp(name, "profile")) c->profile = value;

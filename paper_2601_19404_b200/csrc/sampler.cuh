@@ -197,6 +197,7 @@ __device__ __forceinline__ void scan_row(const T* __restrict__ row, int n, int t
 constexpr int SAMPLER_SMEM = 64 * 1024;
 
 __global__ void __launch_bounds__(1024) sampler_kernel(SamplerArgs a) {
+  pdl_prologue();
   if (a.step_ptr) { a.step = *a.step_ptr; a.out_col = a.step; a.last_step = (a.step == a.n_steps - 1); }
   extern __shared__ __align__(16) uint8_t sampler_smem[];   // SAMPLER_SMEM bytes: the level histograms, in turn
   LaneHist& h1 = *reinterpret_cast<LaneHist*>(sampler_smem);
