@@ -51,6 +51,11 @@ __device__ __forceinline__ void mma_bf16(float* c, const uint32_t* a, uint32_t b
   asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ float ex2(float x) {          // 2^x, one MUFU (ex2.approx: rel. error 2^-22; -inf -> 0)
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
   return *(uint32_t*)&h;
@@ -236,36 +241,47 @@ __global__ void __launch_bounds__(FA_THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_
     const bool shared_tile = it < n_sh_tiles;
     const int key0 = shared_tile ? sh_begin + it * BN : (it - n_sh_tiles) * BN;
     float mx_lo = -INFINITY, mx_hi = -INFINITY;
+    if (shared_tile && key0 + BN <= sh_end) {          // tile fully inside the visible prefix: no masking
 #pragma unroll
-    for (int j = 0; j < BN / 8; ++j) {
+      for (int j = 0; j < BN / 8; ++j) {
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const int key = key0 + j * 8 + tq * 2 + (c & 1);
-        const bool vis = shared_tile ? (key < sh_end) : (key <= ((c & 2) ? t_hi : t_lo));
-        const float v = vis ? s[j][c] * a.scale_log2 : -INFINITY;
-        s[j][c] = v;
-        if (c & 2) mx_hi = fmaxf(mx_hi, v); else mx_lo = fmaxf(mx_lo, v);
+        for (int c = 0; c < 4; ++c) s[j][c] *= a.scale_log2;
+        mx_lo = fmaxf(mx_lo, fmaxf(s[j][0], s[j][1])); mx_hi = fmaxf(mx_hi, fmaxf(s[j][2], s[j][3]));
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < BN / 8; ++j) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int key = key0 + j * 8 + tq * 2 + (c & 1);
+          const bool vis = shared_tile ? (key < sh_end) : (key <= ((c & 2) ? t_hi : t_lo));
+          const float v = vis ? s[j][c] * a.scale_log2 : -INFINITY;
+          s[j][c] = v;
+          if (c & 2) mx_hi = fmaxf(mx_hi, v); else mx_lo = fmaxf(mx_lo, v);
+        }
       }
     }
     mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1)); mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
     mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1)); mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
     const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
     const float mu_lo = (mn_lo == -INFINITY) ? 0.f : mn_lo, mu_hi = (mn_hi == -INFINITY) ? 0.f : mn_hi;
-    const float c_lo = exp2f(m_lo - mu_lo), c_hi = exp2f(m_hi - mu_hi);
+    const float c_lo = fa::ex2(m_lo - mu_lo), c_hi = fa::ex2(m_hi - mu_hi);
     m_lo = mn_lo; m_hi = mn_hi;
     float ps_lo = 0.f, ps_hi = 0.f;
     uint32_t pf[BN / 16][4];
 #pragma unroll
     for (int j = 0; j < BN / 8; ++j) {
-      const float p0 = exp2f(s[j][0] - mu_lo), p1 = exp2f(s[j][1] - mu_lo);
-      const float p2 = exp2f(s[j][2] - mu_hi), p3 = exp2f(s[j][3] - mu_hi);
+      const float p0 = fa::ex2(s[j][0] - mu_lo), p1 = fa::ex2(s[j][1] - mu_lo);
+      const float p2 = fa::ex2(s[j][2] - mu_hi), p3 = fa::ex2(s[j][3] - mu_hi);
       ps_lo += p0 + p1; ps_hi += p2 + p3;
       pf[j >> 1][(j & 1) * 2] = fa::pack_bf16(p0, p1);
       pf[j >> 1][(j & 1) * 2 + 1] = fa::pack_bf16(p2, p3);
     }
     l_lo = l_lo * c_lo + ps_lo; l_hi = l_hi * c_hi + ps_hi;
+    if (!__all_sync(0xffffffffu, c_lo == 1.0f && c_hi == 1.0f)) {   // running maxima unchanged: nothing to rescale
 #pragma unroll
-    for (int i = 0; i < ONT; ++i) { o[i][0] *= c_lo; o[i][1] *= c_lo; o[i][2] *= c_hi; o[i][3] *= c_hi; }
+      for (int i = 0; i < ONT; ++i) { o[i][0] *= c_lo; o[i][1] *= c_lo; o[i][2] *= c_hi; o[i][3] *= c_hi; }
+    }
     // ---- O += P V
 #pragma unroll
     for (int kk = 0; kk < BN / 16; ++kk) {
