@@ -66,9 +66,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // two K/V buffers.  Decode (SHARED) is latency-bound: 32-key tiles, Q fragments re-read from shared
 // memory and a register cap so that four CTAs (16 warps) share an SM and hide each other's waits.
 template <int MODE> struct FaCfg {
-  static constexpr int BN = (MODE == FA_SHARED) ? 32 : 64;     // keys per tile
+  static constexpr int BN = (MODE == FA_SHARED) ? 64 : 64;     // keys per tile
   static constexpr int NST = (MODE == FA_SHARED) ? 2 : 2;      // K/V ring depth
-  static constexpr int MIN_CTAS = (MODE == FA_SHARED) ? 4 : 1;
+  static constexpr int MIN_CTAS = (MODE == FA_SHARED) ? 2 : 1;
   static constexpr bool Q_IN_REGS = (MODE != FA_SHARED);
   template <int DH> static constexpr int smem_bytes() { return (FA_BM + 2 * NST * BN) * DH * 2; }
 };

@@ -182,7 +182,10 @@ __global__ void reduce_partials_kernel(float* __restrict__ x, const float* __res
 }
 
 // RoPE (rotate-half) on q and k, then K/V written to the row's slot of its private segment.
-// qkv row layout: [q heads | k heads | v heads] x head_dim.  Grid: (rows, Hq + 2*Hkv).
+// qkv row layout: [q heads | k heads | v heads] x head_dim.  A group of dh/16 threads owns one
+// (row, head): each thread takes 8 consecutive dimensions of the low half and the 8 dimensions
+// they pair with in the high half (128-bit accesses for 16-bit storage).  Grid: ceil(rows * heads *
+// dh/16 / blockDim) CTAs.
 // With `partial` the projection arrives as n_splits split-K planes [rows, qkv_cols] of float32:
 // they are summed in plane order and rounded to the storage type first, exactly what the
 // unsplit GEMM epilogue would have stored.
@@ -193,40 +196,65 @@ __global__ void rope_kv_kernel(T* __restrict__ qkv, const int32_t* __restrict__ 
                                KVPool<T> pool, int layer, int rows, int hq, int hkv, int max_pos, int* status,
                                const float* __restrict__ partial, int n_splits, int64_t split_stride) {
   pdl_prologue();
-  const int r = blockIdx.x, head = blockIdx.y;
-  if (r >= rows) return;
+  const int dh = pool.head_dim, half = dh / 2, tph = dh / 16, heads = hq + 2 * hkv;
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t unit = gid / tph;                       // (row, head)
+  if (unit >= (int64_t)rows * heads) return;
+  const int r = (int)(unit / heads), head = (int)(unit % heads), i0 = (int)(gid % tph) * 8;
   const int t = row_t[r];
   if (t < 0) return;
-  const int dh = pool.head_dim, half = dh / 2;
   const SeqDesc sd = seqs[row_seq[r]];
   const int pos = sd.shared_len + t;
-  if (pos >= max_pos) { if (threadIdx.x == 0) atomicOr(status, STATUS_BAD_BLOCK); return; }
-  const int64_t off = (int64_t)r * (hq + 2 * hkv) * dh + (int64_t)head * dh;
+  if (pos >= max_pos) { if (i0 == 0) atomicOr(status, STATUS_BAD_BLOCK); return; }
+  const int64_t off = (int64_t)r * heads * dh + (int64_t)head * dh;
   T* src = qkv + off;
-  auto ld = [&](int i) -> float {
-    if (!partial) return to_f32(src[i]);
-    float v = 0.f;
-#pragma unroll 4
-    for (int s = 0; s < n_splits; ++s) v += partial[s * split_stride + off + i];
-    return to_f32(from_f32<T>(v));
-  };
-  T* dst = nullptr;
+  float lo[8], hi[8];
+  if (partial) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { lo[j] = 0.f; hi[j] = 0.f; }
+#pragma unroll 2
+    for (int s = 0; s < n_splits; ++s) {
+      const float4* pl = reinterpret_cast<const float4*>(partial + s * split_stride + off + i0);
+      const float4* ph = reinterpret_cast<const float4*>(partial + s * split_stride + off + half + i0);
+      const float4 a0 = pl[0], a1 = pl[1], b0 = ph[0], b1 = ph[1];
+      lo[0] += a0.x; lo[1] += a0.y; lo[2] += a0.z; lo[3] += a0.w; lo[4] += a1.x; lo[5] += a1.y; lo[6] += a1.z; lo[7] += a1.w;
+      hi[0] += b0.x; hi[1] += b0.y; hi[2] += b0.z; hi[3] += b0.w; hi[4] += b1.x; hi[5] += b1.y; hi[6] += b1.z; hi[7] += b1.w;
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { lo[j] = to_f32(from_f32<T>(lo[j])); hi[j] = to_f32(from_f32<T>(hi[j])); }
+  } else {
+    T tl[8], th[8];
+    *reinterpret_cast<uint4*>(tl) = *reinterpret_cast<const uint4*>(src + i0);
+    if (sizeof(T) == 4) *reinterpret_cast<uint4*>(tl + 4) = *reinterpret_cast<const uint4*>(src + i0 + 4);
+    *reinterpret_cast<uint4*>(th) = *reinterpret_cast<const uint4*>(src + half + i0);
+    if (sizeof(T) == 4) *reinterpret_cast<uint4*>(th + 4) = *reinterpret_cast<const uint4*>(src + half + i0 + 4);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { lo[j] = to_f32(tl[j]); hi[j] = to_f32(th[j]); }
+  }
+  T* dst = src;                                         // q: rotated in place
   if (head >= hq) {
     const int kv = (head - hq) / hkv, kh = (head - hq) % hkv;
     const int blk = block_table[sd.priv_tbl + t / KV_BLOCK];
-    if (blk < 0 || blk >= pool.n_blocks) { if (threadIdx.x == 0) atomicOr(status, STATUS_BAD_BLOCK); return; }
+    if (blk < 0 || blk >= pool.n_blocks) { if (i0 == 0) atomicOr(status, STATUS_BAD_BLOCK); return; }
     dst = pool.at(layer, kv, kh, blk, t % KV_BLOCK);
   }
-  if (head < hq + hkv) {  // q or k: rotate
-    for (int i = threadIdx.x; i < half; i += blockDim.x) {
-      const float2 cs = rope_tab[(int64_t)pos * half + i];
-      const float a = ld(i), b = ld(i + half);
-      const T o1 = from_f32<T>(a * cs.x - b * cs.y), o2 = from_f32<T>(b * cs.x + a * cs.y);
-      if (dst) { dst[i] = o1; dst[i + half] = o2; } else { src[i] = o1; src[i + half] = o2; }
+  __align__(16) T ol[8], oh[8];
+  if (head < hq + hkv) {                                // q or k: rotate
+    const float2* cs = rope_tab + (int64_t)pos * half + i0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float2 c = cs[j];
+      ol[j] = from_f32<T>(lo[j] * c.x - hi[j] * c.y);
+      oh[j] = from_f32<T>(hi[j] * c.x + lo[j] * c.y);
     }
   } else {
-    for (int i = threadIdx.x; i < dh; i += blockDim.x) dst[i] = from_f32<T>(ld(i));
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { ol[j] = from_f32<T>(lo[j]); oh[j] = from_f32<T>(hi[j]); }
   }
+  *reinterpret_cast<uint4*>(dst + i0) = *reinterpret_cast<const uint4*>(ol);
+  if (sizeof(T) == 4) *reinterpret_cast<uint4*>(dst + i0 + 4) = *reinterpret_cast<const uint4*>(ol + 4);
+  *reinterpret_cast<uint4*>(dst + half + i0) = *reinterpret_cast<const uint4*>(oh);
+  if (sizeof(T) == 4) *reinterpret_cast<uint4*>(dst + half + i0 + 4) = *reinterpret_cast<const uint4*>(oh + 4);
 }
 
 // act[r, j] = silu(gu[r, 2j]) * gu[r, 2j+1]   (gate/up interleaved by the fused weight layout)
