@@ -342,7 +342,7 @@ __global__ void __launch_bounds__(128) attn_decode_merge_kernel(bf16* __restrict
 #pragma unroll
   for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
   float l_tot = 0.f, m_run = -INFINITY;        // warp-uniform
-  if (row_t[r] >= 0) {
+  {   // rows of finished sequences are merged like any other: nothing downstream reads them
     const int64_t slot0 = ((int64_t)r * hq + head) * n_slots;
     for (int s0 = 0; s0 < n_slots; s0 += 32) {         // one pass for n_slots <= 32, a second for the 33rd
       const int s = s0 + lane;

@@ -201,18 +201,15 @@ __global__ void rope_kv_kernel(T* __restrict__ qkv, const int32_t* __restrict__ 
   const int64_t unit = gid / tph;                       // (row, head)
   if (unit >= (int64_t)rows * heads) return;
   const int r = (int)(unit / heads), head = (int)(unit % heads), i0 = (int)(gid % tph) * 8;
-  const int t = row_t[r];
-  if (t < 0) return;
-  const SeqDesc sd = seqs[row_seq[r]];
-  const int pos = sd.shared_len + t;
-  if (pos >= max_pos) { if (i0 == 0) atomicOr(status, STATUS_BAD_BLOCK); return; }
   const int64_t off = (int64_t)r * heads * dh + (int64_t)head * dh;
   T* src = qkv + off;
+  // the projection values first: these loads do not depend on the row's metadata, so they are in
+  // flight while the (dependent) metadata chain below resolves
   float lo[8], hi[8];
   if (partial) {
 #pragma unroll
     for (int j = 0; j < 8; ++j) { lo[j] = 0.f; hi[j] = 0.f; }
-#pragma unroll 2
+#pragma unroll 4
     for (int s = 0; s < n_splits; ++s) {
       const float4* pl = reinterpret_cast<const float4*>(partial + s * split_stride + off + i0);
       const float4* ph = reinterpret_cast<const float4*>(partial + s * split_stride + off + half + i0);
@@ -231,6 +228,11 @@ __global__ void rope_kv_kernel(T* __restrict__ qkv, const int32_t* __restrict__ 
 #pragma unroll
     for (int j = 0; j < 8; ++j) { lo[j] = to_f32(tl[j]); hi[j] = to_f32(th[j]); }
   }
+  const int t = row_t[r];
+  if (t < 0) return;
+  const SeqDesc sd = seqs[row_seq[r]];
+  const int pos = sd.shared_len + t;
+  if (pos >= max_pos) { if (i0 == 0) atomicOr(status, STATUS_BAD_BLOCK); return; }
   T* dst = src;                                         // q: rotated in place
   if (head >= hq) {
     const int kv = (head - hq) / hkv, kh = (head - hq) % hkv;

@@ -493,7 +493,7 @@ static int run_layers(rpo_ctx* c, int rows) {
     int qkv_splits = 0;
     RPO_TRY(gemm<T>(c, (const T*)w.h, (const T*)L.wqkv, w.qkv, rows, c->qkv_cols, d, EPI_STORE_T, 0, true, &qkv_splits));
     { ProfScope ps(c, KC_ROPE);
-    LAUNCH(c, rope_kv_kernel<T>, ceil_div((int64_t)rows * (s.n_q_heads + 2 * s.n_kv_heads) * (s.head_dim / 16), 256), 256, 0, (T*)w.qkv, w.row_seq, w.row_t,
+    LAUNCH(c, rope_kv_kernel<T>, ceil_div((int64_t)rows * (s.n_q_heads + 2 * s.n_kv_heads) * (s.head_dim / 16), 64), 64, 0, (T*)w.qkv, w.row_seq, w.row_t,
            (const SeqDesc*)w.seqs, c->d_block_table, (const float2*)c->d_rope, kv_pool<T>(c), l, rows, s.n_q_heads,
            s.n_kv_heads, c->lim.max_positions, c->d_status, qkv_splits > 1 ? (const float*)w.partial : (const float*)nullptr,
            qkv_splits, (int64_t)rows * c->qkv_cols); }
