@@ -7,11 +7,13 @@
 // Three uses:
 //   ROWS   (prefill, teacher-forced log-probs): a tile holds 64 consecutive rows of one sequence
 //          for one query head; output is the normalised attention, written as bf16.
-//   SHARED (decode): two kinds of work item in one grid.  A shared item holds the G * (Hq/Hkv) query
-//          rows of one prompt group that share a KV head, and one split of the group's prefix; the
-//          prefix K/V of a group is therefore read once per group, not once per sample.  A private
-//          item holds the Hq/Hkv query rows of one sequence and that sequence's own suffix keys.
-//          Output of both: (m, l, unnormalised O) partials, merged by attn_decode_merge_kernel.
+//   SHARED (decode): a work item holds the G * (Hq/Hkv) query rows of one prompt group that share a
+//          KV head and one split of the group's prefix; the prefix K/V of a group is therefore read
+//          once per group, not once per sample.  After its prefix tiles the item walks its share
+//          of the *suffix* tiles of the group's sequences (dealt round-robin over the splits): a
+//          suffix tile belongs to one sequence, only that sequence's rows see its keys (causally),
+//          and only the warps holding those rows do the math.  Output: (m, l, unnormalised O)
+//          partials per split, merged by attn_decode_merge_kernel.
 #pragma once
 #include "kernels.cuh"
 
@@ -23,8 +25,7 @@ enum FlashMode { FA_ROWS = 0, FA_SHARED = 1 };
 struct FlashArgs {
   const bf16* qkv; int qkv_cols;
   bf16* out; int out_cols;
-  float* part_ml; float* part_o; int n_splits; int split_chunk;   // SHARED: partial slots 0..n_splits-1 = prefix splits,
-  int n_shared_items; int n_seqs;                                 //         slot n_splits = the sequence's own suffix
+  float* part_ml; float* part_o; int n_splits; int split_chunk;   // SHARED: one partial slot per split
   const int32_t* row_seq; const int32_t* row_t; const SeqDesc* seqs; const int32_t* block_table;
   KVPool<bf16> pool; int layer, hq, hkv; float scale_log2;
   const int2* tiles;      // ROWS: (first row, number of rows)
@@ -62,22 +63,27 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 }  // namespace fa
 
-// Tile shape per mode.  Prefill (ROWS) is compute-bound: 64-key tiles, Q fragments kept in registers,
-// two K/V buffers.  Decode (SHARED) is latency-bound: 32-key tiles, Q fragments re-read from shared
-// memory and a register cap so that four CTAs (16 warps) share an SM and hide each other's waits.
+// Tile shape per mode.  Prefill (ROWS) is compute-bound: four warps, 16 query rows each, Q fragments
+// kept in registers.  Decode (SHARED) is bound by the latency of one CTA's chain of tiles: eight
+// warps, the two halves of every 64-key tile go to different warps (KS = 2) with their own softmax
+// state, merged through shared memory at the end; Q fragments are re-read from shared memory and
+// registers are capped so that two such CTAs share an SM.
 template <int MODE> struct FaCfg {
   static constexpr int BN = (MODE == FA_SHARED) ? 64 : 64;     // keys per tile
   static constexpr int NST = (MODE == FA_SHARED) ? 2 : 2;      // K/V ring depth
   static constexpr int MIN_CTAS = (MODE == FA_SHARED) ? 2 : 1;
+  static constexpr int KS = (MODE == FA_SHARED) ? 2 : 1;       // warps sharing the keys of a tile
+  static constexpr int THREADS = FA_THREADS * KS;
   static constexpr bool Q_IN_REGS = (MODE != FA_SHARED);
   template <int DH> static constexpr int smem_bytes() { return (FA_BM + 2 * NST * BN) * DH * 2; }
 };
 
 template <int DH, int MODE>
-__global__ void __launch_bounds__(FA_THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_kernel(FlashArgs a) {
+__global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_kernel(FlashArgs a) {
   pdl_prologue();
   constexpr int NST = FaCfg<MODE>::NST;
   constexpr int BN = FaCfg<MODE>::BN;
+  constexpr int KS = FaCfg<MODE>::KS, THREADS = FaCfg<MODE>::THREADS, WBN = BN / KS;   // WBN: keys of a tile per warp
   constexpr bool Q_IN_REGS = FaCfg<MODE>::Q_IN_REGS;
   constexpr int CH = DH / 8;                 // 16-byte chunks per row
   constexpr int ROW_BYTES = DH * 2;
@@ -90,11 +96,16 @@ __global__ void __launch_bounds__(FA_THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_
   __shared__ int s_qrow[FA_BM];     // qkv row of each tile row (-1: padding)
   __shared__ int s_head[FA_BM];
   __shared__ int s_t[FA_BM];        // private causal limit (-1: nothing visible / inactive)
+  __shared__ int s_pt_sum[FA_BM + 1];   // SHARED: suffix tiles of the tile's sequences, prefix-summed
+  __shared__ int s_pt_t[FA_BM];         //         their newest suffix index t (-1: finished)
+  __shared__ int s_pt_tbl[FA_BM];       //         their private block-table offsets
+  constexpr int BLK_CACHE = (MODE == FA_SHARED) ? 512 : 1;
+  __shared__ int s_blk[BLK_CACHE];      //         block ids of this split's prefix keys (one fetch, not one per tile)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
+  const int mt = warp & 3, kh = warp >> 2;       // 16-row tile of the warp, its share of each tile's keys
   const int rep = a.hq / a.hkv;
-  int kvh, n_rows, split = 0;
-  bool private_item = false;
+  int kvh, n_rows, split = 0, r0 = 0, sq0 = 0, n_sq = 0;
   SeqDesc sd;
   if (MODE == FA_ROWS) {
     const int2 tile = a.tiles[blockIdx.x];
@@ -107,12 +118,13 @@ __global__ void __launch_bounds__(FA_THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_
       s_head[tid] = head;
       s_t[tid] = v ? a.row_t[tile.x + tid] : -1;
     }
-  } else if ((int)blockIdx.x < a.n_shared_items) {
+  } else {
     const int rows_per_group = a.G * rep;
     const int tiles_per_group = (rows_per_group + FA_BM - 1) / FA_BM;
     const int item = blockIdx.x / a.n_splits;
     split = blockIdx.x % a.n_splits;
-    const int grp = item / tiles_per_group, r0 = (item % tiles_per_group) * FA_BM;
+    const int grp = item / tiles_per_group;
+    r0 = (item % tiles_per_group) * FA_BM;
     kvh = blockIdx.y;
     n_rows = min(FA_BM, rows_per_group - r0);
     sd = a.seqs[grp * a.G];
@@ -123,50 +135,69 @@ __global__ void __launch_bounds__(FA_THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_
       s_head[tid] = kvh * rep + (v ? i % rep : 0);
       s_t[tid] = -1;
     }
-  } else {
-    // private item: the rep query heads of one sequence against its own suffix keys 0..t
-    private_item = true;
-    const int seq = blockIdx.x - a.n_shared_items;
-    kvh = blockIdx.y; split = a.n_splits;
-    n_rows = min(rep, FA_BM);
-    sd = a.seqs[a.row_seq[seq]];
-    const int t = a.row_t[seq];
-    if (tid < FA_BM) {
-      const bool v = tid < n_rows;
-      s_qrow[tid] = v ? seq : -1;
-      s_head[tid] = kvh * rep + (v ? tid : 0);
-      s_t[tid] = v ? t : -1;
+    // the sequences that own rows of this tile, their suffix lengths and block tables
+    sq0 = r0 / rep;
+    n_sq = (r0 + n_rows - 1) / rep - sq0 + 1;              // <= FA_BM
+    if (tid < n_sq) {
+      const int seq = grp * a.G + sq0 + tid;
+      const int t = a.row_t[seq];
+      s_pt_t[tid] = t;
+      s_pt_tbl[tid] = a.seqs[a.row_seq[seq]].priv_tbl;
+      s_pt_sum[tid + 1] = (t >= 0) ? t / BN + 1 : 0;       // suffix tiles of this sequence (prefix-summed below)
     }
   }
   __syncthreads();
+  if (MODE == FA_SHARED) {
+    if (tid == 0) {
+      int run = 0;
+      s_pt_sum[0] = 0;
+      for (int i = 0; i < n_sq; ++i) { run += s_pt_sum[i + 1]; s_pt_sum[i + 1] = run; }
+    }
+    __syncthreads();
+  }
 
   // ---- key ranges
-  int sh_begin = 0, sh_end = 0, pr_end = 0;
-  if (MODE == FA_ROWS || private_item) {
-    sh_end = (MODE == FA_ROWS && sd.shared_tbl >= 0) ? sd.shared_len : 0;
+  int sh_begin = 0, sh_end = 0, pr_end = 0, n_pr_tiles;
+  if (MODE == FA_ROWS) {
+    sh_end = (sd.shared_tbl >= 0) ? sd.shared_len : 0;
     int mt = -1;
     for (int i = 0; i < n_rows; ++i) mt = max(mt, s_t[i]);
     pr_end = mt + 1;
+    n_pr_tiles = (pr_end + BN - 1) / BN;
   } else {
     sh_begin = min(sd.shared_len, split * a.split_chunk);
     sh_end = min(sd.shared_len, sh_begin + a.split_chunk);
+    // suffix tile p of the tile's sequences (in sequence order) is handled by split p % n_splits
+    const int total_p = s_pt_sum[n_sq];
+    n_pr_tiles = (total_p > split) ? (total_p - split - 1) / a.n_splits + 1 : 0;
   }
   const int n_sh_tiles = (sh_end - sh_begin + BN - 1) / BN;
-  const int n_pr_tiles = (pr_end + BN - 1) / BN;
+  if (MODE == FA_SHARED) {
+    const int n_blk = min(BLK_CACHE, (sh_end - sh_begin + KV_BLOCK - 1) / KV_BLOCK);   // sh_begin is a multiple of 16
+    for (int e = tid; e < n_blk; e += THREADS) s_blk[e] = a.block_table[sd.shared_tbl + sh_begin / KV_BLOCK + e];
+    __syncthreads();
+  }
   const int n_tiles = n_sh_tiles + n_pr_tiles;
 
   // ---- loaders: TPR threads per K/V row (a thread pair per Q row), interleaved 16-byte chunks
-  constexpr int TPR = FA_THREADS / BN;
+  constexpr int TPR = THREADS / BN, QTPR = THREADS / FA_BM;
   const int lrow = tid / TPR, lpar = tid % TPR;
   auto sw = [&](int row, int chunk) -> uint32_t { return (uint32_t)(row * ROW_BYTES + ((chunk ^ (row & 7)) << 4)); };
+  int ld_cur = 0, mm_cur = 0;                  // SHARED: sequence cursors of the loader / of the math
   auto load_kv = [&](int it, int buf) {
     int tbl, key0, limit;
     if (it < n_sh_tiles) { tbl = sd.shared_tbl; key0 = sh_begin + it * BN; limit = sh_end; }
-    else { tbl = sd.priv_tbl; key0 = (it - n_sh_tiles) * BN; limit = pr_end; }
+    else if (MODE == FA_ROWS) { tbl = sd.priv_tbl; key0 = (it - n_sh_tiles) * BN; limit = pr_end; }
+    else {
+      const int pt = split + (it - n_sh_tiles) * a.n_splits;           // suffix tile number within the row tile
+      while (s_pt_sum[ld_cur + 1] <= pt) ++ld_cur;                      // its sequence (tiles are met in order)
+      tbl = s_pt_tbl[ld_cur]; key0 = (pt - s_pt_sum[ld_cur]) * BN; limit = s_pt_t[ld_cur] + 1;
+    }
     const int u = key0 + lrow;
     const bf16 *kp = nullptr, *vp = nullptr;
     if (u < limit) {
-      const int blk = a.block_table[tbl + u / KV_BLOCK];
+      const int cached = (MODE == FA_SHARED && it < n_sh_tiles) ? (u - sh_begin) / KV_BLOCK : BLK_CACHE;
+      const int blk = (cached < BLK_CACHE) ? s_blk[cached] : a.block_table[tbl + u / KV_BLOCK];
       if (blk >= 0 && blk < a.pool.n_blocks) {
         kp = a.pool.at(a.layer, 0, kvh, blk, u % KV_BLOCK);
         vp = a.pool.at(a.layer, 1, kvh, blk, u % KV_BLOCK);
@@ -183,12 +214,12 @@ __global__ void __launch_bounds__(FA_THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_
     }
   };
   {
-    const int qrow = tid >> 1, qpar = tid & 1;
+    const int qrow = tid / QTPR, qpar = tid % QTPR;
     const int qr = s_qrow[qrow];
     const bf16* qp = (qr >= 0) ? a.qkv + (int64_t)qr * a.qkv_cols + s_head[qrow] * DH : nullptr;
 #pragma unroll
-    for (int j = 0; j < CH / 2; ++j) {
-      const int ch = 2 * j + qpar;
+    for (int j = 0; j < CH / QTPR; ++j) {
+      const int ch = QTPR * j + qpar;
       if (qp) fa::cp_async16(sQ + sw(qrow, ch), qp + ch * 8); else fa::st_zero16(sQ + sw(qrow, ch));
     }
   }
@@ -203,8 +234,8 @@ __global__ void __launch_bounds__(FA_THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_
   for (int i = 0; i < ONT; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
   float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
   uint32_t qf[Q_IN_REGS ? KSTEPS : 1][4];
-  const int r_lo = warp * 16 + g, r_hi = r_lo + 8;
-  const int t_lo = s_t[r_lo], t_hi = s_t[r_hi];
+  const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
+  int t_lo = s_t[r_lo], t_hi = s_t[r_hi];
 
   for (int it = 0; it < n_tiles; ++it) {
     const int buf = it % NST;
@@ -216,44 +247,58 @@ __global__ void __launch_bounds__(FA_THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_
     if (Q_IN_REGS && it == 0) {
 #pragma unroll
       for (int kk = 0; kk < KSTEPS; ++kk)
-        fa::ldsm_x4(sQ + sw(warp * 16 + (lane & 15), kk * 2 + (lane >> 4)), qf[kk][0], qf[kk][1], qf[kk][2], qf[kk][3]);
+        fa::ldsm_x4(sQ + sw(mt * 16 + (lane & 15), kk * 2 + (lane >> 4)), qf[kk][0], qf[kk][1], qf[kk][2], qf[kk][3]);
     }
-    if (warp * 16 < n_rows) {        // warps whose 16 rows are all padding only help with the loads
+    bool warp_has_work = mt * 16 < n_rows;        // warps whose 16 rows are all padding only help with the loads
+    int suffix_key0 = 0;
+    if (MODE == FA_SHARED && it >= n_sh_tiles) {
+      // suffix tile of one sequence: visible to that sequence's rows only, keys 0..t
+      const int pt = split + (it - n_sh_tiles) * a.n_splits;
+      while (s_pt_sum[mm_cur + 1] <= pt) ++mm_cur;
+      const int row_first = (sq0 + mm_cur) * rep - r0, row_last = row_first + rep - 1;   // tile-local, may stick out
+      const int t_own = s_pt_t[mm_cur];
+      suffix_key0 = (pt - s_pt_sum[mm_cur]) * BN;
+      t_lo = (r_lo >= row_first && r_lo <= row_last) ? t_own : -1;
+      t_hi = (r_hi >= row_first && r_hi <= row_last) ? t_own : -1;
+      warp_has_work = warp_has_work && (mt * 16 <= row_last) && (mt * 16 + 15 >= row_first) &&
+                      (suffix_key0 + kh * WBN <= t_own);
+    }
+    if (warp_has_work) {
     // ---- S = Q K^T
-    float s[BN / 8][4];
+    float s[WBN / 8][4];
 #pragma unroll
-    for (int j = 0; j < BN / 8; ++j) { s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f; }
+    for (int j = 0; j < WBN / 8; ++j) { s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f; }
     const uint32_t kb = sK + buf * TILE_BYTES, vb = sV + buf * TILE_BYTES;
 #pragma unroll
     for (int kk = 0; kk < KSTEPS; ++kk) {
       const int qi = Q_IN_REGS ? kk : 0;
       if (!Q_IN_REGS)
-        fa::ldsm_x4(sQ + sw(warp * 16 + (lane & 15), kk * 2 + (lane >> 4)), qf[0][0], qf[0][1], qf[0][2], qf[0][3]);
+        fa::ldsm_x4(sQ + sw(mt * 16 + (lane & 15), kk * 2 + (lane >> 4)), qf[0][0], qf[0][1], qf[0][2], qf[0][3]);
 #pragma unroll
-      for (int jp = 0; jp < BN / 16; ++jp) {
+      for (int jp = 0; jp < WBN / 16; ++jp) {
         uint32_t b0, b1, b2, b3;
-        fa::ldsm_x4(kb + sw(jp * 16 + (lane & 7) + ((lane >> 4) << 3), kk * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
+        fa::ldsm_x4(kb + sw(kh * WBN + jp * 16 + (lane & 7) + ((lane >> 4) << 3), kk * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
         fa::mma_bf16(s[2 * jp], qf[qi], b0, b1);
         fa::mma_bf16(s[2 * jp + 1], qf[qi], b2, b3);
       }
     }
     // ---- mask + online softmax (base-2 exponent domain)
     const bool shared_tile = it < n_sh_tiles;
-    const int key0 = shared_tile ? sh_begin + it * BN : (it - n_sh_tiles) * BN;
+    const int key0 = shared_tile ? sh_begin + it * BN : (MODE == FA_ROWS ? (it - n_sh_tiles) * BN : suffix_key0);
     float mx_lo = -INFINITY, mx_hi = -INFINITY;
     if (shared_tile && key0 + BN <= sh_end) {          // tile fully inside the visible prefix: no masking
 #pragma unroll
-      for (int j = 0; j < BN / 8; ++j) {
+      for (int j = 0; j < WBN / 8; ++j) {
 #pragma unroll
         for (int c = 0; c < 4; ++c) s[j][c] *= a.scale_log2;
         mx_lo = fmaxf(mx_lo, fmaxf(s[j][0], s[j][1])); mx_hi = fmaxf(mx_hi, fmaxf(s[j][2], s[j][3]));
       }
     } else {
 #pragma unroll
-      for (int j = 0; j < BN / 8; ++j) {
+      for (int j = 0; j < WBN / 8; ++j) {
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          const int key = key0 + j * 8 + tq * 2 + (c & 1);
+          const int key = key0 + kh * WBN + j * 8 + tq * 2 + (c & 1);
           const bool vis = shared_tile ? (key < sh_end) : (key <= ((c & 2) ? t_hi : t_lo));
           const float v = vis ? s[j][c] * a.scale_log2 : -INFINITY;
           s[j][c] = v;
@@ -268,9 +313,9 @@ __global__ void __launch_bounds__(FA_THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_
     const float c_lo = fa::ex2(m_lo - mu_lo), c_hi = fa::ex2(m_hi - mu_hi);
     m_lo = mn_lo; m_hi = mn_hi;
     float ps_lo = 0.f, ps_hi = 0.f;
-    uint32_t pf[BN / 16][4];
+    uint32_t pf[WBN / 16][4];
 #pragma unroll
-    for (int j = 0; j < BN / 8; ++j) {
+    for (int j = 0; j < WBN / 8; ++j) {
       const float p0 = fa::ex2(s[j][0] - mu_lo), p1 = fa::ex2(s[j][1] - mu_lo);
       const float p2 = fa::ex2(s[j][2] - mu_hi), p3 = fa::ex2(s[j][3] - mu_hi);
       ps_lo += p0 + p1; ps_hi += p2 + p3;
@@ -284,11 +329,11 @@ __global__ void __launch_bounds__(FA_THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_
     }
     // ---- O += P V
 #pragma unroll
-    for (int kk = 0; kk < BN / 16; ++kk) {
+    for (int kk = 0; kk < WBN / 16; ++kk) {
 #pragma unroll
       for (int np = 0; np < ONT / 2; ++np) {
         uint32_t b0, b1, b2, b3;
-        fa::ldsm_x4_t(vb + sw(kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), np * 2 + (lane >> 4)), b0, b1, b2, b3);
+        fa::ldsm_x4_t(vb + sw(kh * WBN + kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), np * 2 + (lane >> 4)), b0, b1, b2, b3);
         fa::mma_bf16(o[2 * np], pf[kk], b0, b1);
         fa::mma_bf16(o[2 * np + 1], pf[kk], b2, b3);
       }
@@ -297,6 +342,39 @@ __global__ void __launch_bounds__(FA_THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_
     __syncthreads();
   }
   fa::cp_wait<0>();
+  if (KS == 2) {
+    // The warps of the second key half hand their state to the warp holding the same rows in the
+    // first half, thread to thread ([value][thread] layout: no bank conflicts), through the K/V ring
+    // (free after the loop's last barrier).  m is uniform over a quad, l is still a per-lane partial.
+    float* xch = reinterpret_cast<float*>(fsm + FA_BM * ROW_BYTES);
+    const int xt = mt * 32 + lane;
+    if (kh == 1) {
+#pragma unroll
+      for (int i = 0; i < ONT; ++i) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) xch[(i * 4 + c) * FA_THREADS + xt] = o[i][c];
+      }
+      xch[(ONT * 4 + 0) * FA_THREADS + xt] = m_lo; xch[(ONT * 4 + 1) * FA_THREADS + xt] = m_hi;
+      xch[(ONT * 4 + 2) * FA_THREADS + xt] = l_lo; xch[(ONT * 4 + 3) * FA_THREADS + xt] = l_hi;
+    }
+    __syncthreads();
+    if (kh == 1) return;
+    const float mb_lo = xch[(ONT * 4 + 0) * FA_THREADS + xt], mb_hi = xch[(ONT * 4 + 1) * FA_THREADS + xt];
+    const float mn_lo = fmaxf(m_lo, mb_lo), mn_hi = fmaxf(m_hi, mb_hi);
+    const float mu_lo = (mn_lo == -INFINITY) ? 0.f : mn_lo, mu_hi = (mn_hi == -INFINITY) ? 0.f : mn_hi;
+    const float ca_lo = fa::ex2(m_lo - mu_lo), cb_lo = fa::ex2(mb_lo - mu_lo);
+    const float ca_hi = fa::ex2(m_hi - mu_hi), cb_hi = fa::ex2(mb_hi - mu_hi);
+    l_lo = l_lo * ca_lo + xch[(ONT * 4 + 2) * FA_THREADS + xt] * cb_lo;
+    l_hi = l_hi * ca_hi + xch[(ONT * 4 + 3) * FA_THREADS + xt] * cb_hi;
+    m_lo = mn_lo; m_hi = mn_hi;
+#pragma unroll
+    for (int i = 0; i < ONT; ++i) {
+      o[i][0] = o[i][0] * ca_lo + xch[(i * 4 + 0) * FA_THREADS + xt] * cb_lo;
+      o[i][1] = o[i][1] * ca_lo + xch[(i * 4 + 1) * FA_THREADS + xt] * cb_lo;
+      o[i][2] = o[i][2] * ca_hi + xch[(i * 4 + 2) * FA_THREADS + xt] * cb_hi;
+      o[i][3] = o[i][3] * ca_hi + xch[(i * 4 + 3) * FA_THREADS + xt] * cb_hi;
+    }
+  }
   l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1); l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
   l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1); l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
 
@@ -314,7 +392,7 @@ __global__ void __launch_bounds__(FA_THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_
       for (int i = 0; i < ONT; ++i)
         *(uint32_t*)(dst + i * 8 + tq * 2) = fa::pack_bf16(o[i][half * 2] * inv, o[i][half * 2 + 1] * inv);
     } else {
-      const int64_t slot = ((int64_t)qr * a.hq + s_head[r]) * (a.n_splits + 1) + split;
+      const int64_t slot = ((int64_t)qr * a.hq + s_head[r]) * a.n_splits + split;
       if (tq == 0) { a.part_ml[slot * 2] = m; a.part_ml[slot * 2 + 1] = l; }
       float* dst = a.part_o + slot * DH;
 #pragma unroll

@@ -418,7 +418,7 @@ static int launch_flash(rpo_ctx* c, const FlashArgs& a, dim3 grid) {
     CUDA_TRY(cudaFuncSetAttribute(flash_attn_kernel<DH, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     attr_done = true;
   }
-  LAUNCH(c, (flash_attn_kernel<DH, MODE>), grid, FA_THREADS, smem, a);
+  LAUNCH(c, (flash_attn_kernel<DH, MODE>), grid, FaCfg<MODE>::THREADS, smem, a);
   return RPO_OK;
 }
 
@@ -443,14 +443,13 @@ static int attention(rpo_ctx* c, int layer, int rows) {
         return s.head_dim == 128 ? launch_flash<128, FA_ROWS>(c, a, grid) : launch_flash<64, FA_ROWS>(c, a, grid);
       }
       const int rep = s.n_q_heads / s.n_kv_heads;
-      a.n_shared_items = c->attn_groups * ceil_div(c->attn_G * rep, FA_BM) * c->attn_splits; a.n_seqs = rows;
-      dim3 grid(a.n_shared_items + rows, s.n_kv_heads);
+      dim3 grid(c->attn_groups * ceil_div(c->attn_G * rep, FA_BM) * c->attn_splits, s.n_kv_heads);
       RPO_TRY((s.head_dim == 128 ? launch_flash<128, FA_SHARED>(c, a, grid) : launch_flash<64, FA_SHARED>(c, a, grid)));
       const int mgrid = ceil_div((int64_t)rows * s.n_q_heads, 4);
       if (s.head_dim == 128)
-        LAUNCH(c, (attn_decode_merge_kernel<128>), mgrid, 128, 0, a.out, a.part_ml, a.part_o, a.n_splits + 1, w.row_t, rows, a.hq);
+        LAUNCH(c, (attn_decode_merge_kernel<128>), mgrid, 128, 0, a.out, a.part_ml, a.part_o, a.n_splits, w.row_t, rows, a.hq);
       else
-        LAUNCH(c, (attn_decode_merge_kernel<64>), mgrid, 128, 0, a.out, a.part_ml, a.part_o, a.n_splits + 1, w.row_t, rows, a.hq);
+        LAUNCH(c, (attn_decode_merge_kernel<64>), mgrid, 128, 0, a.out, a.part_ml, a.part_o, a.n_splits, w.row_t, rows, a.hq);
       return RPO_OK;
     }
   }
