@@ -70,18 +70,19 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // registers are capped so that two such CTAs share an SM.
 template <int MODE> struct FaCfg {
   static constexpr int BN = (MODE == FA_SHARED) ? 64 : 64;     // keys per tile
-  static constexpr int NST = (MODE == FA_SHARED) ? 2 : 2;      // K/V ring depth
+  static constexpr int NSK = (MODE == FA_SHARED) ? 3 : 2;      // K ring depth: K tiles are fetched NSK-1 tiles ahead,
+  static constexpr int NSV = 2;                                //   V tiles (needed half a tile later) NSV-1 ahead
   static constexpr int MIN_CTAS = (MODE == FA_SHARED) ? 2 : 1;
   static constexpr int KS = (MODE == FA_SHARED) ? 2 : 1;       // warps sharing the keys of a tile
   static constexpr int THREADS = FA_THREADS * KS;
   static constexpr bool Q_IN_REGS = (MODE != FA_SHARED);
-  template <int DH> static constexpr int smem_bytes() { return (FA_BM + 2 * NST * BN) * DH * 2; }
+  template <int DH> static constexpr int smem_bytes() { return (FA_BM + (NSK + NSV) * BN) * DH * 2; }
 };
 
 template <int DH, int MODE>
 __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_kernel(FlashArgs a) {
   pdl_prologue();
-  constexpr int NST = FaCfg<MODE>::NST;
+  constexpr int NSK = FaCfg<MODE>::NSK, NSV = FaCfg<MODE>::NSV;
   constexpr int BN = FaCfg<MODE>::BN;
   constexpr int KS = FaCfg<MODE>::KS, THREADS = FaCfg<MODE>::THREADS, WBN = BN / KS;   // WBN: keys of a tile per warp
   constexpr bool Q_IN_REGS = FaCfg<MODE>::Q_IN_REGS;
@@ -91,8 +92,8 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
   constexpr int KSTEPS = DH / 16, ONT = DH / 8;
   extern __shared__ __align__(128) uint8_t fsm[];
   const uint32_t sQ = (uint32_t)__cvta_generic_to_shared(fsm);
-  const uint32_t sK = sQ + FA_BM * ROW_BYTES;          // NST buffers
-  const uint32_t sV = sK + NST * TILE_BYTES;           // NST buffers
+  const uint32_t sK = sQ + FA_BM * ROW_BYTES;          // NSK buffers
+  const uint32_t sV = sK + NSK * TILE_BYTES;           // NSV buffers
   __shared__ int s_qrow[FA_BM];     // qkv row of each tile row (-1: padding)
   __shared__ int s_head[FA_BM];
   __shared__ int s_t[FA_BM];        // private causal limit (-1: nothing visible / inactive)
@@ -106,7 +107,18 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
   const int mt = warp & 3, kh = warp >> 2;       // 16-row tile of the warp, its share of each tile's keys
   const int rep = a.hq / a.hkv;
   int kvh, n_rows, split = 0, r0 = 0, sq0 = 0, n_sq = 0;
+  int sh_begin = 0, sh_end = 0;
   SeqDesc sd;
+  auto sw = [&](int row, int chunk) -> uint32_t { return (uint32_t)(row * ROW_BYTES + ((chunk ^ (row & 7)) << 4)); };
+  constexpr int QTPR = THREADS / FA_BM;          // threads per Q row
+  auto load_q = [&](int qrow, int qpar, int qr, int qhead) {   // qr: qkv row (-1: zero padding)
+    const bf16* qp = (qr >= 0) ? a.qkv + (int64_t)qr * a.qkv_cols + qhead * DH : nullptr;
+#pragma unroll
+    for (int j = 0; j < CH / QTPR; ++j) {
+      const int ch = QTPR * j + qpar;
+      if (qp) fa::cp_async16(sQ + sw(qrow, ch), qp + ch * 8); else fa::st_zero16(sQ + sw(qrow, ch));
+    }
+  };
   if (MODE == FA_ROWS) {
     const int2 tile = a.tiles[blockIdx.x];
     const int head = blockIdx.y;
@@ -127,6 +139,11 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
     r0 = (item % tiles_per_group) * FA_BM;
     kvh = blockIdx.y;
     n_rows = min(FA_BM, rows_per_group - r0);
+    {   // the Q rows go first: their addresses need nothing from memory
+      const int qrow = tid / QTPR, i = r0 + qrow;
+      const bool v = qrow < n_rows;
+      load_q(qrow, tid % QTPR, v ? grp * a.G + i / rep : -1, kvh * rep + (v ? i % rep : 0));
+    }
     sd = a.seqs[grp * a.G];
     if (tid < FA_BM) {
       const bool v = tid < n_rows;
@@ -142,9 +159,14 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
       const int seq = grp * a.G + sq0 + tid;
       const int t = a.row_t[seq];
       s_pt_t[tid] = t;
-      s_pt_tbl[tid] = a.seqs[a.row_seq[seq]].priv_tbl;
+      s_pt_tbl[tid] = a.seqs[seq].priv_tbl;               // decode passes: row i is sequence i
       s_pt_sum[tid + 1] = (t >= 0) ? t / BN + 1 : 0;       // suffix tiles of this sequence (prefix-summed below)
     }
+    // block ids of this split's prefix keys: one fetch up front instead of one per tile
+    sh_begin = min(sd.shared_len, split * a.split_chunk);  // a multiple of 16
+    sh_end = min(sd.shared_len, sh_begin + a.split_chunk);
+    const int n_blk = min(BLK_CACHE, (sh_end - sh_begin + KV_BLOCK - 1) / KV_BLOCK);
+    for (int e = tid; e < n_blk; e += THREADS) s_blk[e] = a.block_table[sd.shared_tbl + sh_begin / KV_BLOCK + e];
   }
   __syncthreads();
   if (MODE == FA_SHARED) {
@@ -157,7 +179,7 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
   }
 
   // ---- key ranges
-  int sh_begin = 0, sh_end = 0, pr_end = 0, n_pr_tiles;
+  int pr_end = 0, n_pr_tiles;
   if (MODE == FA_ROWS) {
     sh_end = (sd.shared_tbl >= 0) ? sd.shared_len : 0;
     int mt = -1;
@@ -165,42 +187,34 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
     pr_end = mt + 1;
     n_pr_tiles = (pr_end + BN - 1) / BN;
   } else {
-    sh_begin = min(sd.shared_len, split * a.split_chunk);
-    sh_end = min(sd.shared_len, sh_begin + a.split_chunk);
     // suffix tile p of the tile's sequences (in sequence order) is handled by split p % n_splits
     const int total_p = s_pt_sum[n_sq];
     n_pr_tiles = (total_p > split) ? (total_p - split - 1) / a.n_splits + 1 : 0;
   }
   const int n_sh_tiles = (sh_end - sh_begin + BN - 1) / BN;
-  if (MODE == FA_SHARED) {
-    const int n_blk = min(BLK_CACHE, (sh_end - sh_begin + KV_BLOCK - 1) / KV_BLOCK);   // sh_begin is a multiple of 16
-    for (int e = tid; e < n_blk; e += THREADS) s_blk[e] = a.block_table[sd.shared_tbl + sh_begin / KV_BLOCK + e];
-    __syncthreads();
-  }
   const int n_tiles = n_sh_tiles + n_pr_tiles;
 
   // ---- loaders: TPR threads per K/V row (a thread pair per Q row), interleaved 16-byte chunks
-  constexpr int TPR = THREADS / BN, QTPR = THREADS / FA_BM;
+  constexpr int TPR = THREADS / BN;
   const int lrow = tid / TPR, lpar = tid % TPR;
-  auto sw = [&](int row, int chunk) -> uint32_t { return (uint32_t)(row * ROW_BYTES + ((chunk ^ (row & 7)) << 4)); };
-  int ld_cur = 0, mm_cur = 0;                  // SHARED: sequence cursors of the loader / of the math
-  auto load_kv = [&](int it, int buf) {
+  int ld_cur = 0, ldv_cur = 0, mm_cur = 0;     // SHARED: sequence cursors of the K loader, the V loader, the math
+  auto load_tile = [&](int it, int buf, bool want_v) {   // K (cursor ld_cur) or V (cursor ldv_cur) rows of tile `it`
     int tbl, key0, limit;
     if (it < n_sh_tiles) { tbl = sd.shared_tbl; key0 = sh_begin + it * BN; limit = sh_end; }
     else if (MODE == FA_ROWS) { tbl = sd.priv_tbl; key0 = (it - n_sh_tiles) * BN; limit = pr_end; }
     else {
       const int pt = split + (it - n_sh_tiles) * a.n_splits;           // suffix tile number within the row tile
-      while (s_pt_sum[ld_cur + 1] <= pt) ++ld_cur;                      // its sequence (tiles are met in order)
-      tbl = s_pt_tbl[ld_cur]; key0 = (pt - s_pt_sum[ld_cur]) * BN; limit = s_pt_t[ld_cur] + 1;
+      int& cur = want_v ? ldv_cur : ld_cur;
+      while (s_pt_sum[cur + 1] <= pt) ++cur;                            // its sequence (tiles are met in order)
+      tbl = s_pt_tbl[cur]; key0 = (pt - s_pt_sum[cur]) * BN; limit = s_pt_t[cur] + 1;
     }
     const int u = key0 + lrow;
-    const bf16 *kp = nullptr, *vp = nullptr;
+    const bf16* kp = nullptr;
     if (u < limit) {
       const int cached = (MODE == FA_SHARED && it < n_sh_tiles) ? (u - sh_begin) / KV_BLOCK : BLK_CACHE;
       const int blk = (cached < BLK_CACHE) ? s_blk[cached] : a.block_table[tbl + u / KV_BLOCK];
       if (blk >= 0 && blk < a.pool.n_blocks) {
-        kp = a.pool.at(a.layer, 0, kvh, blk, u % KV_BLOCK);
-        vp = a.pool.at(a.layer, 1, kvh, blk, u % KV_BLOCK);
+        kp = a.pool.at(a.layer, want_v ? 1 : 0, kvh, blk, u % KV_BLOCK);
       } else {
         atomicOr(a.status, STATUS_BAD_BLOCK);
       }
@@ -209,25 +223,17 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
     for (int j = 0; j < CH / TPR; ++j) {
       const int ch = TPR * j + lpar;
       const uint32_t off = sw(lrow, ch);
-      if (kp) { fa::cp_async16(sK + buf * TILE_BYTES + off, kp + ch * 8); fa::cp_async16(sV + buf * TILE_BYTES + off, vp + ch * 8); }
-      else { fa::st_zero16(sK + buf * TILE_BYTES + off); fa::st_zero16(sV + buf * TILE_BYTES + off); }
+      const uint32_t dst = (want_v ? sV : sK) + buf * TILE_BYTES + off;
+      if (kp) fa::cp_async16(dst, kp + ch * 8); else fa::st_zero16(dst);
     }
   };
-  {
-    const int qrow = tid / QTPR, qpar = tid % QTPR;
-    const int qr = s_qrow[qrow];
-    const bf16* qp = (qr >= 0) ? a.qkv + (int64_t)qr * a.qkv_cols + s_head[qrow] * DH : nullptr;
+  if (MODE == FA_ROWS) load_q(tid / QTPR, tid % QTPR, s_qrow[tid / QTPR], s_head[tid / QTPR]);
+  // prologue: K tiles 0..NSK-2 (the first group also carries Q), then V tiles 0..NSV-2.  Every
+  // step commits a group even when it loads nothing, so that the wait counts below stay constant.
 #pragma unroll
-    for (int j = 0; j < CH / QTPR; ++j) {
-      const int ch = QTPR * j + qpar;
-      if (qp) fa::cp_async16(sQ + sw(qrow, ch), qp + ch * 8); else fa::st_zero16(sQ + sw(qrow, ch));
-    }
-  }
+  for (int st = 0; st < NSK - 1; ++st) { if (st < n_tiles) load_tile(st, st, false); fa::cp_commit(); }
 #pragma unroll
-  for (int st = 0; st < NST - 1; ++st) {      // prologue: tiles 0..NST-2 (the first group also carries Q)
-    if (st < n_tiles) load_kv(st, st);
-    fa::cp_commit();
-  }
+  for (int st = 0; st < NSV - 1; ++st) { if (st < n_tiles) load_tile(st, st, true); fa::cp_commit(); }
 
   float o[ONT][4];
 #pragma unroll
@@ -238,12 +244,14 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
   int t_lo = s_t[r_lo], t_hi = s_t[r_hi];
 
   for (int it = 0; it < n_tiles; ++it) {
-    const int buf = it % NST;
-    // tile it+NST-1 goes into the buffer that iteration it-1 finished reading (its trailing barrier)
-    if (it + NST - 1 < n_tiles) load_kv(it + NST - 1, (it + NST - 1) % NST);
+    // K tile it+NSK-1 goes into the buffer whose tile every warp finished multiplying before it
+    // passed the V barrier of iteration it-1.  Groups younger than K(it): NSK+NSV-2.
+    if (it + NSK - 1 < n_tiles) load_tile(it + NSK - 1, (it + NSK - 1) % NSK, false);
     fa::cp_commit();
-    fa::cp_wait<NST - 1>();                   // all but the newest NST-1 groups have landed: tile `it` is in
-    __syncthreads();
+    fa::cp_wait<NSK + NSV - 2>();
+    __syncthreads();                          // K(it) visible to all; every warp is done with P V of tile it-1
+    if (it + NSV - 1 < n_tiles) load_tile(it + NSV - 1, (it + NSV - 1) % NSV, true);
+    fa::cp_commit();
     if (Q_IN_REGS && it == 0) {
 #pragma unroll
       for (int kk = 0; kk < KSTEPS; ++kk)
@@ -263,12 +271,13 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
       warp_has_work = warp_has_work && (mt * 16 <= row_last) && (mt * 16 + 15 >= row_first) &&
                       (suffix_key0 + kh * WBN <= t_own);
     }
+    uint32_t pf[WBN / 16][4];                     // P as bf16 A-fragments, handed from the softmax to P V
     if (warp_has_work) {
     // ---- S = Q K^T
     float s[WBN / 8][4];
 #pragma unroll
     for (int j = 0; j < WBN / 8; ++j) { s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f; }
-    const uint32_t kb = sK + buf * TILE_BYTES, vb = sV + buf * TILE_BYTES;
+    const uint32_t kb = sK + (it % NSK) * TILE_BYTES;
 #pragma unroll
     for (int kk = 0; kk < KSTEPS; ++kk) {
       const int qi = Q_IN_REGS ? kk : 0;
@@ -313,7 +322,6 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
     const float c_lo = fa::ex2(m_lo - mu_lo), c_hi = fa::ex2(m_hi - mu_hi);
     m_lo = mn_lo; m_hi = mn_hi;
     float ps_lo = 0.f, ps_hi = 0.f;
-    uint32_t pf[WBN / 16][4];
 #pragma unroll
     for (int j = 0; j < WBN / 8; ++j) {
       const float p0 = fa::ex2(s[j][0] - mu_lo), p1 = fa::ex2(s[j][1] - mu_lo);
@@ -327,7 +335,12 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
 #pragma unroll
       for (int i = 0; i < ONT; ++i) { o[i][0] *= c_lo; o[i][1] *= c_lo; o[i][2] *= c_hi; o[i][3] *= c_hi; }
     }
+    }
+    fa::cp_wait<2 * (NSV - 1)>();             // groups younger than V(it): 2 per iteration of look-ahead
+    __syncthreads();                          // V(it) visible to all; every warp is done with Q K^T of tile it
+    if (warp_has_work) {
     // ---- O += P V
+    const uint32_t vb = sV + (it % NSV) * TILE_BYTES;
 #pragma unroll
     for (int kk = 0; kk < WBN / 16; ++kk) {
 #pragma unroll
@@ -339,10 +352,10 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
       }
     }
     }
-    __syncthreads();
   }
   fa::cp_wait<0>();
   if (KS == 2) {
+    __syncthreads();                          // every warp is done with the ring
     // The warps of the second key half hand their state to the warp holding the same rows in the
     // first half, thread to thread ([value][thread] layout: no bank conflicts), through the K/V ring
     // (free after the loop's last barrier).  m is uniform over a quad, l is still a per-lane partial.
