@@ -1,6 +1,11 @@
 // bf16 attention on tensor cores (mma.sync m16n8k16, float32 softmax and accumulation) over the
-// paged KV cache, flash style: a 64-row query tile stays in registers while 64-key K/V tiles are
-// streamed through a double-buffered, XOR-swizzled shared-memory ring with cp.async.
+// paged KV cache, flash style.  A dedicated producer warp streams 64-key K and V tiles into two
+// shared-memory rings with bulk async copies (cp.async.bulk: ONE contiguous copy per 16-token KV
+// block, found through the block table; the pool already stores a block in the swizzled layout
+// ldmatrix wants, see KVPool), guarded by full/empty mbarriers; the consumer warps never issue a
+// global load in the tile loop and do no address arithmetic for K/V.  Keys past
+// the end of a segment are masked, not zero-filled: the pool is zeroed at creation, so whatever a
+// box brings along is finite.  Every mbarrier wait is bounded (status bit 0 on expiry).
 //
 // Key space of a query row = [shared segment: the group's prefix blocks, all visible]
 //                         ++ [private segment: the sequence's own blocks, keys 0..t visible].
@@ -15,6 +20,7 @@
 //          and only the warps holding those rows do the math.  Output: (m, l, unnormalised O)
 //          partials per split, merged by attn_decode_merge_kernel.
 #pragma once
+#include "gemm_tc.cuh"
 #include "kernels.cuh"
 
 namespace rpo {
@@ -72,15 +78,16 @@ template <int MODE> struct FaCfg {
   static constexpr int BN = (MODE == FA_SHARED) ? 64 : 64;     // keys per tile
   static constexpr int NSK = (MODE == FA_SHARED) ? 3 : 2;      // K ring depth: K tiles are fetched NSK-1 tiles ahead,
   static constexpr int NSV = 2;                                //   V tiles (needed half a tile later) NSV-1 ahead
-  static constexpr int MIN_CTAS = (MODE == FA_SHARED) ? 2 : 1;
-  static constexpr int KS = (MODE == FA_SHARED) ? 2 : 1;       // warps sharing the keys of a tile
+  static constexpr int MIN_CTAS = 2;
+  static constexpr int KS = (MODE == FA_SHARED) ? 1 : 1;       // warps sharing the keys of a tile
   static constexpr int THREADS = FA_THREADS * KS;
-  static constexpr bool Q_IN_REGS = (MODE != FA_SHARED);
-  template <int DH> static constexpr int smem_bytes() { return (FA_BM + (NSK + NSV) * BN) * DH * 2; }
+  static constexpr bool Q_IN_REGS = true;
+  template <int DH> static constexpr int smem_bytes() { return (FA_BM + (NSK + NSV) * BN) * DH * 2 + 1024 /*align*/ + 128 /*barriers*/; }
 };
 
 template <int DH, int MODE>
-__global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) flash_attn_kernel(FlashArgs a) {
+__global__ void __launch_bounds__(FaCfg<MODE>::THREADS + 32, FaCfg<MODE>::MIN_CTAS)
+flash_attn_kernel(FlashArgs a) {
   pdl_prologue();
   constexpr int NSK = FaCfg<MODE>::NSK, NSV = FaCfg<MODE>::NSV;
   constexpr int BN = FaCfg<MODE>::BN;
@@ -90,10 +97,17 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
   constexpr int ROW_BYTES = DH * 2;
   constexpr int TILE_BYTES = BN * ROW_BYTES;
   constexpr int KSTEPS = DH / 16, ONT = DH / 8;
-  extern __shared__ __align__(128) uint8_t fsm[];
-  const uint32_t sQ = (uint32_t)__cvta_generic_to_shared(fsm);
-  const uint32_t sK = sQ + FA_BM * ROW_BYTES;          // NSK buffers
-  const uint32_t sV = sK + NSK * TILE_BYTES;           // NSV buffers
+  constexpr int BLK_BYTES = KV_BLOCK * ROW_BYTES;   // one KV block of K (or V) for one head
+  constexpr int PER_HALF = DH < 64 ? DH : 64;       // dims per 128-byte (or shorter) row of the block layout
+  constexpr int NW = THREADS / 32;           // consumer warps; warp NW is the producer
+  extern __shared__ uint8_t fsm_raw[];
+  uint8_t* fsm = (uint8_t*)(((uintptr_t)fsm_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t sK = (uint32_t)__cvta_generic_to_shared(fsm);   // NSK buffers (1024-byte aligned: swizzle atoms)
+  const uint32_t sV = sK + NSK * TILE_BYTES;                       // NSV buffers
+  const uint32_t sQ = sV + NSV * TILE_BYTES;
+  uint64_t* bars = (uint64_t*)(fsm + (NSK + NSV) * TILE_BYTES + FA_BM * ROW_BYTES);
+  uint64_t *full_k = bars, *empty_k = bars + NSK, *full_v = bars + 2 * NSK, *empty_v = bars + 2 * NSK + NSV;
+  __shared__ int s_abort;
   __shared__ int s_qrow[FA_BM];     // qkv row of each tile row (-1: padding)
   __shared__ int s_head[FA_BM];
   __shared__ int s_t[FA_BM];        // private causal limit (-1: nothing visible / inactive)
@@ -109,7 +123,20 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
   int kvh, n_rows, split = 0, r0 = 0, sq0 = 0, n_sq = 0;
   int sh_begin = 0, sh_end = 0;
   SeqDesc sd;
+  // Q tile: rows of DH*2 bytes, 16-byte chunks XOR-swizzled by the row.  K/V tiles: BN/16 blocks
+  // back to back, each in the pool's block layout [half][token][chunk ^ (token & 7)].
   auto sw = [&](int row, int chunk) -> uint32_t { return (uint32_t)(row * ROW_BYTES + ((chunk ^ (row & 7)) << 4)); };
+  auto swkv = [&](int row, int chunk) -> uint32_t {
+    constexpr int CPH = PER_HALF / 8;          // chunks per half row
+    return (uint32_t)((row >> 4) * BLK_BYTES + (chunk / CPH) * (KV_BLOCK * PER_HALF * 2) + (row & 15) * (PER_HALF * 2) +
+                      (((chunk % CPH) ^ (row & 7)) << 4));
+  };
+  if (tid == 0) {
+    for (int i = 0; i < NSK; ++i) { tc::mbar_init(&full_k[i], 1); tc::mbar_init(&empty_k[i], NW); }
+    for (int i = 0; i < NSV; ++i) { tc::mbar_init(&full_v[i], 1); tc::mbar_init(&empty_v[i], NW); }
+    s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
   constexpr int QTPR = THREADS / FA_BM;          // threads per Q row
   auto load_q = [&](int qrow, int qpar, int qr, int qhead) {   // qr: qkv row (-1: zero padding)
     const bf16* qp = (qr >= 0) ? a.qkv + (int64_t)qr * a.qkv_cols + qhead * DH : nullptr;
@@ -139,7 +166,7 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
     r0 = (item % tiles_per_group) * FA_BM;
     kvh = blockIdx.y;
     n_rows = min(FA_BM, rows_per_group - r0);
-    {   // the Q rows go first: their addresses need nothing from memory
+    if (tid < THREADS) {   // the Q rows go first: their addresses need nothing from memory
       const int qrow = tid / QTPR, i = r0 + qrow;
       const bool v = qrow < n_rows;
       load_q(qrow, tid % QTPR, v ? grp * a.G + i / rep : -1, kvh * rep + (v ? i % rep : 0));
@@ -155,7 +182,7 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
     // the sequences that own rows of this tile, their suffix lengths and block tables
     sq0 = r0 / rep;
     n_sq = (r0 + n_rows - 1) / rep - sq0 + 1;              // <= FA_BM
-    if (tid < n_sq) {
+    if (tid < n_sq) {                                      // n_sq <= FA_BM <= THREADS
       const int seq = grp * a.G + sq0 + tid;
       const int t = a.row_t[seq];
       s_pt_t[tid] = t;
@@ -166,7 +193,7 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
     sh_begin = min(sd.shared_len, split * a.split_chunk);  // a multiple of 16
     sh_end = min(sd.shared_len, sh_begin + a.split_chunk);
     const int n_blk = min(BLK_CACHE, (sh_end - sh_begin + KV_BLOCK - 1) / KV_BLOCK);
-    for (int e = tid; e < n_blk; e += THREADS) s_blk[e] = a.block_table[sd.shared_tbl + sh_begin / KV_BLOCK + e];
+    for (int e = tid; e < n_blk; e += THREADS + 32) s_blk[e] = a.block_table[sd.shared_tbl + sh_begin / KV_BLOCK + e];
   }
   __syncthreads();
   if (MODE == FA_SHARED) {
@@ -194,46 +221,74 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
   const int n_sh_tiles = (sh_end - sh_begin + BN - 1) / BN;
   const int n_tiles = n_sh_tiles + n_pr_tiles;
 
-  // ---- loaders: TPR threads per K/V row (a thread pair per Q row), interleaved 16-byte chunks
-  constexpr int TPR = THREADS / BN;
-  const int lrow = tid / TPR, lpar = tid % TPR;
-  int ld_cur = 0, ldv_cur = 0, mm_cur = 0;     // SHARED: sequence cursors of the K loader, the V loader, the math
-  auto load_tile = [&](int it, int buf, bool want_v) {   // K (cursor ld_cur) or V (cursor ldv_cur) rows of tile `it`
-    int tbl, key0, limit;
+  // ---- tile bookkeeping shared by the producer and the consumers: segment, first key, key limit
+  auto tile_info = [&](int it, int& cur, int& tbl, int& key0, int& limit) {
     if (it < n_sh_tiles) { tbl = sd.shared_tbl; key0 = sh_begin + it * BN; limit = sh_end; }
     else if (MODE == FA_ROWS) { tbl = sd.priv_tbl; key0 = (it - n_sh_tiles) * BN; limit = pr_end; }
     else {
       const int pt = split + (it - n_sh_tiles) * a.n_splits;           // suffix tile number within the row tile
-      int& cur = want_v ? ldv_cur : ld_cur;
       while (s_pt_sum[cur + 1] <= pt) ++cur;                            // its sequence (tiles are met in order)
       tbl = s_pt_tbl[cur]; key0 = (pt - s_pt_sum[cur]) * BN; limit = s_pt_t[cur] + 1;
     }
-    const int u = key0 + lrow;
-    const bf16* kp = nullptr;
-    if (u < limit) {
-      const int cached = (MODE == FA_SHARED && it < n_sh_tiles) ? (u - sh_begin) / KV_BLOCK : BLK_CACHE;
-      const int blk = (cached < BLK_CACHE) ? s_blk[cached] : a.block_table[tbl + u / KV_BLOCK];
-      if (blk >= 0 && blk < a.pool.n_blocks) {
-        kp = a.pool.at(a.layer, want_v ? 1 : 0, kvh, blk, u % KV_BLOCK);
-      } else {
-        atomicOr(a.status, STATUS_BAD_BLOCK);
-      }
-    }
-#pragma unroll
-    for (int j = 0; j < CH / TPR; ++j) {
-      const int ch = TPR * j + lpar;
-      const uint32_t off = sw(lrow, ch);
-      const uint32_t dst = (want_v ? sV : sK) + buf * TILE_BYTES + off;
-      if (kp) fa::cp_async16(dst, kp + ch * 8); else fa::st_zero16(dst);
-    }
   };
-  if (MODE == FA_ROWS) load_q(tid / QTPR, tid % QTPR, s_qrow[tid / QTPR], s_head[tid / QTPR]);
-  // prologue: K tiles 0..NSK-2 (the first group also carries Q), then V tiles 0..NSV-2.  Every
-  // step commits a group even when it loads nothing, so that the wait counts below stay constant.
-#pragma unroll
-  for (int st = 0; st < NSK - 1; ++st) { if (st < n_tiles) load_tile(st, st, false); fa::cp_commit(); }
-#pragma unroll
-  for (int st = 0; st < NSV - 1; ++st) { if (st < n_tiles) load_tile(st, st, true); fa::cp_commit(); }
+  volatile int* abort_flag = &s_abort;
+  if (MODE == FA_ROWS && tid < THREADS) load_q(tid / QTPR, tid % QTPR, s_qrow[tid / QTPR], s_head[tid / QTPR]);
+
+  if (warp == NW) {
+    // ------------------------------------------------------------------ producer warp
+    // Lane b looks up the KV block of the tile's b-th group of 16 keys; lane 0 then sends one box
+    // per block and half head.  Groups past the end of the segment re-send the last valid block
+    // (finite data, masked by the consumers), so a tile always carries TILE_BYTES.
+    int cur = 0;
+    auto blocks_of = [&](int it) -> int {       // lane b: block id of keys key0 + 16 b ..
+      int tbl, key0, limit;
+      tile_info(it, cur, tbl, key0, limit);
+      const int nb = max(1, min(BN / KV_BLOCK, (limit - key0 + KV_BLOCK - 1) / KV_BLOCK));
+      const int u = key0 + min(lane, nb - 1) * KV_BLOCK;
+      int blk = 0;
+      if (lane < BN / KV_BLOCK) {
+        const int cached = (MODE == FA_SHARED && it < n_sh_tiles) ? (u - sh_begin) / KV_BLOCK : BLK_CACHE;
+        blk = (cached < BLK_CACHE) ? s_blk[cached] : a.block_table[tbl + u / KV_BLOCK];
+        if (blk < 0 || blk >= a.pool.n_blocks) { atomicOr(a.status, STATUS_BAD_BLOCK); blk = 0; }
+      }
+      return blk;
+    };
+    auto send = [&](int blk_lane, int kv, uint32_t dst, uint64_t* bar) {   // lane b copies block b of the tile
+      if (lane < BN / KV_BLOCK)
+        tc::bulk_load(dst + lane * BLK_BYTES, a.pool.block(a.layer, kv, kvh, blk_lane), BLK_BYTES, bar);
+    };
+    // Order K0 | K1 V0 | K2 V1 | ...: a K tile is requested one tile ahead of the matching V tile.
+    bool ok = true;
+    int blk_next = (n_tiles > 0) ? blocks_of(0) : 0, blk_prev_v = 0;
+    for (int it = -1; it < n_tiles && ok; ++it) {
+      const int itk = it + 1;
+      int blk_k = blk_next;
+      if (itk < n_tiles) {
+        const int sk = itk % NSK;
+        if (lane == 0) {
+          ok = tc::mbar_wait(&empty_k[sk], ((itk / NSK) & 1) ^ 1, abort_flag);
+          if (ok) tc::mbar_expect_tx(&full_k[sk], TILE_BYTES);
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        send(blk_k, 0, sK + sk * TILE_BYTES, &full_k[sk]);
+        if (itk + 1 < n_tiles) blk_next = blocks_of(itk + 1);      // look the next tile's blocks up early
+      }
+      if (it >= 0) {
+        // the V tile of `it` uses the same blocks as its K tile: keep them from the previous round
+        const int sv = it % NSV;
+        if (lane == 0) {
+          ok = tc::mbar_wait(&empty_v[sv], ((it / NSV) & 1) ^ 1, abort_flag);
+          if (ok) tc::mbar_expect_tx(&full_v[sv], TILE_BYTES);
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        send(blk_prev_v, 1, sV + sv * TILE_BYTES, &full_v[sv]);
+      }
+      blk_prev_v = blk_k;
+    }
+    return;                                     // the consumers use named barrier 1 from here on
+  }
 
   float o[ONT][4];
 #pragma unroll
@@ -243,15 +298,12 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
   const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
   int t_lo = s_t[r_lo], t_hi = s_t[r_hi];
 
-  for (int it = 0; it < n_tiles; ++it) {
-    // K tile it+NSK-1 goes into the buffer whose tile every warp finished multiplying before it
-    // passed the V barrier of iteration it-1.  Groups younger than K(it): NSK+NSV-2.
-    if (it + NSK - 1 < n_tiles) load_tile(it + NSK - 1, (it + NSK - 1) % NSK, false);
-    fa::cp_commit();
-    fa::cp_wait<NSK + NSV - 2>();
-    __syncthreads();                          // K(it) visible to all; every warp is done with P V of tile it-1
-    if (it + NSV - 1 < n_tiles) load_tile(it + NSV - 1, (it + NSV - 1) % NSV, true);
-    fa::cp_commit();
+  int mm_cur = 0;                              // SHARED: sequence cursor of the math
+  asm volatile("cp.async.wait_all;" ::: "memory");                              // this thread's Q chunks
+  asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory");                    // all of Q (consumers only)
+  bool ok = true;
+  for (int it = 0; it < n_tiles && ok; ++it) {
+    if (!tc::mbar_wait(&full_k[it % NSK], (it / NSK) & 1, abort_flag)) { ok = false; break; }
     if (Q_IN_REGS && it == 0) {
 #pragma unroll
       for (int kk = 0; kk < KSTEPS; ++kk)
@@ -286,7 +338,7 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
 #pragma unroll
       for (int jp = 0; jp < WBN / 16; ++jp) {
         uint32_t b0, b1, b2, b3;
-        fa::ldsm_x4(kb + sw(kh * WBN + jp * 16 + (lane & 7) + ((lane >> 4) << 3), kk * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
+        fa::ldsm_x4(kb + swkv(kh * WBN + jp * 16 + (lane & 7) + ((lane >> 4) << 3), kk * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
         fa::mma_bf16(s[2 * jp], qf[qi], b0, b1);
         fa::mma_bf16(s[2 * jp + 1], qf[qi], b2, b3);
       }
@@ -336,8 +388,9 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
       for (int i = 0; i < ONT; ++i) { o[i][0] *= c_lo; o[i][1] *= c_lo; o[i][2] *= c_hi; o[i][3] *= c_hi; }
     }
     }
-    fa::cp_wait<2 * (NSV - 1)>();             // groups younger than V(it): 2 per iteration of look-ahead
-    __syncthreads();                          // V(it) visible to all; every warp is done with Q K^T of tile it
+    __syncwarp();
+    if (lane == 0) tc::mbar_arrive(&empty_k[it % NSK]);        // this warp is done with K(it)
+    if (!tc::mbar_wait(&full_v[it % NSV], (it / NSV) & 1, abort_flag)) { ok = false; break; }
     if (warp_has_work) {
     // ---- O += P V
     const uint32_t vb = sV + (it % NSV) * TILE_BYTES;
@@ -346,20 +399,22 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
 #pragma unroll
       for (int np = 0; np < ONT / 2; ++np) {
         uint32_t b0, b1, b2, b3;
-        fa::ldsm_x4_t(vb + sw(kh * WBN + kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), np * 2 + (lane >> 4)), b0, b1, b2, b3);
+        fa::ldsm_x4_t(vb + swkv(kh * WBN + kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), np * 2 + (lane >> 4)), b0, b1, b2, b3);
         fa::mma_bf16(o[2 * np], pf[kk], b0, b1);
         fa::mma_bf16(o[2 * np + 1], pf[kk], b2, b3);
       }
     }
     }
+    __syncwarp();
+    if (lane == 0) tc::mbar_arrive(&empty_v[it % NSV]);        // ... and with V(it)
   }
-  fa::cp_wait<0>();
+  if (!ok && lane == 0) atomicOr(a.status, STATUS_TIMEOUT);
   if (KS == 2) {
-    __syncthreads();                          // every warp is done with the ring
+    asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory");   // every consumer warp is done with the rings
     // The warps of the second key half hand their state to the warp holding the same rows in the
     // first half, thread to thread ([value][thread] layout: no bank conflicts), through the K/V ring
     // (free after the loop's last barrier).  m is uniform over a quad, l is still a per-lane partial.
-    float* xch = reinterpret_cast<float*>(fsm + FA_BM * ROW_BYTES);
+    float* xch = reinterpret_cast<float*>(fsm);
     const int xt = mt * 32 + lane;
     if (kh == 1) {
 #pragma unroll
@@ -370,7 +425,7 @@ __global__ void __launch_bounds__(FaCfg<MODE>::THREADS, FaCfg<MODE>::MIN_CTAS) f
       xch[(ONT * 4 + 0) * FA_THREADS + xt] = m_lo; xch[(ONT * 4 + 1) * FA_THREADS + xt] = m_hi;
       xch[(ONT * 4 + 2) * FA_THREADS + xt] = l_lo; xch[(ONT * 4 + 3) * FA_THREADS + xt] = l_hi;
     }
-    __syncthreads();
+    asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory");
     if (kh == 1) return;
     const float mb_lo = xch[(ONT * 4 + 0) * FA_THREADS + xt], mb_hi = xch[(ONT * 4 + 1) * FA_THREADS + xt];
     const float mn_lo = fmaxf(m_lo, mb_lo), mn_hi = fmaxf(m_hi, mb_hi);

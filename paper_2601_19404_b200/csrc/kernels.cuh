@@ -15,14 +15,28 @@ struct SeqDesc {
   int32_t reserved;
 };
 
+// One KV block = 16 tokens of one (layer, K|V, kv head).  For 16-bit storage its head_dim*32 bytes
+// are laid out the way the attention kernels want them in shared memory, so that a block is moved
+// with ONE contiguous bulk copy and read with conflict-free ldmatrix:
+//     [half head h = dim / 64][token 0..15][8 chunks of 16 bytes, chunk c stored at c ^ (token & 7)]
+// (for head_dim 64 there is one half).  float32 storage (plain CUDA-core attention only) keeps
+// [token][dim].  chunk() returns the address of the 8-element chunk that holds `dim` (dim % 8 == 0).
 template <typename T>
 struct KVPool {
   T* base;
   int64_t layer_stride, kv_stride, head_stride;  // elements
   int32_t n_blocks, head_dim;
-  __device__ __forceinline__ T* at(int layer, int kv, int head, int block, int off) const {
-    return base + layer * layer_stride + kv * kv_stride + head * head_stride +
-           ((int64_t)block * KV_BLOCK + off) * head_dim;
+  __device__ __forceinline__ T* block(int layer, int kv, int head, int block) const {
+    return base + layer * layer_stride + kv * kv_stride + head * head_stride + (int64_t)block * KV_BLOCK * head_dim;
+  }
+  __device__ __forceinline__ T* chunk(int layer, int kv, int head, int blk, int token, int dim) const {
+    T* b = block(layer, kv, head, blk);
+    if (sizeof(T) == 2) {
+      const int per_half = head_dim < 64 ? head_dim : 64;
+      const int h = dim / per_half, c = (dim % per_half) >> 3;
+      return b + h * (KV_BLOCK * per_half) + token * per_half + ((c ^ (token & 7)) << 3);
+    }
+    return b + token * head_dim + dim;
   }
 };
 
@@ -233,12 +247,13 @@ __global__ void rope_kv_kernel(T* __restrict__ qkv, const int32_t* __restrict__ 
   const SeqDesc sd = seqs[row_seq[r]];
   const int pos = sd.shared_len + t;
   if (pos >= max_pos) { if (i0 == 0) atomicOr(status, STATUS_BAD_BLOCK); return; }
-  T* dst = src;                                         // q: rotated in place
+  T *dst_lo = src + i0, *dst_hi = src + half + i0;      // q: rotated in place
   if (head >= hq) {
     const int kv = (head - hq) / hkv, kh = (head - hq) % hkv;
     const int blk = block_table[sd.priv_tbl + t / KV_BLOCK];
     if (blk < 0 || blk >= pool.n_blocks) { if (i0 == 0) atomicOr(status, STATUS_BAD_BLOCK); return; }
-    dst = pool.at(layer, kv, kh, blk, t % KV_BLOCK);
+    dst_lo = pool.chunk(layer, kv, kh, blk, t % KV_BLOCK, i0);
+    dst_hi = pool.chunk(layer, kv, kh, blk, t % KV_BLOCK, half + i0);
   }
   __align__(16) T ol[8], oh[8];
   if (head < hq + hkv) {                                // q or k: rotate
@@ -253,10 +268,10 @@ __global__ void rope_kv_kernel(T* __restrict__ qkv, const int32_t* __restrict__ 
 #pragma unroll
     for (int j = 0; j < 8; ++j) { ol[j] = from_f32<T>(lo[j]); oh[j] = from_f32<T>(hi[j]); }
   }
-  *reinterpret_cast<uint4*>(dst + i0) = *reinterpret_cast<const uint4*>(ol);
-  if (sizeof(T) == 4) *reinterpret_cast<uint4*>(dst + i0 + 4) = *reinterpret_cast<const uint4*>(ol + 4);
-  *reinterpret_cast<uint4*>(dst + half + i0) = *reinterpret_cast<const uint4*>(oh);
-  if (sizeof(T) == 4) *reinterpret_cast<uint4*>(dst + half + i0 + 4) = *reinterpret_cast<const uint4*>(oh + 4);
+  *reinterpret_cast<uint4*>(dst_lo) = *reinterpret_cast<const uint4*>(ol);
+  if (sizeof(T) == 4) *reinterpret_cast<uint4*>(dst_lo + 4) = *reinterpret_cast<const uint4*>(ol + 4);
+  *reinterpret_cast<uint4*>(dst_hi) = *reinterpret_cast<const uint4*>(oh);
+  if (sizeof(T) == 4) *reinterpret_cast<uint4*>(dst_hi + 4) = *reinterpret_cast<const uint4*>(oh + 4);
 }
 
 // act[r, j] = silu(gu[r, 2j]) * gu[r, 2j+1]   (gate/up interleaved by the fused weight layout)

@@ -95,8 +95,9 @@ __global__ void __launch_bounds__(128) attn_ref_kernel(const T* __restrict__ qkv
     if (u < n_shared) { tbl = sd.shared_tbl; idx = u; } else { tbl = sd.priv_tbl; idx = u - n_shared; }
     const int blk = block_table[tbl + idx / KV_BLOCK];
     if (blk < 0 || blk >= pool.n_blocks) { if (lane == 0) atomicOr(status, STATUS_BAD_BLOCK); continue; }
-    const T* kp = pool.at(layer, 0, kvh, blk, idx % KV_BLOCK) + lane * DPL;
-    const T* vp = pool.at(layer, 1, kvh, blk, idx % KV_BLOCK) + lane * DPL;
+    const int dim0 = lane * DPL;                  // DPL divides 8: the lane's dims sit inside one chunk
+    const T* kp = pool.chunk(layer, 0, kvh, blk, idx % KV_BLOCK, dim0 & ~7) + (dim0 & 7);
+    const T* vp = pool.chunk(layer, 1, kvh, blk, idx % KV_BLOCK, dim0 & ~7) + (dim0 & 7);
     float s = 0.f;
 #pragma unroll
     for (int i = 0; i < DPL; ++i) s = fmaf(q[i], to_f32(kp[i]), s);

@@ -274,6 +274,12 @@ extern "C" int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limit
   w.partial_elems = (size_t)c->sm_count * 128 * 256;
   ALLOC(w.partial, w.partial_elems * 4);
   if (rc == RPO_OK) rc = tc_create(c);
+  // The attention kernels mask keys beyond a segment's end instead of zero-filling them, so the
+  // pool must never hold NaN/Inf bit patterns: start from zeros.
+  if (rc == RPO_OK && cudaMemsetAsync(c->kv_base, 0, (size_t)std::max(1, s.n_layers) * c->kv_layer_stride * e, c->stream) != cudaSuccess) {
+    cudaGetLastError();
+    rc = RPO_ERR_CUDA;
+  }
 #undef ALLOC
   if (rc != RPO_OK) { rpo_destroy(c); return rc; }
   cudaMemsetAsync(c->d_status, 0, 16, c->stream);
@@ -418,7 +424,7 @@ static int launch_flash(rpo_ctx* c, const FlashArgs& a, dim3 grid) {
     CUDA_TRY(cudaFuncSetAttribute(flash_attn_kernel<DH, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     attr_done = true;
   }
-  LAUNCH(c, (flash_attn_kernel<DH, MODE>), grid, FaCfg<MODE>::THREADS, smem, a);
+  LAUNCH(c, (flash_attn_kernel<DH, MODE>), grid, FaCfg<MODE>::THREADS + 32, smem, a);
   return RPO_OK;
 }
 
