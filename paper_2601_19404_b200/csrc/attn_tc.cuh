@@ -111,7 +111,7 @@ flash_attn_kernel(FlashArgs a) {
   __shared__ int s_qrow[FA_BM];     // qkv row of each tile row (-1: padding)
   __shared__ int s_head[FA_BM];
   __shared__ int s_t[FA_BM];        // private causal limit (-1: nothing visible / inactive)
-  __shared__ int s_pt_sum[FA_BM + 1];   // SHARED: suffix tiles of the tile's sequences, prefix-summed
+  __shared__ int s_pt_sum[FA_BM + 1];   // SHARED: suffix tiles of the tile's sequences that fall to this split, prefix-summed
   __shared__ int s_pt_t[FA_BM];         //         their newest suffix index t (-1: finished)
   __shared__ int s_pt_tbl[FA_BM];       //         their private block-table offsets
   constexpr int BLK_CACHE = (MODE == FA_SHARED) ? 512 : 1;
@@ -187,7 +187,11 @@ flash_attn_kernel(FlashArgs a) {
       const int t = a.row_t[seq];
       s_pt_t[tid] = t;
       s_pt_tbl[tid] = a.seqs[seq].priv_tbl;               // decode passes: row i is sequence i
-      s_pt_sum[tid + 1] = (t >= 0) ? t / BN + 1 : 0;       // suffix tiles of this sequence (prefix-summed below)
+      // Suffix tile j of the group's sequence i belongs to split (i + j) % n_splits: a sequence's
+      // arithmetic does not depend on how far its siblings have got.  Tiles of this split: j0, j0 + n_splits, ..
+      const int nt = (t >= 0) ? t / BN + 1 : 0;
+      const int j0 = ((split - (sq0 + tid)) % a.n_splits + a.n_splits) % a.n_splits;
+      s_pt_sum[tid + 1] = (nt > j0) ? (nt - j0 - 1) / a.n_splits + 1 : 0;      // prefix-summed below
     }
     // block ids of this split's prefix keys: one fetch up front instead of one per tile
     sh_begin = min(sd.shared_len, split * a.split_chunk);  // a multiple of 16
@@ -214,9 +218,7 @@ flash_attn_kernel(FlashArgs a) {
     pr_end = mt + 1;
     n_pr_tiles = (pr_end + BN - 1) / BN;
   } else {
-    // suffix tile p of the tile's sequences (in sequence order) is handled by split p % n_splits
-    const int total_p = s_pt_sum[n_sq];
-    n_pr_tiles = (total_p > split) ? (total_p - split - 1) / a.n_splits + 1 : 0;
+    n_pr_tiles = s_pt_sum[n_sq];
   }
   const int n_sh_tiles = (sh_end - sh_begin + BN - 1) / BN;
   const int n_tiles = n_sh_tiles + n_pr_tiles;
@@ -226,9 +228,10 @@ flash_attn_kernel(FlashArgs a) {
     if (it < n_sh_tiles) { tbl = sd.shared_tbl; key0 = sh_begin + it * BN; limit = sh_end; }
     else if (MODE == FA_ROWS) { tbl = sd.priv_tbl; key0 = (it - n_sh_tiles) * BN; limit = pr_end; }
     else {
-      const int pt = split + (it - n_sh_tiles) * a.n_splits;           // suffix tile number within the row tile
-      while (s_pt_sum[cur + 1] <= pt) ++cur;                            // its sequence (tiles are met in order)
-      tbl = s_pt_tbl[cur]; key0 = (pt - s_pt_sum[cur]) * BN; limit = s_pt_t[cur] + 1;
+      const int q = it - n_sh_tiles;                                    // q-th suffix tile of this work item
+      while (s_pt_sum[cur + 1] <= q) ++cur;                             // its sequence (tiles are met in order)
+      const int j0 = ((split - (sq0 + cur)) % a.n_splits + a.n_splits) % a.n_splits;
+      tbl = s_pt_tbl[cur]; key0 = (j0 + (q - s_pt_sum[cur]) * a.n_splits) * BN; limit = s_pt_t[cur] + 1;
     }
   };
   volatile int* abort_flag = &s_abort;
@@ -313,11 +316,12 @@ flash_attn_kernel(FlashArgs a) {
     int suffix_key0 = 0;
     if (MODE == FA_SHARED && it >= n_sh_tiles) {
       // suffix tile of one sequence: visible to that sequence's rows only, keys 0..t
-      const int pt = split + (it - n_sh_tiles) * a.n_splits;
-      while (s_pt_sum[mm_cur + 1] <= pt) ++mm_cur;
+      const int q = it - n_sh_tiles;
+      while (s_pt_sum[mm_cur + 1] <= q) ++mm_cur;
+      const int j0 = ((split - (sq0 + mm_cur)) % a.n_splits + a.n_splits) % a.n_splits;
       const int row_first = (sq0 + mm_cur) * rep - r0, row_last = row_first + rep - 1;   // tile-local, may stick out
       const int t_own = s_pt_t[mm_cur];
-      suffix_key0 = (pt - s_pt_sum[mm_cur]) * BN;
+      suffix_key0 = (j0 + (q - s_pt_sum[mm_cur]) * a.n_splits) * BN;
       t_lo = (r_lo >= row_first && r_lo <= row_last) ? t_own : -1;
       t_hi = (r_hi >= row_first && r_hi <= row_last) ? t_own : -1;
       warp_has_work = warp_has_work && (mt * 16 <= row_last) && (mt * 16 + 15 >= row_first) &&

