@@ -36,6 +36,21 @@ def measured_peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_sustained=1400.0, source="fallback")
 
 
+def ncu_traffic_per_launch():
+    """DRAM bytes per launch of the decode GEMM from the committed ncu capture, or None once the
+    kernel source has changed since the counters were taken."""
+    import hashlib
+    prof = os.path.join(ROOT, "profiles", "decode_step_kernels_cfg2_reduced.txt")
+    src = os.path.join(ROOT, "paper_2601_19404_b200", "csrc", "gemm_tc.cuh")
+    try:
+        vals = dict(l.split(" = ") for l in open(prof).read().splitlines() if " = " in l)
+        if vals["gemm_tc_cuh_sha256"].strip() != hashlib.sha256(open(src, "rb").read()).hexdigest():
+            return None
+        return float(vals["gemm_decode_traffic_bytes_per_launch"])
+    except Exception:
+        return None
+
+
 class ClockSampler:
     """nvidia-smi clocks / throttle reasons sampled every 200 ms while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -164,8 +179,8 @@ def main():
     ap.add_argument("--config", default="cfg2_1p5b_16x8")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-profile", action="store_true")
-    ap.add_argument("--ref-prefix", type=int, default=128)
-    ap.add_argument("--ref-suffix", type=int, default=4)
+    ap.add_argument("--ref-prefix", type=int, default=1024)
+    ap.add_argument("--ref-suffix", type=int, default=8)
     ap.add_argument("--options", default="", help="comma list name=value passed to rpo_set_option")
     ap.add_argument("--layers", type=int, default=0, help="override n_layers (reduced case for profiler captures)")
     ap.add_argument("--suffix", type=int, default=0, help="override the suffix length (reduced case for profiler captures)")
@@ -322,14 +337,19 @@ def main():
         ctx.set_option("profile", 0)
         phases = {p: {k: {"ms": round(v[0], 3), "launches": v[1]} for k, v in d.items() if v[1]} for p, d in prof.items()}
         gemm_ms, gemm_n = prof["decode"]["gemm"]
-        # dominant decode kernel: the weight-streaming GEMM. algorithmic bytes per launch = all weight
-        # bytes a decode step reads / GEMM launches per decode step
+        # Dominant kernel of the path: the weight-streaming tensor-core GEMM of the decode step (all
+        # layer matrices + lm_head once per step).  Algorithmic bytes per launch = weight bytes a step
+        # reads / GEMM launches per step; duration = mean of CUDA-event pairs bracketing every launch
+        # of the profiled step (bracketing adds a few microseconds per launch: the fraction is a floor).
         if gemm_n:
             per_launch_bytes = ab["weights"] * (S - 1) / gemm_n
             achieved = per_launch_bytes / (gemm_ms / gemm_n * 1e-3) / 1e9
-            roofline = {"bound": "hbm", "kernel": "decode weight GEMM", "achieved": achieved, "peak": peaks["hbm_gbs"],
-                        "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
-                        "peak_source": peaks["source"], "ms_per_launch": gemm_ms / gemm_n}
+            roofline = {"bound": "hbm", "kernel": "gemm_tc_kernel (decode weight GEMMs)", "achieved": achieved,
+                        "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                        "traffic": ncu_traffic_per_launch() if not reduced else None,
+                        "algorithmic_bytes_per_launch": per_launch_bytes, "launches_per_step": gemm_n / max(S - 1, 1),
+                        "peak_source": peaks["source"] + " copy bandwidth (MEASURED_PEAKS.json)" if peaks["source"] == "measured" else "fallback",
+                        "ms_per_launch": gemm_ms / gemm_n}
     decode_gbs = ab["total"] / (dec_step_ms * 1e-3) / 1e9
     pf = prefill_flops(shape, lens)
     prefill_tfs = pf / (pre_ms * 1e-3) / 1e12
