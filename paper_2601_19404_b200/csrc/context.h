@@ -87,6 +87,7 @@ struct rpo_ctx {
   int sm_count = 148;
   // options
   int use_tcgen05 = 1, use_tc_attention = 1, use_graph = 1;
+  int use_tc5_attention = 1, tc5_v_variant = 0;   // tcgen05 prefill attention (and the descriptor reading under test)
   int use_pdl = 1;                    // programmatic dependent launch between the library's kernels
   int gemm_bn = 0, gemm_splits = 0;   // > 0: override the GEMM planner (tests, sweeps)
   // attention plan of the pass being enqueued: 0 = row tiles (prefill / teacher), 1 = decode

@@ -12,6 +12,7 @@
 #include <utility>
 
 #include "attn_tc.cuh"
+#include "attn_tc5.cuh"
 #include "context.h"
 #include "gemm_tc.cuh"
 #include "kernels.cuh"
@@ -428,6 +429,11 @@ static int launch_flash(rpo_ctx* c, const FlashArgs& a, dim3 grid) {
   return RPO_OK;
 }
 
+// The tcgen05 attention serves prefill / teacher-forced passes of bf16 models with head_dim 128.
+static bool tc5_attention(rpo_ctx* c) {
+  return c->bf16 && c->use_tc_attention && c->use_tc5_attention && c->shape.head_dim == T5_DH;
+}
+
 template <typename T>
 static int attention(rpo_ctx* c, int layer, int rows) {
   const rpo_shape& s = c->shape;
@@ -444,6 +450,24 @@ static int attention(rpo_ctx* c, int layer, int rows) {
       a.pool = kv_pool<bf16>(c); a.layer = layer; a.hq = s.n_q_heads; a.hkv = s.n_kv_heads;
       a.scale_log2 = scale * 1.4426950408889634f; a.tiles = (const int2*)w.tiles; a.G = c->attn_G; a.status = c->d_status;
       a.n_splits = c->attn_splits; a.split_chunk = c->attn_split_chunk;
+      if (c->attn_mode == 0 && tc5_attention(c)) {
+        // tcgen05 path: 128-row tiles, Q through a tensor map over the fused qkv buffer
+        const CUtensorMap* qm = tc_map(c, w.qkv, w.R, c->qkv_cols, T5_BM);
+        if (!qm) return RPO_ERR_CUDA;
+        Flash5Args f;
+        memset(&f, 0, sizeof(f));
+        f.out = (bf16*)w.attn; f.out_cols = s.n_q_heads * s.head_dim; f.row_seq = w.row_seq; f.row_t = w.row_t;
+        f.seqs = (const SeqDesc*)w.seqs; f.block_table = c->d_block_table; f.pool = kv_pool<bf16>(c); f.layer = layer;
+        f.hq = s.n_q_heads; f.hkv = s.n_kv_heads; f.scale_log2 = scale * 1.4426950408889634f; f.tiles = (const int2*)w.tiles;
+        f.q_col0 = 0; f.v_desc_variant = c->tc5_v_variant; f.status = c->d_status;
+        static bool attr_done = false;
+        if (!attr_done) {
+          CUDA_TRY(cudaFuncSetAttribute(flash_attn_tc5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, T5_SMEM));
+          attr_done = true;
+        }
+        LAUNCH(c, flash_attn_tc5_kernel, dim3(c->attn_tiles, s.n_q_heads), 192, T5_SMEM, *qm, f);
+        return RPO_OK;
+      }
       if (c->attn_mode == 0) {
         dim3 grid(c->attn_tiles, s.n_q_heads);
         return s.head_dim == 128 ? launch_flash<128, FA_ROWS>(c, a, grid) : launch_flash<64, FA_ROWS>(c, a, grid);
@@ -471,12 +495,14 @@ static int attention(rpo_ctx* c, int layer, int rows) {
   return RPO_OK;
 }
 
-// 64-row query tiles of a pass whose sequences own consecutive row ranges.
+// Query-row tiles (128 rows for the tcgen05 attention, else 64) of a pass whose sequences own
+// consecutive row ranges.
 static int upload_row_tiles(rpo_ctx* c, const std::vector<int>& rows_per_seq) {
   std::vector<int2> tiles;
+  const int bm = tc5_attention(c) ? T5_BM : FA_BM;
   int r = 0;
   for (int n : rows_per_seq) {
-    for (int r0 = 0; r0 < n; r0 += FA_BM) tiles.push_back(make_int2(r + r0, std::min(FA_BM, n - r0)));
+    for (int r0 = 0; r0 < n; r0 += bm) tiles.push_back(make_int2(r + r0, std::min(bm, n - r0)));
     r += n;
   }
   c->attn_mode = 0; c->attn_tiles = (int)tiles.size();
@@ -1004,6 +1030,8 @@ extern "C" int rpo_set_option(rpo_ctx* c, const char* name, int32_t value) {
   else if (!strcmp(name, "use_tc_attention")) c->use_tc_attention = value;
   else if (!strcmp(name, "use_graph")) c->use_graph = value;
   else if (!strcmp(name, "use_pdl")) c->use_pdl = value;
+  else if (!strcmp(name, "use_tc5_attention")) c->use_tc5_attention = value;
+  else if (!strcmp(name, "tc5_v_variant")) c->tc5_v_variant = value;
   else if (!strcmp(name, "gemm_bn")) { if (value != 0 && value != 32 && value != 64 && value != 96 && value != 128 && value != 256) return RPO_ERR_INVALID_ARG; c->gemm_bn = value; }
   else if (!strcmp(name, "gemm_splits")) c->gemm_splits = value;
   else if (!strcmp(name, "profile")) c->profile = value;
