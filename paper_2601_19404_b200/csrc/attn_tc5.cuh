@@ -196,15 +196,23 @@ flash_attn_tc5_kernel(const __grid_constant__ CUtensorMap q_map, Flash5Args a) {
       const int lim = shared_tile ? sh_end - 1 : t_row;                       // last visible key of this row in the segment
       if (!tc::mbar_wait(&s_full[sb], (it >> 1) & 1, abort_flag)) { ok = false; break; }
       tc::tmem_fence_after();
-      // pass 1: row maximum
+      // pass 1: row maximum (on the raw scores: the scale is positive).  Tiles whose keys this row
+      // sees in full skip the per-key visibility test.
+      const bool whole = key0 + T5_BN - 1 <= lim;
       float mx = -INFINITY;
 #pragma unroll 1
       for (int c0 = 0; c0 < T5_BN; c0 += 32) {
         uint32_t v[32];
         tc::tmem_ld32(t_lane + sb * T5_BN + c0, v);
+        if (whole) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) if (key0 + c0 + j <= lim) mx = fmaxf(mx, __uint_as_float(v[j]) * a.scale_log2);
+          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(v[j]));
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) if (key0 + c0 + j <= lim) mx = fmaxf(mx, __uint_as_float(v[j]));
+        }
       }
+      mx *= a.scale_log2;
       const float m_new = fmaxf(m, mx), mu = (m_new == -INFINITY) ? 0.f : m_new;
       const float c_prev = corr;                                              // factor that goes with O_tile(it-1)
       corr = fa::ex2(m - mu);
@@ -230,12 +238,22 @@ flash_attn_tc5_kernel(const __grid_constant__ CUtensorMap q_map, Flash5Args a) {
         uint32_t v[32];
         tc::tmem_ld32(t_lane + sb * T5_BN + c0, v);
         uint32_t pk[16];
+        if (whole) {
 #pragma unroll
-        for (int j = 0; j < 32; j += 2) {
-          const float p0 = (key0 + c0 + j <= lim) ? fa::ex2(__uint_as_float(v[j]) * a.scale_log2 - mu) : 0.f;
-          const float p1 = (key0 + c0 + j + 1 <= lim) ? fa::ex2(__uint_as_float(v[j + 1]) * a.scale_log2 - mu) : 0.f;
-          ps += p0 + p1;
-          pk[j >> 1] = fa::pack_bf16(p0, p1);
+          for (int j = 0; j < 32; j += 2) {
+            const float p0 = fa::ex2(fmaf(__uint_as_float(v[j]), a.scale_log2, -mu));
+            const float p1 = fa::ex2(fmaf(__uint_as_float(v[j + 1]), a.scale_log2, -mu));
+            ps += p0 + p1;
+            pk[j >> 1] = fa::pack_bf16(p0, p1);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            const float p0 = (key0 + c0 + j <= lim) ? fa::ex2(fmaf(__uint_as_float(v[j]), a.scale_log2, -mu)) : 0.f;
+            const float p1 = (key0 + c0 + j + 1 <= lim) ? fa::ex2(fmaf(__uint_as_float(v[j + 1]), a.scale_log2, -mu)) : 0.f;
+            ps += p0 + p1;
+            pk[j >> 1] = fa::pack_bf16(p0, p1);
+          }
         }
         const uint32_t base = sP + (c0 >> 6) * (T5_TILE / 2) + r * 128;
 #pragma unroll
