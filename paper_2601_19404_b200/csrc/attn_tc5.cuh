@@ -6,14 +6,15 @@
 //   S = Q K^T      tcgen05.mma, A = Q tile (TMA, 128-byte swizzle, K-major), B = K tile (KV blocks bulk-
 //                  copied from the pool, whose block layout IS the 128-byte-swizzled K-major layout),
 //                  accumulator in tensor memory, two buffers
-//   softmax        four warps, thread = query row = TMEM lane: tcgen05.ld the row, online max / sum
-//                  in the exp2 domain without any shuffle, P written to shared memory as bf16 in the
-//                  swizzled K-major layout
+//   softmax        eight warps, two threads per query row (= TMEM lane), 64 columns each: tcgen05.ld,
+//                  online max / sum in the exp2 domain without any shuffle, P written to shared
+//                  memory as bf16 in the swizzled K-major layout
 //   O_tile = P V   tcgen05.mma, A = P (shared memory), B = V blocks as stored ([token][dim] rows of
 //                  128 bytes = an MN-major operand), one MMA per 16-token block; accumulator in TMEM
 //   O += O_tile    the row's running output lives in registers: O = O * 2^(m_old - m_new) + O_tile
 //
-// Warp roles: 0 = producer (bulk copies K/V, TMA Q), 1 = MMA issuer and TMEM owner, 2..5 = softmax.
+// Warp roles: 0 = producer (bulk copies K/V, TMA Q), 1 = MMA issuer and TMEM owner, 2..9 = softmax
+// (two warps per TMEM lane quadrant, each on half of the columns).
 // All mbarrier waits are bounded; on expiry the CTA raises STATUS_TIMEOUT and leaves.
 #pragma once
 #include "attn_tc.cuh"
@@ -23,7 +24,7 @@ namespace rpo {
 constexpr int T5_BM = 128, T5_BN = 128, T5_DH = 128;
 constexpr int T5_NSK = 2, T5_NSV = 2;
 constexpr int T5_TILE = T5_BN * T5_DH * 2;                       // 32 KB: one K or V tile, also Q and P
-constexpr int T5_SMEM = (2 + T5_NSK + T5_NSV) * T5_TILE + 1024 + 256;
+constexpr int T5_SMEM = (2 + T5_NSK + T5_NSV) * T5_TILE + 1024 + 256 + 3072;   // tiles, alignment, barriers, row-maximum exchange
 
 struct Flash5Args {
   const bf16* qkv_unused;
@@ -54,7 +55,7 @@ __device__ __forceinline__ uint64_t desc_mn_sw128(uint32_t addr, uint32_t mn_str
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 }  // namespace t5
 
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(320, 1)
 flash_attn_tc5_kernel(const __grid_constant__ CUtensorMap q_map, Flash5Args a) {
   pdl_prologue();
   extern __shared__ uint8_t t5_raw[];
@@ -80,9 +81,10 @@ flash_attn_tc5_kernel(const __grid_constant__ CUtensorMap q_map, Flash5Args a) {
     for (int i = 0; i < 2; ++i) {
       tc::mbar_init(&full_k[i], 1); tc::mbar_init(&empty_k[i], 1);
       tc::mbar_init(&full_v[i], 1); tc::mbar_init(&empty_v[i], 1);
-      tc::mbar_init(&s_full[i], 1); tc::mbar_init(&s_free[i], 4);
+      tc::mbar_init(&s_full[i], 1); tc::mbar_init(&s_free[i], 8);
     }
-    tc::mbar_init(p_full, 4); tc::mbar_init(o_full, 1); tc::mbar_init(o_free, 4); tc::mbar_init(q_full, 1);
+    tc::mbar_init(p_full, 8); tc::mbar_init(o_full, 1); tc::mbar_init(o_free, 8); tc::mbar_init(q_full, 1);
+    for (int i = 0; i < 4; ++i) tc::mbar_init(&bars[17 + i], 2);      // one per lane quadrant: its two softmax warps
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -179,40 +181,48 @@ flash_attn_tc5_kernel(const __grid_constant__ CUtensorMap q_map, Flash5Args a) {
       }
     }
   } else {
-    // ------------------------------------------------------------------ softmax warps: thread = query row
-    const int quad = warp & 3, r = quad * 32 + lane;
+    // ------------------------------------------------------------------ softmax warps
+    // Eight warps: warps w and w+4 serve the same TMEM lane quadrant (32 query rows) and split the
+    // columns: thread (row r, half hf) owns keys / output dims [64 hf, 64 hf + 64).  The two threads
+    // of a row agree on the running maximum through shared memory once per tile.
+    const int sw = warp - 2, quad = warp & 3, hf = sw >> 2, r = quad * 32 + lane;
     const bool row_valid = r < n_rows;
     const int t_row = row_valid ? a.row_t[row0 + r] : -1;
-    const uint32_t t_lane = tmem + ((uint32_t)(quad * 32) << 16);
-    float o[T5_DH];
+    const uint32_t t_lane = tmem + ((uint32_t)(quad * 32) << 16) + hf * 64;
+    float* xmax = reinterpret_cast<float*>(bars + 24);                 // [2 slots][2 halves][128 rows], then [2 halves][128] sums
+    uint64_t* pair_bar = &bars[17 + quad];                             // bounded rendezvous of the row's two threads
+    float o[64];
 #pragma unroll
-    for (int i = 0; i < T5_DH; ++i) o[i] = 0.f;
+    for (int i = 0; i < 64; ++i) o[i] = 0.f;
     float m = -INFINITY, l = 0.f, corr = 0.f;
     bool ok = true;
     for (int it = 0; it < n_tiles && ok; ++it) {
       const int sb = it & 1;
       const bool shared_tile = it < n_sh;
-      const int key0 = shared_tile ? it * T5_BN : (it - n_sh) * T5_BN;
+      const int key0 = (shared_tile ? it * T5_BN : (it - n_sh) * T5_BN) + hf * 64;   // first key of my half
       const int lim = shared_tile ? sh_end - 1 : t_row;                       // last visible key of this row in the segment
       if (!tc::mbar_wait(&s_full[sb], (it >> 1) & 1, abort_flag)) { ok = false; break; }
       tc::tmem_fence_after();
-      // pass 1: row maximum (on the raw scores: the scale is positive).  Tiles whose keys this row
-      // sees in full skip the per-key visibility test.
-      const bool whole = key0 + T5_BN - 1 <= lim;
+      // my 64 scores, kept in registers for both passes
+      uint32_t v[64];
+      tc::tmem_ld32_nowait(t_lane + sb * T5_BN, v);
+      tc::tmem_ld32_nowait(t_lane + sb * T5_BN + 32, v + 32);
+      tc::tmem_ld_wait();
+      const bool whole = key0 + 63 <= lim;
       float mx = -INFINITY;
-#pragma unroll 1
-      for (int c0 = 0; c0 < T5_BN; c0 += 32) {
-        uint32_t v[32];
-        tc::tmem_ld32(t_lane + sb * T5_BN + c0, v);
-        if (whole) {
+      if (whole) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(v[j]));
-        } else {
+        for (int j = 0; j < 64; ++j) mx = fmaxf(mx, __uint_as_float(v[j]));
+      } else {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) if (key0 + c0 + j <= lim) mx = fmaxf(mx, __uint_as_float(v[j]));
-        }
+        for (int j = 0; j < 64; ++j) if (key0 + j <= lim) mx = fmaxf(mx, __uint_as_float(v[j]));
       }
       mx *= a.scale_log2;
+      xmax[(sb * 2 + hf) * 128 + r] = mx;
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(pair_bar);                               // release: my warp's maxima are written
+      if (!tc::mbar_wait(pair_bar, it & 1, abort_flag)) { ok = false; break; }
+      mx = fmaxf(mx, xmax[(sb * 2 + (hf ^ 1)) * 128 + r]);
       const float m_new = fmaxf(m, mx), mu = (m_new == -INFINITY) ? 0.f : m_new;
       const float c_prev = corr;                                              // factor that goes with O_tile(it-1)
       corr = fa::ex2(m - mu);
@@ -220,48 +230,32 @@ flash_attn_tc5_kernel(const __grid_constant__ CUtensorMap q_map, Flash5Args a) {
       if (it > 0) {
         if (!tc::mbar_wait(o_full, (it - 1) & 1, abort_flag)) { ok = false; break; }
         tc::tmem_fence_after();
+        uint32_t w[64];
+        tc::tmem_ld32_nowait(t_lane + 2 * T5_BN, w);
+        tc::tmem_ld32_nowait(t_lane + 2 * T5_BN + 32, w + 32);
+        tc::tmem_ld_wait();
 #pragma unroll
-        for (int c0 = 0; c0 < T5_DH; c0 += 32) {          // fully unrolled: o[] must stay in registers
-          uint32_t v[32];
-          tc::tmem_ld32(t_lane + 2 * T5_BN + c0, v);
-#pragma unroll
-          for (int j = 0; j < 32; ++j) o[c0 + j] = o[c0 + j] * c_prev + __uint_as_float(v[j]);
-        }
+        for (int j = 0; j < 64; ++j) o[j] = o[j] * c_prev + __uint_as_float(w[j]);
         tc::tmem_fence_before();
         __syncwarp();
         if (lane == 0) tc::mbar_arrive(o_free);
       }
-      // pass 2: P = 2^(s - m) as bf16 into the swizzled K-major tile, row sum
+      // P = 2^(s - m) as bf16 into the swizzled K-major tile (plane hf), row sum of my half
       float ps = 0.f;
-#pragma unroll 1
-      for (int c0 = 0; c0 < T5_BN; c0 += 32) {
-        uint32_t v[32];
-        tc::tmem_ld32(t_lane + sb * T5_BN + c0, v);
-        uint32_t pk[16];
-        if (whole) {
+      const uint32_t base = sP + hf * (T5_TILE / 2) + r * 128;
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            const float p0 = fa::ex2(fmaf(__uint_as_float(v[j]), a.scale_log2, -mu));
-            const float p1 = fa::ex2(fmaf(__uint_as_float(v[j + 1]), a.scale_log2, -mu));
-            ps += p0 + p1;
-            pk[j >> 1] = fa::pack_bf16(p0, p1);
-          }
-        } else {
+      for (int q = 0; q < 8; ++q) {
+        uint32_t pk[4];
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            const float p0 = (key0 + c0 + j <= lim) ? fa::ex2(fmaf(__uint_as_float(v[j]), a.scale_log2, -mu)) : 0.f;
-            const float p1 = (key0 + c0 + j + 1 <= lim) ? fa::ex2(fmaf(__uint_as_float(v[j + 1]), a.scale_log2, -mu)) : 0.f;
-            ps += p0 + p1;
-            pk[j >> 1] = fa::pack_bf16(p0, p1);
-          }
+        for (int j = 0; j < 8; j += 2) {
+          const int k = 8 * q + j;
+          float p0 = fa::ex2(fmaf(__uint_as_float(v[k]), a.scale_log2, -mu));
+          float p1 = fa::ex2(fmaf(__uint_as_float(v[k + 1]), a.scale_log2, -mu));
+          if (!whole) { p0 = (key0 + k <= lim) ? p0 : 0.f; p1 = (key0 + k + 1 <= lim) ? p1 : 0.f; }
+          ps += p0 + p1;
+          pk[j >> 1] = fa::pack_bf16(p0, p1);
         }
-        const uint32_t base = sP + (c0 >> 6) * (T5_TILE / 2) + r * 128;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int ch = ((c0 & 63) >> 3) + q;
-          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(base + ((ch ^ (r & 7)) << 4)), "r"(pk[4 * q]), "r"(pk[4 * q + 1]),
-                       "r"(pk[4 * q + 2]), "r"(pk[4 * q + 3]) : "memory");
-        }
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(base + ((q ^ (r & 7)) << 4)), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
       }
       l = l * corr + ps;
       m = m_new;
@@ -273,24 +267,28 @@ flash_attn_tc5_kernel(const __grid_constant__ CUtensorMap q_map, Flash5Args a) {
     if (ok && n_tiles > 0) {
       if (tc::mbar_wait(o_full, (n_tiles - 1) & 1, abort_flag)) {
         tc::tmem_fence_after();
+        uint32_t w[64];
+        tc::tmem_ld32_nowait(t_lane + 2 * T5_BN, w);
+        tc::tmem_ld32_nowait(t_lane + 2 * T5_BN + 32, w + 32);
+        tc::tmem_ld_wait();
 #pragma unroll
-        for (int c0 = 0; c0 < T5_DH; c0 += 32) {
-          uint32_t v[32];
-          tc::tmem_ld32(t_lane + 2 * T5_BN + c0, v);
-#pragma unroll
-          for (int j = 0; j < 32; ++j) o[c0 + j] = o[c0 + j] * corr + __uint_as_float(v[j]);
-        }
+        for (int j = 0; j < 64; ++j) o[j] = o[j] * corr + __uint_as_float(w[j]);
       }
     }
+    // the row's sum: both halves used the same sequence of maxima, so the partial sums just add
+    xmax[512 + hf * 128 + r] = l;
+    __syncwarp();
+    if (lane == 0) tc::mbar_arrive(pair_bar);
+    if (ok && tc::mbar_wait(pair_bar, n_tiles & 1, abort_flag)) l += xmax[512 + (hf ^ 1) * 128 + r];
     if (row_valid) {
       const float inv = (l > 0.f) ? 1.0f / l : 0.f;
-      bf16* dst = a.out + (int64_t)(row0 + r) * a.out_cols + head * T5_DH;
+      bf16* dst = a.out + (int64_t)(row0 + r) * a.out_cols + head * T5_DH + hf * 64;
 #pragma unroll
-      for (int i = 0; i < T5_DH; i += 8) {
-        uint4 w;
-        w.x = fa::pack_bf16(o[i] * inv, o[i + 1] * inv); w.y = fa::pack_bf16(o[i + 2] * inv, o[i + 3] * inv);
-        w.z = fa::pack_bf16(o[i + 4] * inv, o[i + 5] * inv); w.w = fa::pack_bf16(o[i + 6] * inv, o[i + 7] * inv);
-        *reinterpret_cast<uint4*>(dst + i) = w;
+      for (int i = 0; i < 64; i += 8) {
+        uint4 w4;
+        w4.x = fa::pack_bf16(o[i] * inv, o[i + 1] * inv); w4.y = fa::pack_bf16(o[i + 2] * inv, o[i + 3] * inv);
+        w4.z = fa::pack_bf16(o[i + 4] * inv, o[i + 5] * inv); w4.w = fa::pack_bf16(o[i + 6] * inv, o[i + 7] * inv);
+        *reinterpret_cast<uint4*>(dst + i) = w4;
       }
     }
   }

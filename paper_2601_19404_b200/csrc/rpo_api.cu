@@ -465,7 +465,7 @@ static int attention(rpo_ctx* c, int layer, int rows) {
           CUDA_TRY(cudaFuncSetAttribute(flash_attn_tc5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, T5_SMEM));
           attr_done = true;
         }
-        LAUNCH(c, flash_attn_tc5_kernel, dim3(c->attn_tiles, s.n_q_heads), 192, T5_SMEM, *qm, f);
+        LAUNCH(c, flash_attn_tc5_kernel, dim3(c->attn_tiles, s.n_q_heads), 320, T5_SMEM, *qm, f);
         return RPO_OK;
       }
       if (c->attn_mode == 0) {
