@@ -17,4 +17,4 @@ invariants, brute force on tiny inputs, torch CPU library routines).  The only
 unpinned statement is about the *trained* model of the paper (weights, tokenizer and
 datasets are not available): "parity unpinned" for that, by necessity.
 """
-from . import philox, exactmath, init, decoder, sampler, rollout  # noqa: F401
+from . import philox, exactmath, init, decoder, sampler, rollout, objective  # noqa: F401
