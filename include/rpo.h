@@ -160,6 +160,34 @@ int rpo_token_logprobs(rpo_ctx* ctx, int32_t n_groups, const rpo_group* h_groups
                        const int32_t* d_tokens, const int32_t* d_lens, float inv_temperature,
                        float* d_logprobs_out, float* d_logits_dbg);
 
+/* Hyper-parameters of the objective (Section 4: clip as in GRPO/DAPO, m = 0.5, M = 1, alpha = 0.01). */
+typedef struct rpo_objective_cfg {
+  float clip_eps;          /* epsilon of clip(r, 1 - eps, 1 + eps), Eq. 6                      */
+  float beta;              /* weight of the KL term of Eq. 5 (0: off)                          */
+  float alpha;             /* length sensitivity of Eq. 11                                     */
+  float reward_min;        /* m of Eq. 11                                                      */
+  float reward_max;        /* M of Eq. 11                                                      */
+  int32_t length_shaping;  /* 0: use the raw rewards as R_i                                    */
+} rpo_objective_cfg;
+
+/* Forward value of the RPO objective of one rollout batch (Section 3.2, Eq. 5-7; Section 3.4,
+ * Eq. 11), on the device, from the log-probabilities rpo_token_logprobs produces:
+ *   R_i  = clip(raw_i / (1 + exp(-alpha (l_ref - len_i))), m, M), l_ref = group mean of len  (Eq. 11)
+ *   A_i  = (R_i - mean_R) / std_R over the sampling group (population std; 0 if std = 0)    (Eq. 7)
+ *   l_ij = min(r_ij A_i, clip(r_ij, 1 +- eps) A_i), r_ij = exp(logp_new - logp_old)           (Eq. 6, 7)
+ *   J    = mean over groups of 1/G sum_i 1/|o_i| sum_j [l_ij - beta k3_ij]                    (Eq. 5)
+ * with k3 = exp(d) - d - 1, d = logp_ref - logp_new, the per-token KL estimator of GRPO.
+ *   d_logp_new/old/ref float [B*max_new] (ref NULL: no KL term), d_lens int32 [B] = |o_i| (tokens
+ *   generated in this rollout), d_resp_lens int32 [B] or NULL (= d_lens): len_i of Eq. 11,
+ *   d_raw_rewards float [B]; outputs d_rewards_out [B], d_advantages_out [B], d_token_loss_out
+ *   [B*max_new] or NULL (0 beyond len), d_group_objective_out [n_groups], d_objective_out [1].
+ * Errors: RPO_ERR_LIMIT (G > 64), RPO_ERR_INVALID_ARG. */
+int rpo_policy_objective(rpo_ctx* ctx, int32_t n_groups, int32_t G, int32_t max_new, const float* d_logp_new,
+                         const float* d_logp_old, const float* d_logp_ref, const int32_t* d_lens,
+                         const int32_t* d_resp_lens, const float* d_raw_rewards, const rpo_objective_cfg* cfg,
+                         float* d_rewards_out, float* d_advantages_out, float* d_token_loss_out,
+                         float* d_group_objective_out, float* d_objective_out);
+
 /* Return the groups' shared KV blocks and slots to the pool (host bookkeeping; work
  * already enqueued on the stream is unaffected because later work is ordered after it). */
 int rpo_release_groups(rpo_ctx* ctx, int32_t n_groups, const rpo_group* h_groups);

@@ -4,5 +4,5 @@
 exposes the same calls as `include/rpo.h`; it only marshals arguments.  There is no
 CPU path: importing works anywhere, computing needs a CUDA device.
 """
-from .binding import (Context, Sampler, Group, shape_preset, load_library, RpoError, EXPORTED_SYMBOLS,
+from .binding import (Context, Sampler, Group, ObjectiveCfg, shape_preset, load_library, RpoError, EXPORTED_SYMBOLS,
                       sample_rows_noalloc)  # noqa: F401

@@ -14,7 +14,7 @@ _LIB = None
 EXPORTED_SYMBOLS = [
     "rpo_strerror", "rpo_shape_preset", "rpo_create", "rpo_destroy", "rpo_init_weights", "rpo_read_tensor",
     "rpo_write_tensor", "rpo_prefill_prefix", "rpo_decode_suffix", "rpo_token_logprobs", "rpo_release_groups",
-    "rpo_rollout_host", "rpo_sample_rows", "rpo_sample_rows_noalloc", "rpo_gemm", "rpo_gemm_bench", "rpo_device_status", "rpo_counters", "rpo_set_option", "rpo_profile_read",
+    "rpo_policy_objective", "rpo_rollout_host", "rpo_sample_rows", "rpo_sample_rows_noalloc", "rpo_gemm", "rpo_gemm_bench", "rpo_device_status", "rpo_counters", "rpo_set_option", "rpo_profile_read",
 ]
 
 
@@ -43,6 +43,14 @@ class Sampler(C.Structure):
         super().__init__(float(temperature), float(top_p), int(bool(greedy)), int(eos_id), int(seed))
 
 
+class ObjectiveCfg(C.Structure):
+    _fields_ = [("clip_eps", C.c_float), ("beta", C.c_float), ("alpha", C.c_float), ("reward_min", C.c_float),
+                ("reward_max", C.c_float), ("length_shaping", C.c_int32)]
+
+    def __init__(self, clip_eps=0.2, beta=0.0, alpha=0.01, reward_min=0.5, reward_max=1.0, length_shaping=True):
+        super().__init__(float(clip_eps), float(beta), float(alpha), float(reward_min), float(reward_max), int(bool(length_shaping)))
+
+
 class Group(C.Structure):
     _fields_ = [("group_id", C.c_int32), ("prefix_len", C.c_int32), ("slot", C.c_int32), ("n_blocks", C.c_int32)]
 
@@ -68,6 +76,7 @@ def load_library(path=None):
     lib.rpo_prefill_prefix.argtypes = [vp, i32, vp, vp, vp, C.POINTER(Group)]
     lib.rpo_decode_suffix.argtypes = [vp, i32, C.POINTER(Group), i32, i32, C.POINTER(Sampler), vp, vp, vp, vp, vp]
     lib.rpo_token_logprobs.argtypes = [vp, i32, C.POINTER(Group), i32, i32, vp, vp, f32, vp, vp]
+    lib.rpo_policy_objective.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, C.POINTER(ObjectiveCfg), vp, vp, vp, vp, vp]
     lib.rpo_release_groups.argtypes = [vp, i32, C.POINTER(Group)]
     lib.rpo_rollout_host.argtypes = [vp, i32, vp, vp, vp, i32, i32, C.POINTER(Sampler), vp, vp, vp, i32, vp]
     lib.rpo_sample_rows.argtypes = [vp, i32, i32, vp, C.POINTER(Sampler), vp, i32, vp, vp]
@@ -209,6 +218,14 @@ class Context:
         _check(self.lib.rpo_token_logprobs(self.handle, len(groups), groups, int(G), int(max_new), _ptr(d_tokens),
                                            _ptr(d_lens), float(inv_temperature), _ptr(d_logprobs_out),
                                            _ptr(d_logits_dbg)), "rpo_token_logprobs")
+
+    def policy_objective(self, n_groups, G, max_new, d_logp_new, d_logp_old, d_lens, d_raw_rewards, cfg, d_rewards_out,
+                         d_advantages_out, d_group_objective_out, d_objective_out, d_logp_ref=None, d_resp_lens=None,
+                         d_token_loss_out=None):
+        _check(self.lib.rpo_policy_objective(self.handle, int(n_groups), int(G), int(max_new), _ptr(d_logp_new), _ptr(d_logp_old),
+                                             _ptr(d_logp_ref), _ptr(d_lens), _ptr(d_resp_lens), _ptr(d_raw_rewards), C.byref(cfg),
+                                             _ptr(d_rewards_out), _ptr(d_advantages_out), _ptr(d_token_loss_out),
+                                             _ptr(d_group_objective_out), _ptr(d_objective_out)), "rpo_policy_objective")
 
     def release_groups(self, groups):
         _check(self.lib.rpo_release_groups(self.handle, len(groups), groups), "rpo_release_groups")

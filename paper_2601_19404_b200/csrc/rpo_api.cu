@@ -16,6 +16,7 @@
 #include "context.h"
 #include "gemm_tc.cuh"
 #include "kernels.cuh"
+#include "objective.cuh"
 #include "ref_kernels.cuh"
 #include "sampler.cuh"
 
@@ -892,6 +893,32 @@ extern "C" int rpo_token_logprobs(rpo_ctx* c, int32_t n_groups, const rpo_group*
                                     d_logprobs_out, d_logits_dbg)
                  : logprobs_t<float>(c, n_groups, h_groups, G, max_new, d_tokens, d_lens, inv_temperature,
                                      d_logprobs_out, d_logits_dbg);
+}
+
+// ---------------------------------------------------------------------------------------------
+// objective forward (Eq. 5-7, Eq. 11)
+// ---------------------------------------------------------------------------------------------
+extern "C" int rpo_policy_objective(rpo_ctx* c, int32_t n_groups, int32_t G, int32_t max_new, const float* d_logp_new,
+                                    const float* d_logp_old, const float* d_logp_ref, const int32_t* d_lens,
+                                    const int32_t* d_resp_lens, const float* d_raw_rewards, const rpo_objective_cfg* cfg,
+                                    float* d_rewards_out, float* d_advantages_out, float* d_token_loss_out,
+                                    float* d_group_objective_out, float* d_objective_out) {
+  if (!c || n_groups <= 0 || G <= 0 || max_new <= 0 || !d_logp_new || !d_logp_old || !d_lens || !d_raw_rewards || !cfg ||
+      !d_rewards_out || !d_advantages_out || !d_group_objective_out || !d_objective_out)
+    return RPO_ERR_INVALID_ARG;
+  if (G > OBJ_MAX_G) return RPO_ERR_LIMIT;
+  if (!(cfg->clip_eps >= 0.f) || !(cfg->reward_max >= cfg->reward_min)) return RPO_ERR_INVALID_ARG;
+  ObjectiveArgs a;
+  memset(&a, 0, sizeof(a));
+  a.logp_new = d_logp_new; a.logp_old = d_logp_old; a.logp_ref = d_logp_ref; a.lens = d_lens; a.resp_lens = d_resp_lens;
+  a.raw_rewards = d_raw_rewards; a.G = G; a.S = max_new; a.clip_eps = cfg->clip_eps; a.beta = cfg->beta; a.alpha = cfg->alpha;
+  a.r_min = cfg->reward_min; a.r_max = cfg->reward_max; a.length_shaping = cfg->length_shaping;
+  a.rewards_out = d_rewards_out; a.adv_out = d_advantages_out; a.token_loss_out = d_token_loss_out;
+  a.group_obj_out = d_group_objective_out;
+  const int threads = std::max(64, std::min(1024, G * 32));
+  LAUNCH(c, objective_group_kernel, n_groups, threads, 0, a);
+  LAUNCH(c, objective_reduce_kernel, 1, 32, 0, (const float*)d_group_objective_out, n_groups, d_objective_out);
+  return RPO_OK;
 }
 
 // ---------------------------------------------------------------------------------------------
