@@ -58,3 +58,36 @@ def test_objective_matches_oracle(n_groups, G, S):
                 z = torch.zeros(130, device=DEV)
                 ctx.policy_objective(2, 65, 1, z, z, torch.ones(130, dtype=torch.int32, device=DEV), z, rpo.ObjectiveCfg(), z, z, z, z)
         assert ctx.device_status() == 0
+
+
+def test_rollout_stage_end_to_end_on_the_tiny_decoder():
+    """Algorithm 1's inner loop for two iterations on the tiny fp32 decoder with a synthetic reward."""
+    from paper_2601_19404_b200 import experience as ex
+    shape = workloads.SHAPES["tiny"]
+    rng = np.random.default_rng(5)
+    cache = ex.ExperienceCache()
+    for q in range(3):
+        cache.put(q, rng.integers(0, 1024, 12), rng.integers(0, 1024, 40 + 7 * q))
+    G, S = 4, 12
+    with make_ctx(shape, 3, G, 120, S, chunk=512) as ctx:
+        ctx.init_weights(0, 0.02)
+        reward = lambda q, qt, o: float(int(o[-1]) % 2 == 0)                     # stands in for the verifier
+        stage = ex.RolloutStage(ctx, cache, G, S, rpo.Sampler(1.0, 0.95, False, -1, 3), reward, L=10, dynamic_factor=0.5, eps=0.5,
+                                seed=1, objective_cfg=rpo.ObjectiveCfg(0.2, 0.0, 0.01, 0.5, 1.0, True))
+        before = {q: cache.retrieve(q)[1].copy() for q in range(3)}
+        for it in range(2):
+            res = stage.run([0, 1, 2])
+            assert res["tokens"].shape == (3 * G, S) and np.all(res["lens"] == S)
+            # first iteration: fixed L = 10; afterwards L = 0.5 * the shortest response of the last group (Eq. 4)
+            assert all(0 <= m <= (10 if it == 0 else 0.5 * before[q].size + 1) for q, m in enumerate(res["truncations"]))
+            # decode-time and teacher-forced log-probs agree, so every ratio is 1 and the objective is ~0
+            assert np.max(np.abs(res["policy_logprobs"] - res["logprobs"])) < 1e-4
+            o = ob.objective(res["policy_logprobs"], res["logprobs"], res["lens"], res["raw_rewards"], G, resp_lens=res["resp_lens"])
+            assert np.max(np.abs(res["rewards"] - o["rewards"])) < 1e-6 and abs(res["objective"] - o["objective"]) < 1e-4
+            for q in range(3):                                                    # the cache now holds one of the new responses
+                a = cache.retrieve(q)[1]
+                kept = before[q].size - res["truncations"][q]
+                assert np.array_equal(a[:kept], before[q][:kept]) and a.size == kept + S
+                assert np.array_equal(a[kept:], res["tokens"][q * G + res["chosen"][q]])
+                before[q] = a.copy()
+        assert ctx.device_status() == 0
