@@ -69,11 +69,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 }  // namespace fa
 
-// Tile shape per mode.  Prefill (ROWS) is compute-bound: four warps, 16 query rows each, Q fragments
-// kept in registers.  Decode (SHARED) is bound by the latency of one CTA's chain of tiles: eight
-// warps, the two halves of every 64-key tile go to different warps (KS = 2) with their own softmax
-// state, merged through shared memory at the end; Q fragments are re-read from shared memory and
-// registers are capped so that two such CTAs share an SM.
+// Tile shape per mode: 64-key tiles, four consumer warps of 16 query rows each (+ the producer warp),
+// Q fragments kept in registers, two CTAs per SM.  Decode (SHARED) looks one K tile further ahead
+// than prefill.  KS > 1 (several warp sets sharing the keys of a tile, merged through shared memory
+// at the end) is kept as an option; it did not pay at the measured sizes.
 template <int MODE> struct FaCfg {
   static constexpr int BN = (MODE == FA_SHARED) ? 64 : 64;     // keys per tile
   static constexpr int NSK = (MODE == FA_SHARED) ? 3 : 2;      // K ring depth: K tiles are fetched NSK-1 tiles ahead,
@@ -473,8 +472,7 @@ flash_attn_kernel(FlashArgs a) {
   }
 }
 
-// Decode: log-sum-exp merge of the partials of (sequence, query head) -- slots 0..n_splits-1 from the
-// splits of the shared prefix, slot n_splits from the sequence's own suffix keys (n_slots <= 33) -- one
+// Decode: log-sum-exp merge of the per-split partials of (sequence, query head), n_slots <= 33, one
 // warp each.  Lane s first reads (m, l) of slot s, the warp agrees on the maximum and on each
 // slot's weight, then all slots' O rows are accumulated with independent loads in slot order
 // (reproducible); lanes own DH/32 dimensions.

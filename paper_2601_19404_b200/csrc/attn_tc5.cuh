@@ -27,7 +27,6 @@ constexpr int T5_TILE = T5_BN * T5_DH * 2;                       // 32 KB: one K
 constexpr int T5_SMEM = (2 + T5_NSK + T5_NSV) * T5_TILE + 1024 + 256 + 3072;   // tiles, alignment, barriers, row-maximum exchange
 
 struct Flash5Args {
-  const bf16* qkv_unused;
   bf16* out; int out_cols;
   const int32_t* row_seq; const int32_t* row_t; const SeqDesc* seqs; const int32_t* block_table;
   KVPool<bf16> pool; int layer, hq, hkv; float scale_log2;
