@@ -181,6 +181,46 @@ __global__ void rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ 
   }
 }
 
+// RMSNorm for many rows (prefill, log-prob passes): one warp per row, the row held in registers
+// (d <= 4096, d % 128 == 0 not required: lanes take float4 number lane, lane + 32, ...), no shared
+// memory and no block barrier.  Same arithmetic as rmsnorm_kernel without split-K planes.
+template <typename T, int MAXV>
+__global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const float* __restrict__ x, const float* __restrict__ gain,
+                                                           T* __restrict__ h, int rows, int d, float eps) {
+  pdl_prologue();
+  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (r >= rows) return;
+  const int d4 = d >> 2;
+  const float4* xr = reinterpret_cast<const float4*>(x + (int64_t)r * d);
+  float4 v[MAXV];
+  float ss = 0.f;
+#pragma unroll
+  for (int k = 0; k < MAXV; ++k) {
+    const int i = lane + 32 * k;
+    if (i < d4) { v[k] = xr[i]; ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w; }
+  }
+  ss = warp_sum(ss);
+  const float inv = 1.0f / sqrtf(ss / (float)d + eps);
+  const float4* g4 = reinterpret_cast<const float4*>(gain);
+  T* hr = h + (int64_t)r * d;
+#pragma unroll
+  for (int k = 0; k < MAXV; ++k) {
+    const int i = lane + 32 * k;
+    if (i < d4) {
+      const float4 g = g4[i];
+      if (sizeof(T) == 2) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(v[k].x * inv * g.x, v[k].y * inv * g.y);
+        __nv_bfloat162 b = __floats2bfloat162_rn(v[k].z * inv * g.z, v[k].w * inv * g.w);
+        uint2 o; o.x = *reinterpret_cast<uint32_t*>(&a); o.y = *reinterpret_cast<uint32_t*>(&b);
+        *reinterpret_cast<uint2*>(hr + 4 * i) = o;
+      } else {
+        float4 o = make_float4(v[k].x * inv * g.x, v[k].y * inv * g.y, v[k].z * inv * g.z, v[k].w * inv * g.w);
+        *reinterpret_cast<float4*>(hr + 4 * i) = o;
+      }
+    }
+  }
+}
+
 // x[i] += sum_s partial[s*stride + i], fixed order (deterministic split-K reduction). n % 4 == 0.
 __global__ void reduce_partials_kernel(float* __restrict__ x, const float* __restrict__ partial, int n_splits, int64_t n,
                                        int64_t stride) {

@@ -410,6 +410,11 @@ static int rmsnorm(rpo_ctx* c, float* x, const float* g, T* h, int rows) {
   const int d = c->shape.d_model;
   const bool fold = (x == c->ws.x && c->pending_splits > 0 && c->pending_rows == rows);
   if (!fold && x == c->ws.x) RPO_TRY(flush_partials(c));
+  if (!fold && rows >= 1024 && d <= 4096) {     // many rows: a warp per row, the row in registers
+    if (d <= 2048) LAUNCH(c, (rmsnorm_rows_kernel<T, 16>), ceil_div(rows, 8), 256, 0, (const float*)x, g, h, rows, d, c->shape.rms_eps);
+    else LAUNCH(c, (rmsnorm_rows_kernel<T, 32>), ceil_div(rows, 8), 256, 0, (const float*)x, g, h, rows, d, c->shape.rms_eps);
+    return RPO_OK;
+  }
   const int threads = std::min(1024, ((d / 4 + 31) / 32) * 32);
   LAUNCH(c, rmsnorm_kernel<T>, rows, threads, (size_t)d * 4, x, g, h, rows, d, c->shape.rms_eps,
          fold ? (const float*)c->ws.partial : (const float*)nullptr, fold ? c->pending_splits : 0,
