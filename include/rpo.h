@@ -261,9 +261,12 @@ int rpo_counters(rpo_ctx* ctx, int64_t* kernel_launches, int64_t* free_kv_blocks
 /* Runtime switches (tests/benchmarks): name = "use_tcgen05" (bf16 GEMMs on the tensor-core
  * kernel, default 1), "use_tc_attention" (tensor-core attention kernels, default 1),
  * "use_graph" (CUDA graph per decode step, default 1), "use_pdl" (programmatic dependent launch
- * between the library's kernels, default 1), "profile" (see rpo_profile_read),
- * "gemm_bn" (0 = planner, else force the tensor-core tile width: 32/64/96/128/256) and
- * "gemm_splits" (with gemm_bn: force the split-K factor where the caller can reduce planes). */
+ * between the library's kernels, default 1), "use_tc5_attention" (tcgen05 attention for
+ * many-row passes at head_dim 128, default 1), "use_gemm_pairs" (256 x 256 GEMM tiles on CTA
+ * pairs for many-row passes, default 1), "profile" (see rpo_profile_read),
+ * "gemm_bn" (0 = planner, else force the tensor-core tile width: 32/64/96/128/256, or 512 for
+ * the CTA-pair kernel) and "gemm_splits" (with gemm_bn: force the split-K factor where the
+ * caller can reduce planes). */
 int rpo_set_option(rpo_ctx* ctx, const char* name, int32_t value);
 
 /* Per-kernel timing.  With option "profile" = 1 every kernel launch is bracketed by a pair of

@@ -89,7 +89,8 @@ struct rpo_ctx {
   int use_tcgen05 = 1, use_tc_attention = 1, use_graph = 1;
   int use_tc5_attention = 1, tc5_v_variant = 0;   // tcgen05 prefill attention (and the descriptor reading under test)
   int use_pdl = 1;                    // programmatic dependent launch between the library's kernels
-  int gemm_bn = 0, gemm_splits = 0;   // > 0: override the GEMM planner (tests, sweeps)
+  int use_gemm_pairs = 1;             // 256 x 256 tiles on CTA pairs (cta_group::2) for many-row GEMMs
+  int gemm_bn = 0, gemm_splits = 0;   // > 0: override the GEMM planner (tests, sweeps); 512 = pair tiles
   // attention plan of the pass being enqueued: 0 = row tiles (prefill / teacher), 1 = decode
   int attn_mode = 0, attn_tiles = 0, attn_G = 1, attn_groups = 0, attn_splits = 1, attn_split_chunk = 64;
   int pending_splits = 0, pending_rows = 0;   // split-K partials of ws.x not yet reduced

@@ -1,6 +1,6 @@
 // bf16 GEMM on the 5th-generation tensor cores: C[M,N] = A[M,K] * W[N,K]^T, float32 accumulation.
 //
-//   * operands: TMA (cp.async.bulk.tensor.2d, no multicast) into 128-byte-swizzled shared memory,
+//   * operands: TMA (cp.async.bulk.tensor.2d, every CTA fetching its own tiles) into 128-byte-swizzled shared memory,
 //     a ring of NS stages of [128 x 64] (A) and [BN x 64] (W) tiles guarded by mbarriers;
 //   * math: tcgen05.mma kind::f16 (bf16 x bf16 -> f32), M = 128, N = BN, K = 16 per instruction,
 //     issued by one thread; accumulators live in tensor memory, two buffers of BN columns so the
@@ -131,6 +131,52 @@ __device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t* r) {
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 }  // namespace tc
+
+// Epilogue of one 32-column chunk of an accumulator row: r[0..31] are the float32 bit patterns of
+// columns col .. col+31 of output row `row`.
+template <int EPI>
+__device__ __forceinline__ void tc_store_chunk(const TcParams& p, const uint32_t* r, int row, int col, int split) {
+  if (row >= p.M || col >= p.N) return;
+  const int ncol = min(32, p.N - col);       // multiple of 8 (N % 8 == 0)
+  if (EPI == TC_STORE_BF16) {
+    bf16* dst = (bf16*)p.C + (int64_t)row * p.ldc + col;
+    for (int j = 0; j < ncol; j += 8) {
+      uint4 v;
+      __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+      __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+      __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]));
+      __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
+      v.x = *(uint32_t*)&h0; v.y = *(uint32_t*)&h1; v.z = *(uint32_t*)&h2; v.w = *(uint32_t*)&h3;
+      *(uint4*)(dst + j) = v;
+    }
+  } else if (EPI == TC_SWIGLU) {
+    // columns (2j, 2j+1) = (gate_j, up_j)  ->  out[row, col/2 + j]
+    bf16* dst = (bf16*)p.C + (int64_t)row * p.ldc + col / 2;
+    for (int j = 0; j < ncol; j += 16) {
+      uint32_t o[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float g0 = __uint_as_float(r[j + 4 * q]), u0 = __uint_as_float(r[j + 4 * q + 1]);
+        const float g1 = __uint_as_float(r[j + 4 * q + 2]), u1 = __uint_as_float(r[j + 4 * q + 3]);
+        __nv_bfloat162 h = __floats2bfloat162_rn(g0 / (1.0f + __expf(-g0)) * u0, g1 / (1.0f + __expf(-g1)) * u1);
+        o[q] = *(uint32_t*)&h;
+      }
+      *(uint4*)(dst + j / 2) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+  } else {
+    float* dst = (EPI == TC_PARTIAL) ? (float*)p.C + split * p.split_stride + (int64_t)row * p.ldc + col
+                                     : (float*)p.C + (int64_t)row * p.ldc + col;
+    for (int j = 0; j < ncol; j += 4) {
+      float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
+                             __uint_as_float(r[j + 3]));
+      if (EPI == TC_ADD_F32) {
+        const float4 o = *(float4*)(dst + j);
+        v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+      }
+      *(float4*)(dst + j) = v;
+    }
+  }
+}
 
 template <int BN>
 struct TcCfg {
@@ -263,48 +309,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       for (int c0 = 0; c0 < BN; c0 += 32) {
         uint32_t r[32];
         tc::tmem_ld32(t_row + (uint32_t)c0, r);
-        const int col = tn * BN + c0;
-        if (row < p.M && col < p.N) {
-          const int ncol = min(32, p.N - col);       // multiple of 8 (N % 8 == 0)
-          if (EPI == TC_STORE_BF16) {
-            bf16* dst = (bf16*)p.C + (int64_t)row * p.ldc + col;
-            for (int j = 0; j < ncol; j += 8) {
-              uint4 v;
-              __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
-              __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
-              __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]));
-              __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
-              v.x = *(uint32_t*)&h0; v.y = *(uint32_t*)&h1; v.z = *(uint32_t*)&h2; v.w = *(uint32_t*)&h3;
-              *(uint4*)(dst + j) = v;
-            }
-          } else if (EPI == TC_SWIGLU) {
-            // columns (2j, 2j+1) = (gate_j, up_j)  ->  out[row, col/2 + j]
-            bf16* dst = (bf16*)p.C + (int64_t)row * p.ldc + col / 2;
-            for (int j = 0; j < ncol; j += 16) {
-              uint32_t o[4];
-#pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                const float g0 = __uint_as_float(r[j + 4 * q]), u0 = __uint_as_float(r[j + 4 * q + 1]);
-                const float g1 = __uint_as_float(r[j + 4 * q + 2]), u1 = __uint_as_float(r[j + 4 * q + 3]);
-                __nv_bfloat162 h = __floats2bfloat162_rn(g0 / (1.0f + __expf(-g0)) * u0, g1 / (1.0f + __expf(-g1)) * u1);
-                o[q] = *(uint32_t*)&h;
-              }
-              *(uint4*)(dst + j / 2) = make_uint4(o[0], o[1], o[2], o[3]);
-            }
-          } else {
-            float* dst = (EPI == TC_PARTIAL) ? (float*)p.C + split * p.split_stride + (int64_t)row * p.ldc + col
-                                             : (float*)p.C + (int64_t)row * p.ldc + col;
-            for (int j = 0; j < ncol; j += 4) {
-              float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
-                                     __uint_as_float(r[j + 3]));
-              if (EPI == TC_ADD_F32) {
-                const float4 o = *(float4*)(dst + j);
-                v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-              }
-              *(float4*)(dst + j) = v;
-            }
-          }
-        }
+        tc_store_chunk<EPI>(p, r, row, tn * BN + c0, split);
       }
       tc::tmem_fence_before();
       __syncwarp();

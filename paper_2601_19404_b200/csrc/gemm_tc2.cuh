@@ -1,0 +1,261 @@
+// bf16 GEMM for many-row passes (prefill, token log-probs) on CTA pairs: C[M,N] = A[M,K] * W[N,K]^T.
+//
+// A 128 x 256 tile per CTA needs 48 KB of operands per 64-wide k-block, and the path from L2 into
+// shared memory, not the tensor pipe, then sets the pace.  Here two CTAs of a cluster share one
+// 256 x 256 tile: `tcgen05.mma.cta_group::2` (M = 256, N = 256, K = 16) reads rows 128r..128r+127
+// of the A tile and rows 128r..128r+127 of the W tile from the shared memory of the CTA of rank r,
+// and leaves rows 128r.. of the accumulator in that CTA's tensor memory.  Each CTA therefore loads
+// 32 KB per k-block for the same tensor-pipe time: two thirds of the operand traffic per flop.
+//
+//   * both CTAs run a TMA producer for their own halves (tensor loads qualified `.cta_group::2`,
+//     each CTA fetching only what it needs itself), completing on the *leader's* (rank 0) full
+//     barrier, which expects the bytes of both;
+//   * the leader's MMA thread issues the pair-wide instructions and releases ring stages and
+//     accumulators in both CTAs with one `tcgen05.commit` that arrives on both CTAs' barriers;
+//   * each CTA drains its own 128 accumulator rows (two buffers of 256 columns = all 512 columns
+//     of tensor memory, so the epilogue of one tile overlaps the main loop of the next) and tells
+//     the leader when a buffer is free again (remote mbarrier arrive).
+//   * persistent: cluster i walks tiles i, i + n_clusters, ...; every wait is bounded as in
+//     gemm_tc.cuh; no CTA leaves before its peer (cluster barrier at the end).
+#pragma once
+#include "gemm_tc.cuh"
+
+namespace rpo {
+
+constexpr int TC2_NS = 6;
+constexpr int TC2_HALF_BYTES = 128 * TC_BK * 2;          // 16 KB: 128 rows x 64 bf16
+constexpr int TC2_STAGE_BYTES = 2 * TC2_HALF_BYTES;      // A half + W half
+constexpr int TC2_SMEM_BYTES = TC2_NS * TC2_STAGE_BYTES + 1024 + 256;
+
+namespace tc {
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address of the same shared-memory location in the CTA of rank `rank` of this cluster.
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t smem_addr, uint32_t rank) {
+  uint32_t a;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(smem_addr), "r"(rank));
+  return a;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Pair-wide TMA load into this CTA's shared memory; the bytes complete on `bar_cluster_addr`,
+// which may live in the peer CTA.
+__device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorMap* map, int x, int y, uint32_t bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(bar_cluster_addr), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  const uint32_t z = 0;
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n}"
+      ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(z) : "memory");
+}
+// Arrives (once all MMAs issued so far have completed) on the barrier at this shared-memory
+// offset in every CTA of `cta_mask`.
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar, uint16_t cta_mask) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(smem_u32(bar)), "h"(cta_mask) : "memory");
+}
+
+}  // namespace tc
+
+// 192 threads per CTA, clusters of two: warp 0 = TMA producer, warp 1 = tensor-memory owner (and,
+// in the leader, MMA issuer), warps 2..5 = epilogue.  p.tiles_m / p.tiles_n count 256 x 256 tiles.
+template <int EPI>
+__global__ void __launch_bounds__(192, 1)
+gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = (uint64_t*)(smem + TC2_NS * TC2_STAGE_BYTES);
+  uint64_t* full = bars;                         // used in the leader only
+  uint64_t* empty = bars + TC2_NS;
+  uint64_t* acc_full = bars + 2 * TC2_NS;
+  uint64_t* acc_empty = bars + 2 * TC2_NS + 2;   // used in the leader only
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * TC2_NS + 4);
+  volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = tc::cluster_ctarank();
+  const bool leader = (rank == 0);
+  const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+  const int n_items = p.tiles_m * p.tiles_n;
+  pdl_launch_dependents();
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < TC2_NS; ++i) { tc::mbar_init(&full[i], 1); tc::mbar_init(&empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { tc::mbar_init(&acc_full[i], 1); tc::mbar_init(&acc_empty[i], 8); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc::smem_u32(tmem_slot)),
+                 "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc::tmem_fence_before();
+  __syncthreads();
+  tc::cluster_sync_all();                        // the peer's barriers exist before anything arrives on them
+  tc::tmem_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+      pdl_wait();
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      for (int it = cluster_id; it < n_items && ok; it += n_clusters) {
+        const int tn = it % p.tiles_n, tm = it / p.tiles_n;
+        const int row_a = tm * 256 + (int)rank * 128, row_w = tn * 256 + (int)rank * 128;
+        for (int kb = 0; kb < p.kb_total; ++kb) {
+          if (!tc::mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+          uint8_t* sa = smem + stage * TC2_STAGE_BYTES;
+          if (leader) tc::mbar_expect_tx(&full[stage], 2 * TC2_STAGE_BYTES);
+          const uint32_t bar = tc::map_to_rank(tc::smem_u32(&full[stage]), 0);
+          tc::tma_load_2d_pair(sa, &map_a, kb * TC_BK, row_a, bar);
+          tc::tma_load_2d_pair(sa + TC2_HALF_BYTES, &map_w, kb * TC_BK, row_w, bar);
+          if (++stage == TC2_NS) { stage = 0; phase ^= 1; }
+        }
+      }
+      // Drain: every stage this CTA filled has been released, i.e. all arrivals aimed at this
+      // CTA's barriers have landed before its shared memory goes away.
+      for (int i = 0; i < TC2_NS && ok; ++i) {
+        if (!tc::mbar_wait(&empty[stage], phase ^ 1, abort_flag)) ok = false;
+        if (++stage == TC2_NS) { stage = 0; phase ^= 1; }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader only)
+    if (leader && lane == 0) {
+      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+      int stage = 0; uint32_t phase = 0;
+      int acc = 0; uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int it = cluster_id; it < n_items && ok; it += n_clusters) {
+        if (!tc::mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag)) { ok = false; break; }
+        tc::tmem_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * 256);
+        for (int kb = 0; kb < p.kb_total; ++kb) {
+          if (!tc::mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+          tc::tmem_fence_after();
+          const uint32_t sa = tc::smem_u32(smem + stage * TC2_STAGE_BYTES);
+          const uint64_t da = tc::umma_desc_sw128(sa), db = tc::umma_desc_sw128(sa + TC2_HALF_BYTES);
+#pragma unroll
+          for (int k = 0; k < TC_BK / 16; ++k)
+            tc::umma_bf16_pair(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          tc::umma_commit_pair(&empty[stage], 3);       // frees the stage in both CTAs
+          if (++stage == TC2_NS) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        tc::umma_commit_pair(&acc_full[acc], 3);        // accumulator complete, both CTAs
+        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+    const int quad = warp & 3;
+    pdl_wait();
+    int acc = 0; uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int it = cluster_id; it < n_items && ok; it += n_clusters) {
+      const int tn = it % p.tiles_n, tm = it / p.tiles_n;
+      if (!tc::mbar_wait(&acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+      tc::tmem_fence_after();
+      const int row = tm * 256 + (int)rank * 128 + quad * 32 + lane;
+      const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * 256);
+#pragma unroll 1
+      for (int c0 = 0; c0 < 256; c0 += 32) {
+        uint32_t r[32];
+        tc::tmem_ld32(t_row + (uint32_t)c0, r);
+        tc_store_chunk<EPI>(p, r, row, tn * 256 + c0, 0);
+      }
+      tc::tmem_fence_before();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive_cluster(tc::map_to_rank(tc::smem_u32(&acc_empty[acc]), 0));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+    }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  __syncwarp();
+  tc::tmem_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) atomicOr(p.status, STATUS_TIMEOUT);
+    for (int i = 0; i < 64; ++i) __nanosleep(1000000);   // let copies in flight land before shared memory goes away
+    __syncthreads();
+  }
+  tc::cluster_sync_all();                        // the peer no longer touches this CTA's barriers or tensor memory
+  if (warp == 1) {
+    tc::tmem_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+template <int EPI>
+inline int tc2_launch(rpo_ctx* c, const CUtensorMap* ma, const CUtensorMap* mw, const TcParams& p) {
+  static int max_clusters = -1;
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = TC2_SMEM_BYTES; cfg.stream = c->stream;
+  cfg.attrs = attr;
+  if (max_clusters < 0) {
+    if (cudaFuncSetAttribute(gemm_tc2_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC2_SMEM_BYTES) != cudaSuccess)
+      return RPO_ERR_CUDA;
+    cfg.gridDim = dim3(2 * (c->sm_count / 2)); cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_tc2_kernel<EPI>, &cfg) != cudaSuccess || n < 1) { cudaGetLastError(); n = c->sm_count / 2; }
+    max_clusters = std::min(n, c->sm_count / 2);
+  }
+  const int clusters = std::min(p.tiles_m * p.tiles_n, max_clusters);
+  cfg.gridDim = dim3(2 * clusters);
+  cfg.numAttrs = c->use_pdl ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI>, *ma, *mw, p) == cudaSuccess ? RPO_OK : RPO_ERR_CUDA;
+}
+
+// True when the pass is large enough for pair tiles to fill the machine.
+inline bool tc2_wanted(rpo_ctx* c, int M, int N) {
+  if (c->gemm_bn > 0) return c->gemm_bn == 512;           // test / sweep override: 512 = pair tiles
+  if (!c->use_gemm_pairs) return false;
+  const int tiles = ((M + 255) / 256) * ((N + 255) / 256);
+  return M >= 1024 && tiles >= c->sm_count / 2;
+}
+
+inline int tc2_gemm_launch(rpo_ctx* c, const bf16* A, const bf16* W, void* C, int M, int N, int K, int epi, int ldc) {
+  TcParams p;
+  p.C = C; p.M = M; p.N = N; p.K = K; p.ldc = ldc;
+  p.tiles_m = (M + 255) / 256; p.tiles_n = (N + 255) / 256; p.splits = 1; p.kb_total = K / TC_BK; p.kb_per_split = p.kb_total;
+  p.split_stride = 0; p.status = c->d_status;
+  const CUtensorMap* ma = tc_map(c, A, M, K, 128);
+  const CUtensorMap* mw = tc_map(c, W, N, K, 128);
+  if (!ma || !mw) return RPO_ERR_CUDA;
+  switch (epi) {
+    case TC_STORE_BF16: return tc2_launch<TC_STORE_BF16>(c, ma, mw, p);
+    case TC_STORE_F32: return tc2_launch<TC_STORE_F32>(c, ma, mw, p);
+    case TC_ADD_F32: return tc2_launch<TC_ADD_F32>(c, ma, mw, p);
+    case TC_SWIGLU: return tc2_launch<TC_SWIGLU>(c, ma, mw, p);
+    default: return RPO_ERR_INVALID_ARG;
+  }
+}
+
+}  // namespace rpo

@@ -15,6 +15,7 @@
 #include "attn_tc5.cuh"
 #include "context.h"
 #include "gemm_tc.cuh"
+#include "gemm_tc2.cuh"
 #include "kernels.cuh"
 #include "objective.cuh"
 #include "ref_kernels.cuh"
@@ -385,8 +386,11 @@ static int gemm(rpo_ctx* c, const T* A, const T* W, void* C, int M, int N, int K
                      : epi == EPI_ADD_F32 ? TC_ADD_F32 : TC_SWIGLU;
     int splits = 0;
     prof_begin(c);
-    const int rc = tc_gemm_launch(c, (const bf16*)A, (const bf16*)W, C, M, N, K, tc_epi, tc_epi == TC_SWIGLU ? N / 2 : N,
-                                  allow_split && (epi == EPI_ADD_F32 || splits_out), &splits);
+    const int ldc = tc_epi == TC_SWIGLU ? N / 2 : N;
+    const int rc = tc2_wanted(c, M, N)
+                       ? tc2_gemm_launch(c, (const bf16*)A, (const bf16*)W, C, M, N, K, tc_epi, ldc)
+                       : tc_gemm_launch(c, (const bf16*)A, (const bf16*)W, C, M, N, K, tc_epi, ldc,
+                                        allow_split && (epi == EPI_ADD_F32 || splits_out), &splits);
     prof_end(c);
     c->launches++;
     if (rc == RPO_OK && splits > 1) {
@@ -1010,8 +1014,11 @@ extern "C" int rpo_gemm_bench(rpo_ctx* c, int32_t M, int32_t N, int32_t K, const
   auto enqueue = [&]() -> int {
     for (int i = 0; i < iters; ++i) {
       int splits = 0;
-      RPO_TRY(tc_gemm_launch(c, (const bf16*)d_A, (const bf16*)h_W_list[i % n_w], c->ws.logits, M, N, K, TC_STORE_F32, N,
-                             true, &splits));
+      if (tc2_wanted(c, M, N))
+        RPO_TRY(tc2_gemm_launch(c, (const bf16*)d_A, (const bf16*)h_W_list[i % n_w], c->ws.logits, M, N, K, TC_STORE_F32, N));
+      else
+        RPO_TRY(tc_gemm_launch(c, (const bf16*)d_A, (const bf16*)h_W_list[i % n_w], c->ws.logits, M, N, K, TC_STORE_F32, N,
+                               true, &splits));
     }
     return RPO_OK;
   };
@@ -1064,7 +1071,8 @@ extern "C" int rpo_set_option(rpo_ctx* c, const char* name, int32_t value) {
   else if (!strcmp(name, "use_pdl")) c->use_pdl = value;
   else if (!strcmp(name, "use_tc5_attention")) c->use_tc5_attention = value;
   else if (!strcmp(name, "tc5_v_variant")) c->tc5_v_variant = value;
-  else if (!strcmp(name, "gemm_bn")) { if (value != 0 && value != 32 && value != 64 && value != 96 && value != 128 && value != 256) return RPO_ERR_INVALID_ARG; c->gemm_bn = value; }
+  else if (!strcmp(name, "use_gemm_pairs")) c->use_gemm_pairs = value;
+  else if (!strcmp(name, "gemm_bn")) { if (value != 0 && value != 32 && value != 64 && value != 96 && value != 128 && value != 256 && value != 512) return RPO_ERR_INVALID_ARG; c->gemm_bn = value; }
   else if (!strcmp(name, "gemm_splits")) c->gemm_splits = value;
   else if (!strcmp(name, "profile")) c->profile = value;
   else return RPO_ERR_INVALID_ARG;

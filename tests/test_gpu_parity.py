@@ -291,12 +291,16 @@ def test_tensor_core_gemm_against_numpy():
             w = em.round_bf16((rng.standard_normal((N, K)) * 0.05).astype(np.float32))
             dA = torch.from_numpy(a).to(DEV).to(torch.bfloat16); dW = torch.from_numpy(w).to(DEV).to(torch.bfloat16)
             dC = torch.full((M, N), 777.0, dtype=torch.float32, device=DEV)
-            ctx.gemm(dA, dW, dC, impl=2)
-            torch.cuda.synchronize()
-            assert ctx.device_status() == 0
             ref = a.astype(np.float64) @ w.astype(np.float64).T
-            err = np.max(np.abs(dC.cpu().numpy() - ref))
-            assert err < 2e-5 * K ** 0.5, (M, N, K, err)
+            for bn in (0, 512):                      # the planner's kernel, then 256 x 256 tiles on CTA pairs
+                ctx.set_option("gemm_bn", bn)
+                dC.fill_(777.0)
+                ctx.gemm(dA, dW, dC, impl=2)
+                torch.cuda.synchronize()
+                assert ctx.device_status() == 0
+                err = np.max(np.abs(dC.cpu().numpy() - ref))
+                assert err < 2e-5 * K ** 0.5, (M, N, K, bn, err)
+            ctx.set_option("gemm_bn", 0)
         with pytest.raises(rpo.RpoError):
             ctx.gemm(torch.zeros((8, 72), dtype=torch.bfloat16, device=DEV), torch.zeros((16, 72), dtype=torch.bfloat16, device=DEV),
                      torch.zeros((8, 16), dtype=torch.float32, device=DEV), impl=2)      # K % 64 != 0
@@ -326,7 +330,7 @@ def test_tensor_core_gemm_full_size_every_tile_width_and_split(M, N, K):
     dA = torch.randn((M, K), device=DEV, generator=gen).to(torch.bfloat16)
     dW = (torch.randn((N, K), device=DEV, generator=gen) * 0.05).to(torch.bfloat16)
     with make_ctx(shape, 1, 1, 32, 4) as ctx:
-        for bn, splits in [(0, 0), (256, 1), (128, 1), (96, 1), (64, 1), (32, 1), (128, 4), (64, 3), (256, 2)]:
+        for bn, splits in [(0, 0), (512, 1), (256, 1), (128, 1), (96, 1), (64, 1), (32, 1), (128, 4), (64, 3), (256, 2)]:   # 512 = CTA-pair tiles
             ctx.set_option("gemm_bn", bn); ctx.set_option("gemm_splits", splits)
             dC = torch.full((M, N), 777.0, dtype=torch.float32, device=DEV)
             ctx.gemm(dA, dW, dC, impl=2)
