@@ -134,7 +134,9 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 
 // Epilogue of one 32-column chunk of an accumulator row: r[0..31] are the float32 bit patterns of
 // columns col .. col+31 of output row `row`.
-template <int EPI>
+// STREAM: the output is far larger than L2 and not read again by this kernel; streaming stores
+// keep it from evicting the operand tiles other CTAs are about to fetch.
+template <int EPI, bool STREAM = false>
 __device__ __forceinline__ void tc_store_chunk(const TcParams& p, const uint32_t* r, int row, int col, int split) {
   if (row >= p.M || col >= p.N) return;
   const int ncol = min(32, p.N - col);       // multiple of 8 (N % 8 == 0)
@@ -147,7 +149,7 @@ __device__ __forceinline__ void tc_store_chunk(const TcParams& p, const uint32_t
       __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]));
       __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
       v.x = *(uint32_t*)&h0; v.y = *(uint32_t*)&h1; v.z = *(uint32_t*)&h2; v.w = *(uint32_t*)&h3;
-      *(uint4*)(dst + j) = v;
+      if (STREAM) __stcs((uint4*)(dst + j), v); else *(uint4*)(dst + j) = v;
     }
   } else if (EPI == TC_SWIGLU) {
     // columns (2j, 2j+1) = (gate_j, up_j)  ->  out[row, col/2 + j]
@@ -161,7 +163,8 @@ __device__ __forceinline__ void tc_store_chunk(const TcParams& p, const uint32_t
         __nv_bfloat162 h = __floats2bfloat162_rn(g0 / (1.0f + __expf(-g0)) * u0, g1 / (1.0f + __expf(-g1)) * u1);
         o[q] = *(uint32_t*)&h;
       }
-      *(uint4*)(dst + j / 2) = make_uint4(o[0], o[1], o[2], o[3]);
+      if (STREAM) __stcs((uint4*)(dst + j / 2), make_uint4(o[0], o[1], o[2], o[3]));
+      else *(uint4*)(dst + j / 2) = make_uint4(o[0], o[1], o[2], o[3]);
     }
   } else {
     float* dst = (EPI == TC_PARTIAL) ? (float*)p.C + split * p.split_stride + (int64_t)row * p.ldc + col
@@ -173,7 +176,7 @@ __device__ __forceinline__ void tc_store_chunk(const TcParams& p, const uint32_t
         const float4 o = *(float4*)(dst + j);
         v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
       }
-      *(float4*)(dst + j) = v;
+      if (STREAM) __stcs((float4*)(dst + j), v); else *(float4*)(dst + j) = v;
     }
   }
 }

@@ -70,6 +70,18 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t* bar, uint16_t cta_mas
 
 }  // namespace tc
 
+// Tile order: bands of TC2_BAND row tiles, walked column by column, so the clusters working at
+// the same time share a few A slabs and a few W slabs (both stay hot in L2) instead of one A slab
+// and the whole weight matrix.
+constexpr int TC2_BAND = 8;
+__device__ __forceinline__ void tc2_tile(int it, int tiles_m, int tiles_n, int& tm, int& tn) {
+  const int per_band = TC2_BAND * tiles_n;
+  const int band = it / per_band, r = it - band * per_band;
+  const int h = min(TC2_BAND, tiles_m - band * TC2_BAND);
+  tn = r / h;
+  tm = band * TC2_BAND + (r - tn * h);
+}
+
 // 192 threads per CTA, clusters of two: warp 0 = TMA producer, warp 1 = tensor-memory owner (and,
 // in the leader, MMA issuer), warps 2..5 = epilogue.  p.tiles_m / p.tiles_n count 256 x 256 tiles.
 template <int EPI>
@@ -118,7 +130,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
       for (int it = cluster_id; it < n_items && ok; it += n_clusters) {
-        const int tn = it % p.tiles_n, tm = it / p.tiles_n;
+        int tm, tn;
+        tc2_tile(it, p.tiles_m, p.tiles_n, tm, tn);
         const int row_a = tm * 256 + (int)rank * 128, row_w = tn * 256 + (int)rank * 128;
         for (int kb = 0; kb < p.kb_total; ++kb) {
           if (!tc::mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
@@ -171,7 +184,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
     for (int it = cluster_id; it < n_items && ok; it += n_clusters) {
-      const int tn = it % p.tiles_n, tm = it / p.tiles_n;
+      int tm, tn;
+      tc2_tile(it, p.tiles_m, p.tiles_n, tm, tn);
       if (!tc::mbar_wait(&acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc::tmem_fence_after();
       const int row = tm * 256 + (int)rank * 128 + quad * 32 + lane;
@@ -180,7 +194,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       for (int c0 = 0; c0 < 256; c0 += 32) {
         uint32_t r[32];
         tc::tmem_ld32(t_row + (uint32_t)c0, r);
-        tc_store_chunk<EPI>(p, r, row, tn * 256 + c0, 0);
+        tc_store_chunk<EPI, true>(p, r, row, tn * 256 + c0, 0);
       }
       tc::tmem_fence_before();
       __syncwarp();
