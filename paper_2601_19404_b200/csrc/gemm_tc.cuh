@@ -136,8 +136,9 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 // columns col .. col+31 of output row `row`.
 // STREAM: the output is far larger than L2 and not read again by this kernel; streaming stores
 // keep it from evicting the operand tiles other CTAs are about to fetch.
-template <int EPI, bool STREAM = false>
-__device__ __forceinline__ void tc_store_chunk(const TcParams& p, const uint32_t* r, int row, int col, int split) {
+template <int EPI>
+__device__ __forceinline__ void tc_store_chunk(const TcParams& p, const uint32_t* r, int row, int col, int split,
+                                               const bool STREAM = false) {
   if (row >= p.M || col >= p.N) return;
   const int ncol = min(32, p.N - col);       // multiple of 8 (N % 8 == 0)
   if (EPI == TC_STORE_BF16) {

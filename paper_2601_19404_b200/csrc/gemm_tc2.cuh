@@ -126,14 +126,32 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     if (lane == 0) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
-      pdl_wait();
-      int stage = 0; uint32_t phase = 0;
+      // The weights do not depend on the kernel running before this one: the W halves of the first
+      // tile go into the (still empty) ring before the wait for the predecessor, the A halves after.
+      int pre = 0;
+      if (cluster_id < n_items) {
+        int tm, tn;
+        tc2_tile(cluster_id, p.tiles_m, p.tiles_n, tm, tn);
+        pre = min(TC2_NS, p.kb_total);
+        for (int i = 0; i < pre; ++i) {
+          if (leader) tc::mbar_expect_tx(&full[i], 2 * TC2_STAGE_BYTES);
+          tc::tma_load_2d_pair(smem + i * TC2_STAGE_BYTES + TC2_HALF_BYTES, &map_w, i * TC_BK, tn * 256 + (int)rank * 128,
+                               tc::map_to_rank(tc::smem_u32(&full[i]), 0));
+        }
+        pdl_wait();
+        for (int i = 0; i < pre; ++i)
+          tc::tma_load_2d_pair(smem + i * TC2_STAGE_BYTES, &map_a, i * TC_BK, tm * 256 + (int)rank * 128,
+                               tc::map_to_rank(tc::smem_u32(&full[i]), 0));
+      } else {
+        pdl_wait();
+      }
+      int stage = pre % TC2_NS; uint32_t phase = (pre == TC2_NS) ? 1u : 0u;
       bool ok = true;
       for (int it = cluster_id; it < n_items && ok; it += n_clusters) {
         int tm, tn;
         tc2_tile(it, p.tiles_m, p.tiles_n, tm, tn);
         const int row_a = tm * 256 + (int)rank * 128, row_w = tn * 256 + (int)rank * 128;
-        for (int kb = 0; kb < p.kb_total; ++kb) {
+        for (int kb = (it == cluster_id ? pre : 0); kb < p.kb_total; ++kb) {
           if (!tc::mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
           uint8_t* sa = smem + stage * TC2_STAGE_BYTES;
           if (leader) tc::mbar_expect_tx(&full[stage], 2 * TC2_STAGE_BYTES);
@@ -180,6 +198,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
     const int quad = warp & 3;
+    const bool stream_out = p.M >= 2048;           // output far larger than L2: streaming stores
     pdl_wait();
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
@@ -194,7 +213,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       for (int c0 = 0; c0 < 256; c0 += 32) {
         uint32_t r[32];
         tc::tmem_ld32(t_row + (uint32_t)c0, r);
-        tc_store_chunk<EPI, true>(p, r, row, tn * 256 + c0, 0);
+        tc_store_chunk<EPI>(p, r, row, tn * 256 + c0, 0, stream_out);
       }
       tc::tmem_fence_before();
       __syncwarp();
@@ -247,12 +266,14 @@ inline int tc2_launch(rpo_ctx* c, const CUtensorMap* ma, const CUtensorMap* mw, 
   return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI>, *ma, *mw, p) == cudaSuccess ? RPO_OK : RPO_ERR_CUDA;
 }
 
-// True when the pass is large enough for pair tiles to fill the machine.
+// True when the pass is large enough for pair tiles to fill the machine: prefill and log-prob passes,
+// and decode batches of more than 128 sequences against wide matrices (gate/up, lm_head), where a
+// pair streams each weight tile once for 256 rows instead of once per 128-row tile.
 inline bool tc2_wanted(rpo_ctx* c, int M, int N) {
   if (c->gemm_bn > 0) return c->gemm_bn == 512;           // test / sweep override: 512 = pair tiles
   if (!c->use_gemm_pairs) return false;
   const int tiles = ((M + 255) / 256) * ((N + 255) / 256);
-  return M >= 1024 && tiles >= c->sm_count / 2;
+  return M > 128 && tiles >= c->sm_count / 2;             // more than one 128-row tile, a tile for every CTA pair
 }
 
 inline int tc2_gemm_launch(rpo_ctx* c, const bf16* A, const bf16* W, void* C, int M, int N, int K, int epi, int ldc) {

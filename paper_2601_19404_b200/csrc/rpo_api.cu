@@ -775,7 +775,7 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
                                  (uint64_t)a.top_p24, (uint64_t)temp_bits,
                                  (uint64_t)a.greedy, (uint64_t)(uint32_t)a.eos_id, a.seed,
                                  (uint64_t)c->use_tcgen05, (uint64_t)c->use_tc_attention, (uint64_t)c->use_pdl,
-                                 (uint64_t)c->gemm_bn, (uint64_t)c->gemm_splits};
+                                 (uint64_t)c->gemm_bn, (uint64_t)c->gemm_splits, (uint64_t)c->use_gemm_pairs};
     rpo_ctx::StepGraph* sg = nullptr;
     for (auto& g : c->step_graphs) if (g.key == key) sg = &g;
     if (!sg) {
