@@ -101,7 +101,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   const uint32_t rank = tc::cluster_ctarank();
   const bool leader = (rank == 0);
   const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
-  const int n_items = p.tiles_m * p.tiles_n;
+  const int n_items = p.tiles_m * p.tiles_n * p.splits;    // work item = (tile, k-split), split fastest
   pdl_launch_dependents();
 
   if (threadIdx.x == 0) {
@@ -131,16 +131,17 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       int pre = 0;
       if (cluster_id < n_items) {
         int tm, tn;
-        tc2_tile(cluster_id, p.tiles_m, p.tiles_n, tm, tn);
-        pre = min(TC2_NS, p.kb_total);
+        tc2_tile(cluster_id / p.splits, p.tiles_m, p.tiles_n, tm, tn);
+        const int kb0 = (cluster_id % p.splits) * p.kb_per_split, kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+        pre = min(TC2_NS, kb1 - kb0);
         for (int i = 0; i < pre; ++i) {
           if (leader) tc::mbar_expect_tx(&full[i], 2 * TC2_STAGE_BYTES);
-          tc::tma_load_2d_pair(smem + i * TC2_STAGE_BYTES + TC2_HALF_BYTES, &map_w, i * TC_BK, tn * 256 + (int)rank * 128,
+          tc::tma_load_2d_pair(smem + i * TC2_STAGE_BYTES + TC2_HALF_BYTES, &map_w, (kb0 + i) * TC_BK, tn * 256 + (int)rank * 128,
                                tc::map_to_rank(tc::smem_u32(&full[i]), 0));
         }
         pdl_wait();
         for (int i = 0; i < pre; ++i)
-          tc::tma_load_2d_pair(smem + i * TC2_STAGE_BYTES, &map_a, i * TC_BK, tm * 256 + (int)rank * 128,
+          tc::tma_load_2d_pair(smem + i * TC2_STAGE_BYTES, &map_a, (kb0 + i) * TC_BK, tm * 256 + (int)rank * 128,
                                tc::map_to_rank(tc::smem_u32(&full[i]), 0));
       } else {
         pdl_wait();
@@ -149,9 +150,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       bool ok = true;
       for (int it = cluster_id; it < n_items && ok; it += n_clusters) {
         int tm, tn;
-        tc2_tile(it, p.tiles_m, p.tiles_n, tm, tn);
+        tc2_tile(it / p.splits, p.tiles_m, p.tiles_n, tm, tn);
+        const int kb0 = (it % p.splits) * p.kb_per_split, kb1 = min(p.kb_total, kb0 + p.kb_per_split);
         const int row_a = tm * 256 + (int)rank * 128, row_w = tn * 256 + (int)rank * 128;
-        for (int kb = (it == cluster_id ? pre : 0); kb < p.kb_total; ++kb) {
+        for (int kb = kb0 + (it == cluster_id ? pre : 0); kb < kb1; ++kb) {
           if (!tc::mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
           uint8_t* sa = smem + stage * TC2_STAGE_BYTES;
           if (leader) tc::mbar_expect_tx(&full[stage], 2 * TC2_STAGE_BYTES);
@@ -179,14 +181,15 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (!tc::mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag)) { ok = false; break; }
         tc::tmem_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * 256);
-        for (int kb = 0; kb < p.kb_total; ++kb) {
+        const int kb0 = (it % p.splits) * p.kb_per_split, kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!tc::mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
           tc::tmem_fence_after();
           const uint32_t sa = tc::smem_u32(smem + stage * TC2_STAGE_BYTES);
           const uint64_t da = tc::umma_desc_sw128(sa), db = tc::umma_desc_sw128(sa + TC2_HALF_BYTES);
 #pragma unroll
           for (int k = 0; k < TC_BK / 16; ++k)
-            tc::umma_bf16_pair(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            tc::umma_bf16_pair(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb > kb0 || k > 0) ? 1u : 0u);
           tc::umma_commit_pair(&empty[stage], 3);       // frees the stage in both CTAs
           if (++stage == TC2_NS) { stage = 0; phase ^= 1; }
         }
@@ -204,7 +207,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     bool ok = true;
     for (int it = cluster_id; it < n_items && ok; it += n_clusters) {
       int tm, tn;
-      tc2_tile(it, p.tiles_m, p.tiles_n, tm, tn);
+      tc2_tile(it / p.splits, p.tiles_m, p.tiles_n, tm, tn);
       if (!tc::mbar_wait(&acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc::tmem_fence_after();
       const int row = tm * 256 + (int)rank * 128 + quad * 32 + lane;
@@ -213,7 +216,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       for (int c0 = 0; c0 < 256; c0 += 32) {
         uint32_t r[32];
         tc::tmem_ld32(t_row + (uint32_t)c0, r);
-        tc_store_chunk<EPI>(p, r, row, tn * 256 + c0, 0, stream_out);
+        tc_store_chunk<EPI>(p, r, row, tn * 256 + c0, it % p.splits, stream_out);
       }
       tc::tmem_fence_before();
       __syncwarp();
@@ -260,27 +263,49 @@ inline int tc2_launch(rpo_ctx* c, const CUtensorMap* ma, const CUtensorMap* mw, 
     if (cudaOccupancyMaxActiveClusters(&n, gemm_tc2_kernel<EPI>, &cfg) != cudaSuccess || n < 1) { cudaGetLastError(); n = c->sm_count / 2; }
     max_clusters = std::min(n, c->sm_count / 2);
   }
-  const int clusters = std::min(p.tiles_m * p.tiles_n, max_clusters);
+  const int clusters = std::min(p.tiles_m * p.tiles_n * p.splits, max_clusters);
   cfg.gridDim = dim3(2 * clusters);
   cfg.numAttrs = c->use_pdl ? 2 : 1;
   return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI>, *ma, *mw, p) == cudaSuccess ? RPO_OK : RPO_ERR_CUDA;
 }
 
-// True when the pass is large enough for pair tiles to fill the machine: prefill and log-prob passes,
-// and decode batches of more than 128 sequences against wide matrices (gate/up, lm_head), where a
-// pair streams each weight tile once for 256 rows instead of once per 128-row tile.
-inline bool tc2_wanted(rpo_ctx* c, int M, int N) {
-  if (c->gemm_bn > 0) return c->gemm_bn == 512;           // test / sweep override: 512 = pair tiles
-  if (!c->use_gemm_pairs) return false;
-  const int tiles = ((M + 255) / 256) * ((N + 255) / 256);
-  return M > 128 && tiles >= c->sm_count / 2;             // more than one 128-row tile, a tile for every CTA pair
+// Split-K factor of the pair kernel for a pass of few tiles: as many k-splits as give every CTA pair
+// one work item in a single round, each at least eight k-blocks deep, within the partial workspace.
+inline int tc2_splits(rpo_ctx* c, int M, int N, int K, bool allow_split) {
+  const int tiles = ((M + 255) / 256) * ((N + 255) / 256), pairs = c->sm_count / 2, kb_total = K / TC_BK;
+  if (c->gemm_bn == 512 && c->gemm_splits > 0) return allow_split ? std::max(1, std::min(c->gemm_splits, kb_total)) : 1;
+  if (!allow_split || tiles >= pairs) return 1;
+  int sp = std::max(1, std::min(pairs / tiles, kb_total / 8));
+  while (sp > 1 && (size_t)sp * M * N > c->ws.partial_elems) --sp;
+  return sp;
 }
 
-inline int tc2_gemm_launch(rpo_ctx* c, const bf16* A, const bf16* W, void* C, int M, int N, int K, int epi, int ldc) {
+// True when pair tiles fill the machine: prefill and log-prob passes, and decode batches of more
+// than 128 sequences, where a pair streams each weight tile once for 256 rows instead of once per
+// 128-row tile; narrow matrices are split along K to give every pair an item.
+inline bool tc2_wanted(rpo_ctx* c, int M, int N, int K, bool allow_split) {
+  if (c->gemm_bn > 0) return c->gemm_bn == 512;           // test / sweep override: 512 = pair tiles
+  if (!c->use_gemm_pairs || M <= 128) return false;
+  const int tiles = ((M + 255) / 256) * ((N + 255) / 256), sp = tc2_splits(c, M, N, K, allow_split);
+  if (sp > 1 && K / TC_BK / sp < 32) return false;       // shallow splits: measured no better than single-CTA tiles
+  return tiles * sp >= c->sm_count / 2 - 10;
+}
+
+// With allow_split the launch may leave split-K partial planes [splits][M][N] in ws.partial
+// instead of applying `epi`; *splits_out then holds the number of planes (> 1).
+inline int tc2_gemm_launch(rpo_ctx* c, const bf16* A, const bf16* W, void* C, int M, int N, int K, int epi, int ldc,
+                           bool allow_split, int* splits_out) {
+  if (splits_out) *splits_out = 0;
   TcParams p;
   p.C = C; p.M = M; p.N = N; p.K = K; p.ldc = ldc;
-  p.tiles_m = (M + 255) / 256; p.tiles_n = (N + 255) / 256; p.splits = 1; p.kb_total = K / TC_BK; p.kb_per_split = p.kb_total;
-  p.split_stride = 0; p.status = c->d_status;
+  p.tiles_m = (M + 255) / 256; p.tiles_n = (N + 255) / 256; p.kb_total = K / TC_BK;
+  int splits = tc2_splits(c, M, N, K, allow_split);
+  p.kb_per_split = (p.kb_total + splits - 1) / splits;
+  splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
+  if (splits > 1 && (size_t)splits * M * N > c->ws.partial_elems) { splits = 1; p.kb_per_split = p.kb_total; }
+  p.splits = splits;
+  p.split_stride = (int64_t)M * N; p.status = c->d_status;
+  if (splits > 1) { epi = TC_PARTIAL; p.C = c->ws.partial; p.ldc = N; if (splits_out) *splits_out = splits; }
   const CUtensorMap* ma = tc_map(c, A, M, K, 128);
   const CUtensorMap* mw = tc_map(c, W, N, K, 128);
   if (!ma || !mw) return RPO_ERR_CUDA;
@@ -289,7 +314,7 @@ inline int tc2_gemm_launch(rpo_ctx* c, const bf16* A, const bf16* W, void* C, in
     case TC_STORE_F32: return tc2_launch<TC_STORE_F32>(c, ma, mw, p);
     case TC_ADD_F32: return tc2_launch<TC_ADD_F32>(c, ma, mw, p);
     case TC_SWIGLU: return tc2_launch<TC_SWIGLU>(c, ma, mw, p);
-    default: return RPO_ERR_INVALID_ARG;
+    default: return tc2_launch<TC_PARTIAL>(c, ma, mw, p);
   }
 }
 

@@ -387,10 +387,10 @@ static int gemm(rpo_ctx* c, const T* A, const T* W, void* C, int M, int N, int K
     int splits = 0;
     prof_begin(c);
     const int ldc = tc_epi == TC_SWIGLU ? N / 2 : N;
-    const int rc = tc2_wanted(c, M, N)
-                       ? tc2_gemm_launch(c, (const bf16*)A, (const bf16*)W, C, M, N, K, tc_epi, ldc)
-                       : tc_gemm_launch(c, (const bf16*)A, (const bf16*)W, C, M, N, K, tc_epi, ldc,
-                                        allow_split && (epi == EPI_ADD_F32 || splits_out), &splits);
+    const bool may_split = allow_split && (epi == EPI_ADD_F32 || splits_out);
+    const int rc = tc2_wanted(c, M, N, K, may_split)
+                       ? tc2_gemm_launch(c, (const bf16*)A, (const bf16*)W, C, M, N, K, tc_epi, ldc, may_split, &splits)
+                       : tc_gemm_launch(c, (const bf16*)A, (const bf16*)W, C, M, N, K, tc_epi, ldc, may_split, &splits);
     prof_end(c);
     c->launches++;
     if (rc == RPO_OK && splits > 1) {
@@ -1014,8 +1014,9 @@ extern "C" int rpo_gemm_bench(rpo_ctx* c, int32_t M, int32_t N, int32_t K, const
   auto enqueue = [&]() -> int {
     for (int i = 0; i < iters; ++i) {
       int splits = 0;
-      if (tc2_wanted(c, M, N))
-        RPO_TRY(tc2_gemm_launch(c, (const bf16*)d_A, (const bf16*)h_W_list[i % n_w], c->ws.logits, M, N, K, TC_STORE_F32, N));
+      if (tc2_wanted(c, M, N, K, true))
+        RPO_TRY(tc2_gemm_launch(c, (const bf16*)d_A, (const bf16*)h_W_list[i % n_w], c->ws.logits, M, N, K, TC_STORE_F32, N,
+                                true, &splits));
       else
         RPO_TRY(tc_gemm_launch(c, (const bf16*)d_A, (const bf16*)h_W_list[i % n_w], c->ws.logits, M, N, K, TC_STORE_F32, N,
                                true, &splits));
