@@ -735,8 +735,22 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
     for (int g = 0; g < n_groups; ++g) max_p = std::max(max_p, groups[g].prefix_len);
     const int rep = c->shape.n_q_heads / c->shape.n_kv_heads;
     const int pairs = n_groups * c->shape.n_kv_heads * ceil_div(G * rep, FA_BM);
-    const int want = std::max(1, std::min(32, ceil_div(2 * c->sm_count, pairs)));
-    c->attn_split_chunk = std::max(FA_BN, ceil_div(ceil_div(max_p, want), FA_BN) * FA_BN);
+    // Prefix split: the chunk (a multiple of the key tile) that minimises rounds x (keys per CTA +
+    // a fixed per-CTA cost of ~160 keys' worth of set-up and tail), with two CTAs resident per SM;
+    // CTAs whose chunk lies beyond a short prefix carry suffix tiles only and are not counted.
+    const int slots = 2 * c->sm_count, per_group = pairs / std::max(n_groups, 1);
+    double best_cost = 1e30;
+    int best_chunk = std::max(FA_BN, ceil_div(max_p, FA_BN) * FA_BN);
+    for (int want = 1; want <= 32; ++want) {
+      const int chunk = std::max(FA_BN, ceil_div(ceil_div(max_p, want), FA_BN) * FA_BN);
+      int64_t ctas = 0;
+      for (int g = 0; g < n_groups; ++g) ctas += (int64_t)per_group * ceil_div(std::max(groups[g].prefix_len, 1), chunk);
+      const double cost = (double)ceil_div((int)ctas, slots) * (chunk + 160.0);
+      if (cost < best_cost - 1e-9) { best_cost = cost; best_chunk = chunk; }
+    }
+    c->attn_split_chunk = best_chunk;
+    c->attn_splits = std::min(32, ceil_div(max_p, c->attn_split_chunk));
+    if (ceil_div(max_p, c->attn_split_chunk) > 32) c->attn_split_chunk = std::max(FA_BN, ceil_div(ceil_div(max_p, 32), FA_BN) * FA_BN);
     c->attn_splits = ceil_div(max_p, c->attn_split_chunk);
     c->attn_mode = 1; c->attn_G = G; c->attn_groups = n_groups;
   }
