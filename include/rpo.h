@@ -196,7 +196,9 @@ int rpo_release_groups(rpo_ctx* ctx, int32_t n_groups, const rpo_group* h_groups
  * copies the prefix tokens to the device, prefills, decodes, optionally computes the
  * teacher-forced log-probs (want_policy_logprobs != 0 -> h_policy_logprobs_out), copies
  * the results back, releases the groups and synchronises the stream.
- * h_tokens_out [B*max_new], h_lens_out [B], h_logprobs_out [B*max_new] or NULL. */
+ * h_tokens_out [B*max_new], h_lens_out [B], h_logprobs_out [B*max_new] or NULL.
+ * The device staging buffers belong to the context: allocated on the first call, grown
+ * when a later call needs more, freed by rpo_destroy. */
 int rpo_rollout_host(rpo_ctx* ctx, int32_t n_groups, const int32_t* h_tokens, const int32_t* h_offsets,
                      const int32_t* h_group_ids, int32_t G, int32_t max_new, const rpo_sampler* sampler,
                      int32_t* h_tokens_out, int32_t* h_lens_out, float* h_logprobs_out,

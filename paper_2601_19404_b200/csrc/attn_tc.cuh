@@ -67,6 +67,26 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
   return *(uint32_t*)&h;
 }
+// Thread-block cluster: barrier over all threads of all CTAs, and loads from a peer CTA's shared memory.
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_rank(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void ld_cluster_f32x2(uint32_t addr, float& x, float& y) {
+  asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(x), "=f"(y) : "r"(addr) : "memory");
+}
+template <int N> __device__ __forceinline__ void ld_cluster_f32(uint32_t addr, float* v);
+template <> __device__ __forceinline__ void ld_cluster_f32<4>(uint32_t addr, float* v) {
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]) : "r"(addr) : "memory");
+}
+template <> __device__ __forceinline__ void ld_cluster_f32<2>(uint32_t addr, float* v) {
+  asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v[0]), "=f"(v[1]) : "r"(addr) : "memory");
+}
 }  // namespace fa
 
 // Tile shape per mode: 64-key tiles, four consumer warps of 16 query rows each (+ the producer warp),
@@ -84,10 +104,16 @@ template <int MODE> struct FaCfg {
   template <int DH> static constexpr int smem_bytes() { return (FA_BM + (NSK + NSV) * BN) * DH * 2 + 1024 /*align*/ + 128 /*barriers*/; }
 };
 
-template <int DH, int MODE>
+// CLM (SHARED only): the CTAs of the splits of one work item form a thread-block cluster
+// (cluster rank = split) and merge their partials through distributed shared memory instead of
+// global memory and a second kernel; a.n_splits is then the cluster size (1, 2, 4 or 8).
+template <int DH, int MODE, bool CLM = false>
 __global__ void __launch_bounds__(FaCfg<MODE>::THREADS + 32, FaCfg<MODE>::MIN_CTAS)
 flash_attn_kernel(FlashArgs a) {
   pdl_prologue();
+  constexpr bool CL = CLM && MODE == FA_SHARED;
+  static_assert(!(CLM && FaCfg<MODE>::KS != 1), "the in-cluster merge expects one warp set");
+  constexpr int XO_STRIDE = DH + 8;          // floats per row of the partial O kept in shared memory (bank-conflict-free)
   constexpr int NSK = FaCfg<MODE>::NSK, NSV = FaCfg<MODE>::NSV;
   constexpr int BN = FaCfg<MODE>::BN;
   constexpr int KS = FaCfg<MODE>::KS, THREADS = FaCfg<MODE>::THREADS, WBN = BN / KS;   // WBN: keys of a tile per warp
@@ -289,9 +315,10 @@ flash_attn_kernel(FlashArgs a) {
       }
       blk_prev_v = blk_k;
     }
-    return;                                     // the consumers use named barrier 1 from here on
+    if (!CL) return;                            // the consumers use named barrier 1 from here on
   }
 
+  if (warp < NW) {
   float o[ONT][4];
 #pragma unroll
   for (int i = 0; i < ONT; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
@@ -450,6 +477,22 @@ flash_attn_kernel(FlashArgs a) {
   l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1); l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
 
   // ---- write
+  if (CL) {
+    // partial (m, l, O) of this split into the K/V ring (every consumer warp is done with it)
+    float* xo = reinterpret_cast<float*>(fsm);
+    float* xml = xo + FA_BM * XO_STRIDE;
+    asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory");
+    if (ok) {
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const int r = half ? r_hi : r_lo;
+        if (tq == 0) { xml[r * 2] = half ? m_hi : m_lo; xml[r * 2 + 1] = half ? l_hi : l_lo; }
+#pragma unroll
+        for (int i = 0; i < ONT; ++i)
+          *(float2*)(xo + r * XO_STRIDE + i * 8 + tq * 2) = make_float2(o[i][half * 2], o[i][half * 2 + 1]);
+      }
+    }
+  } else {
 #pragma unroll
   for (int half = 0; half < 2; ++half) {
     const int r = half ? r_hi : r_lo;
@@ -469,6 +512,42 @@ flash_attn_kernel(FlashArgs a) {
 #pragma unroll
       for (int i = 0; i < ONT; ++i) *(float2*)(dst + i * 8 + tq * 2) = make_float2(o[i][half * 2], o[i][half * 2 + 1]);
     }
+  }
+  }
+  }   // consumer warps
+
+  if (CL) {
+    // Log-sum-exp merge of the cluster's partials: the CTA of rank k owns rows k, k + n_splits, ..;
+    // a warp per row, lane s reads (m, l) of split s, every lane DH/32 output dimensions of each
+    // split in fixed order (reproducible).  All threads of all CTAs take part in both barriers.
+    constexpr int DPL = DH / 32;
+    fa::cluster_sync();
+    if (warp < NW) {
+      const uint32_t xo_addr = (uint32_t)__cvta_generic_to_shared(fsm), xml_addr = xo_addr + FA_BM * XO_STRIDE * 4;
+      for (int r = split + a.n_splits * warp; r < n_rows; r += a.n_splits * NW) {
+        float ms = -INFINITY, ls = 0.f;
+        if (lane < a.n_splits) fa::ld_cluster_f32x2(fa::map_rank(xml_addr + r * 8, lane), ms, ls);
+        if (!(ls > 0.f)) ms = -INFINITY;
+        const float m_new = warp_max(ms);
+        const float wgt = (ls > 0.f) ? exp2f(ms - m_new) : 0.f;
+        const float l_tot = warp_sum(ls * wgt);
+        float acc[DPL];
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
+        for (int k = 0; k < a.n_splits; ++k) {
+          const float c = __shfl_sync(0xffffffffu, wgt, k);
+          float v[DPL];
+          fa::ld_cluster_f32<DPL>(fa::map_rank(xo_addr + (r * XO_STRIDE + lane * DPL) * 4, k), v);
+#pragma unroll
+          for (int i = 0; i < DPL; ++i) acc[i] += (c != 0.f) ? c * v[i] : 0.f;
+        }
+        const float inv = (l_tot > 0.f) ? 1.0f / l_tot : 0.f;
+        bf16* dst = a.out + (int64_t)s_qrow[r] * a.out_cols + s_head[r] * DH + lane * DPL;
+#pragma unroll
+        for (int i = 0; i < DPL; i += 2) *(uint32_t*)(dst + i) = fa::pack_bf16(acc[i] * inv, acc[i + 1] * inv);
+      }
+    }
+    fa::cluster_sync();                       // no CTA leaves while a peer may still read its partial
   }
 }
 

@@ -88,11 +88,18 @@ struct rpo_ctx {
   // options
   int use_tcgen05 = 1, use_tc_attention = 1, use_graph = 1;
   int use_tc5_attention = 1, tc5_v_variant = 0;   // tcgen05 prefill attention (and the descriptor reading under test)
+  int use_cluster_merge = 0;          // decode attention: splits of a work item merge inside a thread-block cluster
+                                      // (measured slower than partials + merge kernel at 8 splits: off by default)
+  int launch_cluster_x = 0;           // cluster width of the next launch (0: none); cleared by the launch
   int use_pdl = 1;                    // programmatic dependent launch between the library's kernels
   int use_gemm_pairs = 1;             // 256 x 256 tiles on CTA pairs (cta_group::2) for many-row GEMMs
   int gemm_bn = 0, gemm_splits = 0;   // > 0: override the GEMM planner (tests, sweeps); 512 = pair tiles
   // attention plan of the pass being enqueued: 0 = row tiles (prefill / teacher), 1 = decode
   int attn_mode = 0, attn_tiles = 0, attn_G = 1, attn_groups = 0, attn_splits = 1, attn_split_chunk = 64;
+  // device staging of rpo_rollout_host: kept between calls (stable addresses let the decode step's
+  // CUDA graph be reused), grown on demand, freed with the context
+  void* host_stage[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+  size_t host_stage_bytes[5] = {0, 0, 0, 0, 0};
   int pending_splits = 0, pending_rows = 0;   // split-K partials of ws.x not yet reduced
   // optional per-kernel timing: event pairs around every launch, tagged class + 16*phase
   struct ProfEvent { cudaEvent_t a, b; int tag; const char* label; };

@@ -67,10 +67,20 @@ template <typename... KArgs, typename... Args>
 static cudaError_t launch_kernel(rpo_ctx* c, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr; cfg.numAttrs = c->use_pdl ? 1 : 0;
+  cudaLaunchAttribute attr[2];
+  int n_attr = 0;
+  if (c->use_pdl) {
+    attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+    ++n_attr;
+  }
+  if (c->launch_cluster_x > 1) {                     // thread-block clusters along x, requested for this launch only
+    attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+    attr[n_attr].val.clusterDim.x = c->launch_cluster_x; attr[n_attr].val.clusterDim.y = 1; attr[n_attr].val.clusterDim.z = 1;
+    ++n_attr;
+  }
+  c->launch_cluster_x = 0;
+  cfg.attrs = attr; cfg.numAttrs = n_attr;
   return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
 
@@ -155,6 +165,7 @@ extern "C" int rpo_destroy(rpo_ctx* ctx) {
   ctx->step_graphs.clear();
   tc_destroy(ctx);
   for (void* p : ctx->allocations) cudaFree(p);
+  for (void* p : ctx->host_stage) if (p) cudaFree(p);
   if (ctx->own_stream) cudaStreamDestroy(ctx->stream);
   delete ctx;
   return RPO_OK;
@@ -427,17 +438,21 @@ static int rmsnorm(rpo_ctx* c, float* x, const float* g, T* h, int rows) {
   return RPO_OK;
 }
 
-template <int DH, int MODE>
+template <int DH, int MODE, bool CLM = false>
 static int launch_flash(rpo_ctx* c, const FlashArgs& a, dim3 grid) {
   constexpr int smem = FaCfg<MODE>::template smem_bytes<DH>();
   static bool attr_done = false;
   if (!attr_done) {
-    CUDA_TRY(cudaFuncSetAttribute(flash_attn_kernel<DH, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    CUDA_TRY(cudaFuncSetAttribute(flash_attn_kernel<DH, MODE, CLM>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     attr_done = true;
   }
-  LAUNCH(c, (flash_attn_kernel<DH, MODE>), grid, FaCfg<MODE>::THREADS + 32, smem, a);
+  if (CLM) c->launch_cluster_x = a.n_splits;         // the splits of a work item are consecutive along x
+  LAUNCH(c, (flash_attn_kernel<DH, MODE, CLM>), grid, FaCfg<MODE>::THREADS + 32, smem, a);
   return RPO_OK;
 }
+
+// Split counts whose CTAs can merge inside a cluster (portable cluster sizes).
+static bool cluster_mergeable(int n_splits) { return n_splits == 1 || n_splits == 2 || n_splits == 4 || n_splits == 8; }
 
 // The tcgen05 attention serves prefill / teacher-forced passes of bf16 models with head_dim 128.
 static bool tc5_attention(rpo_ctx* c) {
@@ -484,6 +499,8 @@ static int attention(rpo_ctx* c, int layer, int rows) {
       }
       const int rep = s.n_q_heads / s.n_kv_heads;
       dim3 grid(c->attn_groups * ceil_div(c->attn_G * rep, FA_BM) * c->attn_splits, s.n_kv_heads);
+      if (c->use_cluster_merge && cluster_mergeable(a.n_splits))
+        return s.head_dim == 128 ? launch_flash<128, FA_SHARED, true>(c, a, grid) : launch_flash<64, FA_SHARED, true>(c, a, grid);
       RPO_TRY((s.head_dim == 128 ? launch_flash<128, FA_SHARED>(c, a, grid) : launch_flash<64, FA_SHARED>(c, a, grid)));
       const int mgrid = ceil_div((int64_t)rows * s.n_q_heads, 4);
       if (s.head_dim == 128)
@@ -739,15 +756,18 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
     // a fixed per-CTA cost of ~160 keys' worth of set-up and tail), with two CTAs resident per SM;
     // CTAs whose chunk lies beyond a short prefix carry suffix tiles only and are not counted.
     const int slots = 2 * c->sm_count, per_group = pairs / std::max(n_groups, 1);
-    double best_cost = 1e30;
-    int best_chunk = std::max(FA_BN, ceil_div(max_p, FA_BN) * FA_BN);
+    double best_cost = 1e30, best_cl_cost = 1e30;
+    int best_chunk = std::max(FA_BN, ceil_div(max_p, FA_BN) * FA_BN), best_cl_chunk = best_chunk;
     for (int want = 1; want <= 32; ++want) {
       const int chunk = std::max(FA_BN, ceil_div(ceil_div(max_p, want), FA_BN) * FA_BN);
       int64_t ctas = 0;
       for (int g = 0; g < n_groups; ++g) ctas += (int64_t)per_group * ceil_div(std::max(groups[g].prefix_len, 1), chunk);
       const double cost = (double)ceil_div((int)ctas, slots) * (chunk + 160.0);
       if (cost < best_cost - 1e-9) { best_cost = cost; best_chunk = chunk; }
+      if (cluster_mergeable(ceil_div(max_p, chunk)) && cost < best_cl_cost - 1e-9) { best_cl_cost = cost; best_cl_chunk = chunk; }
     }
+    // split counts that merge inside a cluster save the merge kernel: preferred unless clearly costlier
+    if (c->use_cluster_merge && best_cl_cost <= 1.1 * best_cost) best_chunk = best_cl_chunk;
     c->attn_split_chunk = best_chunk;
     c->attn_splits = std::min(32, ceil_div(max_p, c->attn_split_chunk));
     if (ceil_div(max_p, c->attn_split_chunk) > 32) c->attn_split_chunk = std::max(FA_BN, ceil_div(ceil_div(max_p, 32), FA_BN) * FA_BN);
@@ -789,7 +809,7 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
                                  (uint64_t)a.top_p24, (uint64_t)temp_bits,
                                  (uint64_t)a.greedy, (uint64_t)(uint32_t)a.eos_id, a.seed,
                                  (uint64_t)c->use_tcgen05, (uint64_t)c->use_tc_attention, (uint64_t)c->use_pdl,
-                                 (uint64_t)c->gemm_bn, (uint64_t)c->gemm_splits, (uint64_t)c->use_gemm_pairs};
+                                 (uint64_t)c->gemm_bn, (uint64_t)c->gemm_splits, (uint64_t)c->use_gemm_pairs, (uint64_t)c->use_cluster_merge};
     rpo_ctx::StepGraph* sg = nullptr;
     for (auto& g : c->step_graphs) if (g.key == key) sg = &g;
     if (!sg) {
@@ -961,10 +981,21 @@ extern "C" int rpo_rollout_host(rpo_ctx* c, int32_t n_groups, const int32_t* h_t
   std::vector<rpo_group> groups(n_groups);
   int rc = RPO_OK;
   bool prefilled = false;
+  auto stage = [&](int slot, size_t bytes) -> void* {      // persistent device buffer of at least `bytes`
+    if (c->host_stage_bytes[slot] < bytes) {
+      cudaStreamSynchronize(c->stream);
+      if (c->host_stage[slot]) cudaFree(c->host_stage[slot]);
+      c->host_stage[slot] = nullptr; c->host_stage_bytes[slot] = 0;
+      if (cudaMalloc(&c->host_stage[slot], bytes) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+      c->host_stage_bytes[slot] = bytes;
+    }
+    return c->host_stage[slot];
+  };
   do {
-    if (cudaMalloc(&d_tok, std::max<size_t>(n_tok, 1) * 4) != cudaSuccess || cudaMalloc(&d_out, BS * 4) != cudaSuccess ||
-        cudaMalloc(&d_lens, B * 4) != cudaSuccess || cudaMalloc(&d_lp, BS * 4) != cudaSuccess ||
-        (want_policy && cudaMalloc(&d_pol, BS * 4) != cudaSuccess)) { rc = RPO_ERR_CUDA; break; }
+    d_tok = (int32_t*)stage(0, std::max<size_t>(n_tok, 1) * 4); d_out = (int32_t*)stage(1, BS * 4);
+    d_lens = (int32_t*)stage(2, B * 4); d_lp = (float*)stage(3, BS * 4);
+    if (want_policy) d_pol = (float*)stage(4, BS * 4);
+    if (!d_tok || !d_out || !d_lens || !d_lp || (want_policy && !d_pol)) { rc = RPO_ERR_CUDA; break; }
     if (cudaMemcpyAsync(d_tok, h_tokens, n_tok * 4, cudaMemcpyHostToDevice, c->stream) != cudaSuccess) { rc = RPO_ERR_CUDA; break; }
     if ((rc = rpo_prefill_prefix(c, n_groups, d_tok, h_offsets, h_group_ids, groups.data())) != RPO_OK) break;
     prefilled = true;
@@ -980,7 +1011,6 @@ extern "C" int rpo_rollout_host(rpo_ctx* c, int32_t n_groups, const int32_t* h_t
   } while (0);
   if (rc != RPO_OK) { cudaStreamSynchronize(c->stream); cudaGetLastError(); }
   if (prefilled) rpo_release_groups(c, n_groups, groups.data());
-  cudaFree(d_tok); cudaFree(d_out); cudaFree(d_lens); cudaFree(d_lp); cudaFree(d_pol);
   return rc;
 }
 
@@ -1087,6 +1117,7 @@ extern "C" int rpo_set_option(rpo_ctx* c, const char* name, int32_t value) {
   else if (!strcmp(name, "use_tc5_attention")) c->use_tc5_attention = value;
   else if (!strcmp(name, "tc5_v_variant")) c->tc5_v_variant = value;
   else if (!strcmp(name, "use_gemm_pairs")) c->use_gemm_pairs = value;
+  else if (!strcmp(name, "use_cluster_merge")) c->use_cluster_merge = value;
   else if (!strcmp(name, "gemm_bn")) { if (value != 0 && value != 32 && value != 64 && value != 96 && value != 128 && value != 256 && value != 512) return RPO_ERR_INVALID_ARG; c->gemm_bn = value; }
   else if (!strcmp(name, "gemm_splits")) c->gemm_splits = value;
   else if (!strcmp(name, "profile")) c->profile = value;

@@ -57,3 +57,25 @@ def test_bf16_small_decoder_parity(name, fast):
             ref = rollout.token_logprobs(w, sh, toks[off[g]:off[g + 1]], t[g * G:(g + 1) * G], l[g * G:(g + 1) * G])
             assert np.max(np.abs(out.cpu().numpy()[g * G:(g + 1) * G] - ref)) <= 2e-2
         assert ctx.device_status() == 0
+
+
+@pytest.mark.parametrize("name", list(SHAPES))
+def test_in_cluster_merge_equals_merge_kernel(name):
+    """Decode attention: merging the prefix splits inside a thread-block cluster (distributed shared
+    memory) gives the same logits, bit for bit, as partials in global memory + the merge kernel;
+    ragged prefixes, so some splits of the short groups hold suffix tiles only or nothing."""
+    sh_d = SHAPES[name]
+    lens = np.array([200, 37, 129, 64], dtype=np.int32)
+    G, S = 4, 70                                    # suffixes longer than one key tile
+    forced = workloads.teacher_tokens(len(lens) * G, S, sh_d["vocab"], seed=9)
+    outs = []
+    for cl in (1, 0):
+        with make_ctx(sh_d, len(lens), G, int(lens.max()), S, chunk=256) as ctx:
+            ctx.set_option("use_cluster_merge", cl)
+            ctx.init_weights(0, 0.02)
+            toks, off = workloads.prefix_tokens(lens, sh_d["vocab"], seed=2)
+            groups = ctx.prefill_prefix(dev_i32(toks), off)
+            t, l, lp, dbg = run_decode(ctx, groups, G, S, rpo.Sampler(1.0, 0.95, False, -1, 0), forced=forced, want_logits=True)
+            assert ctx.device_status() == 0
+            outs.append((dbg, lp))
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
