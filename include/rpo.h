@@ -265,7 +265,9 @@ int rpo_counters(rpo_ctx* ctx, int64_t* kernel_launches, int64_t* free_kv_blocks
  * "use_graph" (CUDA graph per decode step, default 1), "use_pdl" (programmatic dependent launch
  * between the library's kernels, default 1), "use_tc5_attention" (tcgen05 attention for
  * many-row passes at head_dim 128, default 1), "use_gemm_pairs" (256 x 256 GEMM tiles on CTA
- * pairs for many-row passes, default 1), "profile" (see rpo_profile_read),
+ * pairs for passes of more than 128 rows, default 1), "use_cluster_merge" (decode attention:
+ * the prefix splits of a work item form a thread-block cluster and merge through distributed
+ * shared memory instead of a second kernel; default 0), "profile" (see rpo_profile_read),
  * "gemm_bn" (0 = planner, else force the tensor-core tile width: 32/64/96/128/256, or 512 for
  * the CTA-pair kernel) and "gemm_splits" (with gemm_bn: force the split-K factor where the
  * caller can reduce planes). */
