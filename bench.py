@@ -344,9 +344,11 @@ def main():
         if gemm_n:
             per_launch_bytes = ab["weights"] * (S - 1) / gemm_n
             achieved = per_launch_bytes / (gemm_ms / gemm_n * 1e-3) / 1e9
-            roofline = {"bound": "hbm", "kernel": "gemm_tc_kernel (decode weight GEMMs)", "achieved": achieved,
+            esz = 2 if shape["dtype"] == "bf16" else 4
+            roofline = {"bound": "hbm", "kernel": "gemm_tc_kernel / gemm_tc2_kernel (decode weight GEMMs)", "achieved": achieved,
                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                        "traffic": ncu_traffic_per_launch() if not reduced else None,
+                        "traffic": ncu_traffic_per_launch() if (not reduced and args.config.startswith("cfg2")) else None,
+                        "tensor_tflops": 2.0 * B * (ab["weights"] / esz) * (S - 1) / (gemm_ms * 1e-3) / 1e12,
                         "algorithmic_bytes_per_launch": per_launch_bytes, "launches_per_step": gemm_n / max(S - 1, 1),
                         "peak_source": peaks["source"] + " copy bandwidth (MEASURED_PEAKS.json)" if peaks["source"] == "measured" else "fallback",
                         "ms_per_launch": gemm_ms / gemm_n}

@@ -172,8 +172,8 @@ flash_attn_kernel(FlashArgs a) {
     }
   };
   if (MODE == FA_ROWS) {
-    const int2 tile = a.tiles[blockIdx.x];
-    const int head = blockIdx.y;
+    const int2 tile = a.tiles[blockIdx.y];        // grid (heads, tiles), tile list ordered heaviest first
+    const int head = blockIdx.x;
     kvh = head / rep; n_rows = tile.y;
     sd = a.seqs[a.row_seq[tile.x]];
     if (tid < FA_BM) {

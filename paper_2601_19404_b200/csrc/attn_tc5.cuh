@@ -71,8 +71,10 @@ flash_attn_tc5_kernel(const __grid_constant__ CUtensorMap q_map, Flash5Args a) {
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int2 tile = a.tiles[blockIdx.x];
-  const int head = blockIdx.y, kvh = head / (a.hq / a.hkv);
+  // grid (heads, tiles): the heads of one row tile run together (the query heads of a KV head
+  // share its K/V in L2), and the tile list is ordered heaviest first
+  const int2 tile = a.tiles[blockIdx.y];
+  const int head = blockIdx.x, kvh = head / (a.hq / a.hkv);
   const int row0 = tile.x, n_rows = tile.y;
   const SeqDesc sd = a.seqs[a.row_seq[row0]];
 

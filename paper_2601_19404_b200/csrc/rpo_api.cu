@@ -490,11 +490,11 @@ static int attention(rpo_ctx* c, int layer, int rows) {
           CUDA_TRY(cudaFuncSetAttribute(flash_attn_tc5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, T5_SMEM));
           attr_done = true;
         }
-        LAUNCH(c, flash_attn_tc5_kernel, dim3(c->attn_tiles, s.n_q_heads), 320, T5_SMEM, *qm, f);
+        LAUNCH(c, flash_attn_tc5_kernel, dim3(s.n_q_heads, c->attn_tiles), 320, T5_SMEM, *qm, f);
         return RPO_OK;
       }
       if (c->attn_mode == 0) {
-        dim3 grid(c->attn_tiles, s.n_q_heads);
+        dim3 grid(s.n_q_heads, c->attn_tiles);
         return s.head_dim == 128 ? launch_flash<128, FA_ROWS>(c, a, grid) : launch_flash<64, FA_ROWS>(c, a, grid);
       }
       const int rep = s.n_q_heads / s.n_kv_heads;
@@ -525,13 +525,19 @@ static int attention(rpo_ctx* c, int layer, int rows) {
 // Query-row tiles (128 rows for the tcgen05 attention, else 64) of a pass whose sequences own
 // consecutive row ranges.
 static int upload_row_tiles(rpo_ctx* c, const std::vector<int>& rows_per_seq) {
-  std::vector<int2> tiles;
+  // Tiles deeper into a sequence see more keys (causal attention): heaviest first, so the launch
+  // does not end on a few long tiles.
+  std::vector<std::pair<int, int2>> weighted;
   const int bm = tc5_attention(c) ? T5_BM : FA_BM;
   int r = 0;
   for (int n : rows_per_seq) {
-    for (int r0 = 0; r0 < n; r0 += bm) tiles.push_back(make_int2(r + r0, std::min(bm, n - r0)));
+    for (int r0 = 0; r0 < n; r0 += bm) weighted.push_back({r0 + std::min(bm, n - r0), make_int2(r + r0, std::min(bm, n - r0))});
     r += n;
   }
+  std::stable_sort(weighted.begin(), weighted.end(), [](const std::pair<int, int2>& a, const std::pair<int, int2>& b) { return a.first > b.first; });
+  std::vector<int2> tiles;
+  tiles.reserve(weighted.size());
+  for (const auto& t : weighted) tiles.push_back(t.second);
   c->attn_mode = 0; c->attn_tiles = (int)tiles.size();
   if (!tiles.empty())
     CUDA_TRY(cudaMemcpyAsync(c->ws.tiles, tiles.data(), tiles.size() * sizeof(int2), cudaMemcpyHostToDevice, c->stream));

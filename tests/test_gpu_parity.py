@@ -277,6 +277,16 @@ def test_rollout_host_matches_device_calls():
         assert np.array_equal(ht, t) and np.array_equal(hl, l) and np.array_equal(hp, lp)
         assert np.max(np.abs(hq - hp)) < 1e-4
         assert ctx.counters()[1] == ctx.limits.kv_pool_blocks
+        # the context keeps its device staging between calls: a smaller call, then the first one again
+        # (same addresses, so the decode step's graph is reused), give the same answers
+        t2, off2 = toks[:off[2]], off[:3]
+        h2 = np.zeros((2 * G, S), dtype=np.int32); l2 = np.zeros(2 * G, dtype=np.int32); p2 = np.zeros((2 * G, S), dtype=np.float32)
+        ctx.rollout_host(t2, off2, G, S, smp, h2, l2, p2, None)
+        assert np.array_equal(h2, t[:2 * G]) and np.array_equal(l2, l[:2 * G]) and np.array_equal(p2, lp[:2 * G])
+        ht[:] = 0; hp[:] = 0
+        ctx.rollout_host(toks, off, G, S, smp, ht, hl, hp, hq)
+        assert np.array_equal(ht, t) and np.array_equal(hp, lp)
+        assert ctx.counters()[1] == ctx.limits.kv_pool_blocks and ctx.device_status() == 0
 
 
 def test_tensor_core_gemm_against_numpy():
