@@ -546,8 +546,9 @@ static int upload_row_tiles(rpo_ctx* c, const std::vector<int>& rows_per_seq) {
 
 // The layer stack over `rows` rows of ws.x, whose (sequence, private index) metadata sits in
 // ws.row_seq / ws.row_t and whose sequence descriptors sit in ws.seqs.
+// flush = false leaves the last layer's split-K partials pending for the caller's next RMSNorm on ws.x.
 template <typename T>
-static int run_layers(rpo_ctx* c, int rows) {
+static int run_layers(rpo_ctx* c, int rows, bool flush = true) {
   const rpo_shape& s = c->shape;
   Workspace& w = c->ws;
   const int d = s.d_model, F = s.d_ffn, qo = s.n_q_heads * s.head_dim;
@@ -572,7 +573,7 @@ static int run_layers(rpo_ctx* c, int rows) {
     }
     RPO_TRY(gemm<T>(c, (const T*)w.act, (const T*)L.wd, w.x, rows, d, F, EPI_ADD_F32, 0, true));
   }
-  return flush_partials(c);
+  return flush ? flush_partials(c) : RPO_OK;
 }
 
 // logits[n, V] (float32, ws.logits) from n residual rows in ws.xh.
@@ -799,9 +800,11 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
   auto enqueue_step = [&]() -> int {
     LAUNCH(c, embed_kernel<T>, B, 128, 0, (const int32_t*)w.cur_tok, (const T*)c->embed, w.x, B, d, c->shape.vocab,
            c->d_status, w.step_ctr);
-    RPO_TRY(run_layers<T>(c, B));
-    CUDA_TRY(cudaMemcpyAsync(w.xh, w.x, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, st));
-    RPO_TRY(head<T>(c, B));
+    // every row is a sequence's last row: the final RMSNorm reads ws.x directly and folds the last
+    // layer's split-K partials in (no separate reduction, no copy of the residual rows)
+    RPO_TRY(run_layers<T>(c, B, false));
+    RPO_TRY(rmsnorm<T>(c, w.x, c->gf, (T*)w.hh, B));
+    RPO_TRY(gemm<T>(c, (const T*)w.hh, (const T*)c->lm_head, w.logits, B, c->shape.vocab, d, EPI_STORE_F32));
     RPO_TRY(launch_sampler(c, B, a));
     return RPO_OK;
   };
