@@ -1,0 +1,95 @@
+"""Initialisation of the experience cache: one full-path response per question (Section 3.1,
+Eq. 1; the paper generates them once, before training, spread over its GPUs), with continuous
+batching on top of the rollout library.
+
+Full responses end at very different lengths, so a fixed batch would idle on its longest member.
+Here generation proceeds in *waves* of `wave_tokens` tokens: after every wave the sequences that
+emitted EOS (or reached `max_len`) leave the batch and waiting questions take their slots.  A
+sequence that continues is re-prefilled from its prompt plus what it has generated so far - per
+token, prefill costs two orders of magnitude less than decode, so re-reading a sequence once per
+wave adds a few percent - which keeps the library's interface unchanged: every wave is
+`rpo_prefill_prefix` + `rpo_decode_suffix` with one sample per group.
+
+Determinism: wave w of request r samples from the random stream of group id r * MAX_WAVES + w,
+so a response depends only on (seed, request index, wave size), never on which other requests
+shared its batches.
+"""
+import collections
+
+import numpy as np
+
+MAX_WAVES = 1 << 12
+
+
+def schedule(prompts, engine, max_batch, wave_tokens, max_len, eos_id):
+    """Continuous batching over `engine`.
+
+    prompts: list of int32 arrays (request r = prompts[r]).
+    engine(prefixes, group_ids, max_new) -> (tokens [n, max_new] int32, lens [n] int32): generates
+        up to max_new tokens after each prefix; lens counts tokens up to and including EOS.
+    Returns (responses, stats): responses[r] = generated tokens of request r (ends with eos_id if the
+    model stopped by itself), stats = dict(waves=..., slot_tokens=..., useful_tokens=...)."""
+    if max_batch <= 0 or wave_tokens <= 0 or max_len <= 0:
+        raise ValueError("max_batch, wave_tokens and max_len must be positive")
+    if -(-max_len // wave_tokens) > MAX_WAVES:
+        raise ValueError("too many waves per request")
+    waiting = collections.deque(range(len(prompts)))
+    active = []                                              # request indices, in admission order
+    gen = [np.zeros(0, dtype=np.int32) for _ in prompts]
+    wave_of = [0] * len(prompts)
+    stats = dict(waves=0, slot_tokens=0, useful_tokens=0)
+    while waiting or active:
+        while waiting and len(active) < max_batch:
+            active.append(waiting.popleft())
+        order = sorted(active)                               # batch layout independent of admission history
+        prefixes = [np.concatenate([np.asarray(prompts[r], dtype=np.int32), gen[r]]) for r in order]
+        ids = np.asarray([r * MAX_WAVES + wave_of[r] for r in order], dtype=np.int32)
+        toks, lens = engine(prefixes, ids, wave_tokens)
+        stats["waves"] += 1
+        stats["slot_tokens"] += len(order) * wave_tokens
+        still = []
+        for k, r in enumerate(order):
+            room = max_len - gen[r].size
+            n = int(min(int(lens[k]), room))
+            new = np.asarray(toks[k][:n], dtype=np.int32)
+            gen[r] = np.concatenate([gen[r], new])
+            wave_of[r] += 1
+            stats["useful_tokens"] += n
+            stopped = n > 0 and eos_id >= 0 and new[-1] == eos_id
+            if not stopped and gen[r].size < max_len:
+                still.append(r)
+        keep = set(still)
+        active = [r for r in active if r in keep]
+    return gen, stats
+
+
+def library_engine(ctx, sampler):
+    """engine for schedule(): one group per sequence (G = 1) through ctx (a Context)."""
+    import torch
+    dev = torch.device("cuda", torch.cuda.current_device())
+
+    def engine(prefixes, group_ids, max_new):
+        n = len(prefixes)
+        off = np.zeros(n + 1, dtype=np.int32)
+        off[1:] = np.cumsum([p.size for p in prefixes])
+        toks = np.concatenate(prefixes).astype(np.int32)
+        d_out = torch.zeros((n, max_new), dtype=torch.int32, device=dev)
+        d_len = torch.zeros(n, dtype=torch.int32, device=dev)
+        groups = ctx.prefill_prefix(torch.from_numpy(toks).to(dev), off, group_ids)
+        ctx.decode_suffix(groups, 1, max_new, sampler, d_out, d_len)
+        ctx.release_groups(groups)
+        torch.cuda.synchronize()
+        return d_out.cpu().numpy(), d_len.cpu().numpy()
+
+    return engine
+
+
+def initialise_cache(cache, ctx, sampler, questions, max_batch, wave_tokens, max_len):
+    """Fills `cache` (an ExperienceCache) with one sampled response per question.
+    questions: dict qid -> prompt tokens.  Returns the scheduler's statistics."""
+    qids = sorted(questions)
+    responses, stats = schedule([questions[q] for q in qids], library_engine(ctx, sampler), max_batch, wave_tokens,
+                                max_len, sampler.eos_id)
+    for q, a in zip(qids, responses):
+        cache.put(q, questions[q], a)
+    return stats
