@@ -1,4 +1,5 @@
-// bf16 GEMM for many-row passes (prefill, token log-probs) on CTA pairs: C[M,N] = A[M,K] * W[N,K]^T.
+// bf16 GEMM on CTA pairs for passes of more than 128 rows (prefill, token log-probs, decode batches
+// above 128 sequences): C[M,N] = A[M,K] * W[N,K]^T.
 //
 // A 128 x 256 tile per CTA needs 48 KB of operands per 64-wide k-block, and the path from L2 into
 // shared memory, not the tensor pipe, then sets the pace.  Here two CTAs of a cluster share one
@@ -15,8 +16,13 @@
 //   * each CTA drains its own 128 accumulator rows (two buffers of 256 columns = all 512 columns
 //     of tensor memory, so the epilogue of one tile overlaps the main loop of the next) and tells
 //     the leader when a buffer is free again (remote mbarrier arrive).
-//   * persistent: cluster i walks tiles i, i + n_clusters, ...; every wait is bounded as in
+//   * persistent: cluster i walks work items i, i + n_clusters, ... (an item is a tile, or a
+//     k-split of a tile when a deep, narrow matrix has fewer tiles than the machine has pairs);
+//     tiles are ordered in bands of row tiles for L2 locality; every wait is bounded as in
 //     gemm_tc.cuh; no CTA leaves before its peer (cluster barrier at the end).
+//   * in a decode batch of 256 rows a pair streams every weight tile once for all rows, where
+//     single-CTA tiles stream it once per 128-row tile; the W halves of a CTA's first item are
+//     requested before the wait on the preceding kernel, as in gemm_tc.cuh.
 #pragma once
 #include "gemm_tc.cuh"
 
