@@ -179,6 +179,7 @@ def main():
     ap.add_argument("--config", default="cfg2_1p5b_16x8")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-profile", action="store_true")
+    ap.add_argument("--chunk", type=int, default=0, help="prefill chunk in tokens (0: 16384, or the longest prefix if longer)")
     ap.add_argument("--ref-prefix", type=int, default=1024)
     ap.add_argument("--ref-suffix", type=int, default=8)
     ap.add_argument("--options", default="", help="comma list name=value passed to rpo_set_option")
@@ -226,7 +227,7 @@ def main():
     want_lp = bool(cfg.get("logprobs"))
 
     blocks = int(np.sum(-(-lens // 16))) + B * (-(-S // 16)) + 64
-    chunk = int(min(max(int(lens.max()), 16384), 32768))
+    chunk = args.chunk if args.chunk > 0 else int(min(max(int(lens.max()), 16384), 32768))
     stream = torch.cuda.Stream(device=dev)
     ctx = rpo.Context(binding.shape_from_dict(shape), blocks, max_groups=n_g, max_seqs=B, max_chunk_tokens=chunk,
                       max_positions=int(lens.max()) + S + 1, stream=stream)
