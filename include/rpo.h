@@ -268,8 +268,8 @@ int rpo_counters(rpo_ctx* ctx, int64_t* kernel_launches, int64_t* free_kv_blocks
  * pairs for passes of more than 128 rows, default 1), "use_cluster_merge" (decode attention:
  * the prefix splits of a work item form a thread-block cluster and merge through distributed
  * shared memory instead of a second kernel; default 0), "profile" (see rpo_profile_read),
- * "gemm_bn" (0 = planner, else force the tensor-core tile width: 32/64/96/128/256, or 512 for
- * the CTA-pair kernel) and "gemm_splits" (with gemm_bn: force the split-K factor where the
+ * "gemm_bn" (0 = planner, else force the tensor-core tile width: 32/64/96/128/256, or 512 / 384
+ * for the CTA-pair kernel with 128 / 64 rows per CTA) and "gemm_splits" (with gemm_bn: force the split-K factor where the
  * caller can reduce planes). */
 int rpo_set_option(rpo_ctx* ctx, const char* name, int32_t value);
 

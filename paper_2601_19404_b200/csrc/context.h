@@ -93,7 +93,8 @@ struct rpo_ctx {
   int launch_cluster_x = 0;           // cluster width of the next launch (0: none); cleared by the launch
   int use_pdl = 1;                    // programmatic dependent launch between the library's kernels
   int use_gemm_pairs = 1;             // 256 x 256 tiles on CTA pairs (cta_group::2) for many-row GEMMs
-  int gemm_bn = 0, gemm_splits = 0;   // > 0: override the GEMM planner (tests, sweeps); 512 = pair tiles
+  int use_gemm_pairs_small = 1;       // pair tiles with 64 rows per CTA for wide matrices at up to 128 rows
+  int gemm_bn = 0, gemm_splits = 0;   // > 0: override the GEMM planner (tests, sweeps); 384 / 512 = pair tiles with 64 / 128 rows per CTA
   // attention plan of the pass being enqueued: 0 = row tiles (prefill / teacher), 1 = decode
   int attn_mode = 0, attn_tiles = 0, attn_G = 1, attn_groups = 0, attn_splits = 1, attn_split_chunk = 64;
   // device staging of rpo_rollout_host: kept between calls (stable addresses let the decode step's

@@ -28,10 +28,19 @@
 
 namespace rpo {
 
-constexpr int TC2_NS = 6;
-constexpr int TC2_HALF_BYTES = 128 * TC_BK * 2;          // 16 KB: 128 rows x 64 bf16
-constexpr int TC2_STAGE_BYTES = 2 * TC2_HALF_BYTES;      // A half + W half
-constexpr int TC2_SMEM_BYTES = TC2_NS * TC2_STAGE_BYTES + 1024 + 256;
+// RM = rows of the A tile per CTA: 128 (256 x 256 tiles) or 64 (128 x 256 tiles, for batches of at
+// most 128 rows: the CTA then loads 8 KB of A per 16 KB of W, so more of the bytes it can keep in
+// flight are weight bytes).  With 64 rows per CTA the accumulator of a CTA sits in all 128 lanes of
+// tensor memory, lanes 0..63 holding columns 0..127 of its rows and lanes 64..127 columns 128..255.
+template <int RM>
+struct Tc2Cfg {
+  static constexpr int A_BYTES = RM * TC_BK * 2;           // 16 KB or 8 KB
+  static constexpr int W_BYTES = 128 * TC_BK * 2;          // 16 KB: 128 rows x 64 bf16
+  static constexpr int STAGE_BYTES = A_BYTES + W_BYTES;
+  static constexpr int NS = 192 * 1024 / STAGE_BYTES;      // 6 or 8
+  static constexpr int ACC_COLS = RM == 128 ? 256 : 128;   // tensor-memory columns of one accumulator buffer
+  static constexpr int SMEM_BYTES = NS * STAGE_BYTES + 1024 + 256;
+};
 
 namespace tc {
 
@@ -90,9 +99,12 @@ __device__ __forceinline__ void tc2_tile(int it, int tiles_m, int tiles_n, int& 
 
 // 192 threads per CTA, clusters of two: warp 0 = TMA producer, warp 1 = tensor-memory owner (and,
 // in the leader, MMA issuer), warps 2..5 = epilogue.  p.tiles_m / p.tiles_n count 256 x 256 tiles.
-template <int EPI>
+template <int EPI, int RM = 128>
 __global__ void __launch_bounds__(192, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, TcParams p) {
+  using Cfg = Tc2Cfg<RM>;
+  constexpr int TC2_NS = Cfg::NS, TC2_STAGE_BYTES = Cfg::STAGE_BYTES, TC2_HALF_BYTES = Cfg::A_BYTES;   // W tile follows the A tile
+  constexpr int TM = 2 * RM;                     // rows of a pair tile
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint64_t* bars = (uint64_t*)(smem + TC2_NS * TC2_STAGE_BYTES);
@@ -118,7 +130,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc::smem_u32(tmem_slot)),
-                 "r"(512u) : "memory");
+                 "r"((uint32_t)(2 * Cfg::ACC_COLS)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   tc::tmem_fence_before();
@@ -147,7 +159,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         }
         pdl_wait();
         for (int i = 0; i < pre; ++i)
-          tc::tma_load_2d_pair(smem + i * TC2_STAGE_BYTES, &map_a, (kb0 + i) * TC_BK, tm * 256 + (int)rank * 128,
+          tc::tma_load_2d_pair(smem + i * TC2_STAGE_BYTES, &map_a, (kb0 + i) * TC_BK, tm * TM + (int)rank * RM,
                                tc::map_to_rank(tc::smem_u32(&full[i]), 0));
       } else {
         pdl_wait();
@@ -158,7 +170,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         int tm, tn;
         tc2_tile(it / p.splits, p.tiles_m, p.tiles_n, tm, tn);
         const int kb0 = (it % p.splits) * p.kb_per_split, kb1 = min(p.kb_total, kb0 + p.kb_per_split);
-        const int row_a = tm * 256 + (int)rank * 128, row_w = tn * 256 + (int)rank * 128;
+        const int row_a = tm * TM + (int)rank * RM, row_w = tn * 256 + (int)rank * 128;
         for (int kb = kb0 + (it == cluster_id ? pre : 0); kb < kb1; ++kb) {
           if (!tc::mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
           uint8_t* sa = smem + stage * TC2_STAGE_BYTES;
@@ -179,14 +191,14 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader only)
     if (leader && lane == 0) {
-      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
       bool ok = true;
       for (int it = cluster_id; it < n_items && ok; it += n_clusters) {
         if (!tc::mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag)) { ok = false; break; }
         tc::tmem_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * 256);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * Cfg::ACC_COLS);
         const int kb0 = (it % p.splits) * p.kb_per_split, kb1 = min(p.kb_total, kb0 + p.kb_per_split);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!tc::mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
@@ -216,13 +228,15 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       tc2_tile(it / p.splits, p.tiles_m, p.tiles_n, tm, tn);
       if (!tc::mbar_wait(&acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc::tmem_fence_after();
-      const int row = tm * 256 + (int)rank * 128 + quad * 32 + lane;
-      const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * 256);
+      // RM = 128: lane = row, 256 columns.  RM = 64: lanes 64.. hold columns 128..255 of rows 0..63.
+      const int row = tm * TM + (int)rank * RM + (RM == 128 ? quad * 32 : (quad & 1) * 32) + lane;
+      const int col_base = tn * 256 + (RM == 128 ? 0 : (quad >> 1) * 128);
+      const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * Cfg::ACC_COLS);
 #pragma unroll 1
-      for (int c0 = 0; c0 < 256; c0 += 32) {
+      for (int c0 = 0; c0 < Cfg::ACC_COLS; c0 += 32) {
         uint32_t r[32];
         tc::tmem_ld32(t_row + (uint32_t)c0, r);
-        tc_store_chunk<EPI>(p, r, row, tn * 256 + c0, it % p.splits, stream_out);
+        tc_store_chunk<EPI>(p, r, row, col_base + c0, it % p.splits, stream_out);
       }
       tc::tmem_fence_before();
       __syncwarp();
@@ -243,15 +257,16 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   tc::cluster_sync_all();                        // the peer no longer touches this CTA's barriers or tensor memory
   if (warp == 1) {
     tc::tmem_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)(2 * Cfg::ACC_COLS)) : "memory");
   }
 }
 
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
-template <int EPI>
+template <int EPI, int RM>
 inline int tc2_launch(rpo_ctx* c, const CUtensorMap* ma, const CUtensorMap* mw, const TcParams& p) {
+  using Cfg = Tc2Cfg<RM>;
   static int max_clusters = -1;
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[2];
@@ -259,40 +274,55 @@ inline int tc2_launch(rpo_ctx* c, const CUtensorMap* ma, const CUtensorMap* mw, 
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
-  cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = TC2_SMEM_BYTES; cfg.stream = c->stream;
+  cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = Cfg::SMEM_BYTES; cfg.stream = c->stream;
   cfg.attrs = attr;
   if (max_clusters < 0) {
-    if (cudaFuncSetAttribute(gemm_tc2_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC2_SMEM_BYTES) != cudaSuccess)
+    if (cudaFuncSetAttribute(gemm_tc2_kernel<EPI, RM>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
       return RPO_ERR_CUDA;
     cfg.gridDim = dim3(2 * (c->sm_count / 2)); cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_tc2_kernel<EPI>, &cfg) != cudaSuccess || n < 1) { cudaGetLastError(); n = c->sm_count / 2; }
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_tc2_kernel<EPI, RM>, &cfg) != cudaSuccess || n < 1) { cudaGetLastError(); n = c->sm_count / 2; }
     max_clusters = std::min(n, c->sm_count / 2);
   }
   const int clusters = std::min(p.tiles_m * p.tiles_n * p.splits, max_clusters);
   cfg.gridDim = dim3(2 * clusters);
   cfg.numAttrs = c->use_pdl ? 2 : 1;
-  return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI>, *ma, *mw, p) == cudaSuccess ? RPO_OK : RPO_ERR_CUDA;
+  return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI, RM>, *ma, *mw, p) == cudaSuccess ? RPO_OK : RPO_ERR_CUDA;
+}
+
+// Rows per CTA of the pair kernel for a pass of M rows: 64 (128-row pair tiles) up to 128 rows,
+// else 128 (256-row pair tiles).  gemm_bn = 384 / 512 force the one or the other (tests, sweeps).
+inline int tc2_rows(rpo_ctx* c, int M) {
+  if (c->gemm_bn == 384) return 64;
+  if (c->gemm_bn == 512) return 128;
+  return M <= 128 ? 64 : 128;
 }
 
 // Split-K factor of the pair kernel for a pass of few tiles: as many k-splits as give every CTA pair
 // one work item in a single round, each at least eight k-blocks deep, within the partial workspace.
 inline int tc2_splits(rpo_ctx* c, int M, int N, int K, bool allow_split) {
-  const int tiles = ((M + 255) / 256) * ((N + 255) / 256), pairs = c->sm_count / 2, kb_total = K / TC_BK;
-  if (c->gemm_bn == 512 && c->gemm_splits > 0) return allow_split ? std::max(1, std::min(c->gemm_splits, kb_total)) : 1;
+  const int tm = 2 * tc2_rows(c, M);
+  const int tiles = ((M + tm - 1) / tm) * ((N + 255) / 256), pairs = c->sm_count / 2, kb_total = K / TC_BK;
+  if (c->gemm_bn >= 384 && c->gemm_splits > 0) return allow_split ? std::max(1, std::min(c->gemm_splits, kb_total)) : 1;
   if (!allow_split || tiles >= pairs) return 1;
   int sp = std::max(1, std::min(pairs / tiles, kb_total / 8));
   while (sp > 1 && (size_t)sp * M * N > c->ws.partial_elems) --sp;
   return sp;
 }
 
-// True when pair tiles fill the machine: prefill and log-prob passes, and decode batches of more
-// than 128 sequences, where a pair streams each weight tile once for 256 rows instead of once per
-// 128-row tile; narrow matrices are split along K to give every pair an item.
+// True when pair tiles fill the machine.  More than 128 rows (prefill, log-prob passes, decode
+// batches above 128 sequences): a pair streams each weight tile once for 256 rows instead of once
+// per 128-row tile; deep narrow matrices are split along K to give every pair an item.  Up to 128
+// rows: 64 rows per CTA, for matrices wide enough for several rounds of tiles (lm_head) - a
+// weight-streaming launch runs as fast as it has weight bytes in flight, and a CTA that loads 8 KB
+// of activations per 16 KB of weights keeps a third more of them in flight; launches of a single
+// round lose more to the pair's start-up than they gain.
 inline bool tc2_wanted(rpo_ctx* c, int M, int N, int K, bool allow_split) {
-  if (c->gemm_bn > 0) return c->gemm_bn == 512;           // test / sweep override: 512 = pair tiles
-  if (!c->use_gemm_pairs || M <= 128) return false;
-  const int tiles = ((M + 255) / 256) * ((N + 255) / 256), sp = tc2_splits(c, M, N, K, allow_split);
+  if (c->gemm_bn > 0) return c->gemm_bn >= 384;           // test / sweep override: 384 / 512 = pair tiles
+  if (!c->use_gemm_pairs) return false;
+  const int tm = 2 * tc2_rows(c, M);
+  const int tiles = ((M + tm - 1) / tm) * ((N + 255) / 256), sp = tc2_splits(c, M, N, K, allow_split);
+  if (M <= 128) return c->use_gemm_pairs_small && M > 64 && tiles >= 3 * (c->sm_count / 2);   // several rounds: measured +6 % on lm_head, -10 % on one-round launches
   if (sp > 1 && K / TC_BK / sp < 32) return false;       // shallow splits: measured no better than single-CTA tiles
   return tiles * sp >= c->sm_count / 2 - 10;
 }
@@ -302,25 +332,35 @@ inline bool tc2_wanted(rpo_ctx* c, int M, int N, int K, bool allow_split) {
 inline int tc2_gemm_launch(rpo_ctx* c, const bf16* A, const bf16* W, void* C, int M, int N, int K, int epi, int ldc,
                            bool allow_split, int* splits_out) {
   if (splits_out) *splits_out = 0;
+  const int rm = tc2_rows(c, M), tm = 2 * rm;
   TcParams p;
   p.C = C; p.M = M; p.N = N; p.K = K; p.ldc = ldc;
-  p.tiles_m = (M + 255) / 256; p.tiles_n = (N + 255) / 256; p.kb_total = K / TC_BK;
-  int splits = tc2_splits(c, M, N, K, allow_split);
+  p.tiles_m = (M + tm - 1) / tm; p.tiles_n = (N + 255) / 256; p.kb_total = K / TC_BK;
+  int splits = (M <= 128 && c->gemm_bn == 0) ? 1 : tc2_splits(c, M, N, K, allow_split);
   p.kb_per_split = (p.kb_total + splits - 1) / splits;
   splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
   if (splits > 1 && (size_t)splits * M * N > c->ws.partial_elems) { splits = 1; p.kb_per_split = p.kb_total; }
   p.splits = splits;
   p.split_stride = (int64_t)M * N; p.status = c->d_status;
   if (splits > 1) { epi = TC_PARTIAL; p.C = c->ws.partial; p.ldc = N; if (splits_out) *splits_out = splits; }
-  const CUtensorMap* ma = tc_map(c, A, M, K, 128);
+  const CUtensorMap* ma = tc_map(c, A, M, K, rm);
   const CUtensorMap* mw = tc_map(c, W, N, K, 128);
   if (!ma || !mw) return RPO_ERR_CUDA;
+  if (rm == 64) {
+    switch (epi) {
+      case TC_STORE_BF16: return tc2_launch<TC_STORE_BF16, 64>(c, ma, mw, p);
+      case TC_STORE_F32: return tc2_launch<TC_STORE_F32, 64>(c, ma, mw, p);
+      case TC_ADD_F32: return tc2_launch<TC_ADD_F32, 64>(c, ma, mw, p);
+      case TC_SWIGLU: return tc2_launch<TC_SWIGLU, 64>(c, ma, mw, p);
+      default: return tc2_launch<TC_PARTIAL, 64>(c, ma, mw, p);
+    }
+  }
   switch (epi) {
-    case TC_STORE_BF16: return tc2_launch<TC_STORE_BF16>(c, ma, mw, p);
-    case TC_STORE_F32: return tc2_launch<TC_STORE_F32>(c, ma, mw, p);
-    case TC_ADD_F32: return tc2_launch<TC_ADD_F32>(c, ma, mw, p);
-    case TC_SWIGLU: return tc2_launch<TC_SWIGLU>(c, ma, mw, p);
-    default: return tc2_launch<TC_PARTIAL>(c, ma, mw, p);
+    case TC_STORE_BF16: return tc2_launch<TC_STORE_BF16, 128>(c, ma, mw, p);
+    case TC_STORE_F32: return tc2_launch<TC_STORE_F32, 128>(c, ma, mw, p);
+    case TC_ADD_F32: return tc2_launch<TC_ADD_F32, 128>(c, ma, mw, p);
+    case TC_SWIGLU: return tc2_launch<TC_SWIGLU, 128>(c, ma, mw, p);
+    default: return tc2_launch<TC_PARTIAL, 128>(c, ma, mw, p);
   }
 }
 

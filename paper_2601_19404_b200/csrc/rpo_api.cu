@@ -818,7 +818,7 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
                                  (uint64_t)a.top_p24, (uint64_t)temp_bits,
                                  (uint64_t)a.greedy, (uint64_t)(uint32_t)a.eos_id, a.seed,
                                  (uint64_t)c->use_tcgen05, (uint64_t)c->use_tc_attention, (uint64_t)c->use_pdl,
-                                 (uint64_t)c->gemm_bn, (uint64_t)c->gemm_splits, (uint64_t)c->use_gemm_pairs, (uint64_t)c->use_cluster_merge};
+                                 (uint64_t)c->gemm_bn, (uint64_t)c->gemm_splits, (uint64_t)c->use_gemm_pairs, (uint64_t)c->use_cluster_merge, (uint64_t)c->use_gemm_pairs_small};
     rpo_ctx::StepGraph* sg = nullptr;
     for (auto& g : c->step_graphs) if (g.key == key) sg = &g;
     if (!sg) {
@@ -1127,7 +1127,8 @@ extern "C" int rpo_set_option(rpo_ctx* c, const char* name, int32_t value) {
   else if (!strcmp(name, "tc5_v_variant")) c->tc5_v_variant = value;
   else if (!strcmp(name, "use_gemm_pairs")) c->use_gemm_pairs = value;
   else if (!strcmp(name, "use_cluster_merge")) c->use_cluster_merge = value;
-  else if (!strcmp(name, "gemm_bn")) { if (value != 0 && value != 32 && value != 64 && value != 96 && value != 128 && value != 256 && value != 512) return RPO_ERR_INVALID_ARG; c->gemm_bn = value; }
+  else if (!strcmp(name, "use_gemm_pairs_small")) c->use_gemm_pairs_small = value;
+  else if (!strcmp(name, "gemm_bn")) { if (value != 0 && value != 32 && value != 64 && value != 96 && value != 128 && value != 256 && value != 384 && value != 512) return RPO_ERR_INVALID_ARG; c->gemm_bn = value; }
   else if (!strcmp(name, "gemm_splits")) c->gemm_splits = value;
   else if (!strcmp(name, "profile")) c->profile = value;
   else return RPO_ERR_INVALID_ARG;

@@ -302,7 +302,7 @@ def test_tensor_core_gemm_against_numpy():
             dA = torch.from_numpy(a).to(DEV).to(torch.bfloat16); dW = torch.from_numpy(w).to(DEV).to(torch.bfloat16)
             dC = torch.full((M, N), 777.0, dtype=torch.float32, device=DEV)
             ref = a.astype(np.float64) @ w.astype(np.float64).T
-            for bn in (0, 512):                      # the planner's kernel, then 256 x 256 tiles on CTA pairs
+            for bn in (0, 512, 384):                 # the planner's kernel, then CTA-pair tiles of 256 and of 128 rows
                 ctx.set_option("gemm_bn", bn)
                 dC.fill_(777.0)
                 ctx.gemm(dA, dW, dC, impl=2)
@@ -340,7 +340,7 @@ def test_tensor_core_gemm_full_size_every_tile_width_and_split(M, N, K):
     dA = torch.randn((M, K), device=DEV, generator=gen).to(torch.bfloat16)
     dW = (torch.randn((N, K), device=DEV, generator=gen) * 0.05).to(torch.bfloat16)
     with make_ctx(shape, 1, 1, 32, 4) as ctx:
-        for bn, splits in [(0, 0), (512, 1), (512, 3), (256, 1), (128, 1), (96, 1), (64, 1), (32, 1), (128, 4), (64, 3), (256, 2)]:   # 512 = CTA-pair tiles
+        for bn, splits in [(0, 0), (512, 1), (512, 3), (384, 1), (384, 2), (256, 1), (128, 1), (96, 1), (64, 1), (32, 1), (128, 4), (64, 3), (256, 2)]:   # 512 / 384 = CTA-pair tiles with 128 / 64 rows per CTA
             ctx.set_option("gemm_bn", bn); ctx.set_option("gemm_splits", splits)
             dC = torch.full((M, N), 777.0, dtype=torch.float32, device=DEV)
             ctx.gemm(dA, dW, dC, impl=2)
