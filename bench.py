@@ -41,10 +41,12 @@ def ncu_traffic_per_launch():
     kernel source has changed since the counters were taken."""
     import hashlib
     prof = os.path.join(ROOT, "profiles", "decode_step_kernels_cfg2_reduced.txt")
-    src = os.path.join(ROOT, "paper_2601_19404_b200", "csrc", "gemm_tc.cuh")
     try:
         vals = dict(l.split(" = ") for l in open(prof).read().splitlines() if " = " in l)
-        if vals["gemm_tc_cuh_sha256"].strip() != hashlib.sha256(open(src, "rb").read()).hexdigest():
+        h = hashlib.sha256()
+        for name in ("gemm_tc.cuh", "gemm_tc2.cuh"):
+            h.update(open(os.path.join(ROOT, "paper_2601_19404_b200", "csrc", name), "rb").read())
+        if vals["gemm_sources_sha256"].strip() != h.hexdigest():
             return None
         return float(vals["gemm_decode_traffic_bytes_per_launch"])
     except Exception:
