@@ -569,8 +569,32 @@ __global__ void __launch_bounds__(128) attn_decode_merge_kernel(bf16* __restrict
 #pragma unroll
   for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
   float l_tot = 0.f, m_run = -INFINITY;        // warp-uniform
-  {   // rows of finished sequences are merged like any other: nothing downstream reads them
-    const int64_t slot0 = ((int64_t)r * hq + head) * n_slots;
+  const int64_t slot0 = ((int64_t)r * hq + head) * n_slots;
+  if (n_slots <= 8) {
+    // Few splits: the (m, l) pairs and every split's partial output are requested together (one
+    // round trip to L2 instead of two); the arithmetic and its order are those of the loop below.
+    float ms = -INFINITY, ls = 0.f;
+    if (lane < n_slots) { const float2 ml = *reinterpret_cast<const float2*>(part_ml + (slot0 + lane) * 2); ms = ml.x; ls = ml.y; }
+    float v[8][DPL];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const float* po = part_o + (slot0 + min(k, n_slots - 1)) * DH + lane * DPL;
+#pragma unroll
+      for (int i = 0; i < DPL; ++i) v[k][i] = po[i];
+    }
+    if (!(ls > 0.f)) ms = -INFINITY;
+    const float m_new = warp_max(ms);
+    const float wgt = (ls > 0.f) ? exp2f(ms - m_new) : 0.f;
+    l_tot = warp_sum(ls * wgt);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const float c = __shfl_sync(0xffffffffu, wgt, k);
+      if (k < n_slots) {
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) acc[i] += (c != 0.f) ? c * v[k][i] : 0.f;
+      }
+    }
+  } else {   // rows of finished sequences are merged like any other: nothing downstream reads them
     for (int s0 = 0; s0 < n_slots; s0 += 32) {         // one pass for n_slots <= 32, a second for the 33rd
       const int s = s0 + lane;
       float ms = -INFINITY, ls = 0.f;
