@@ -129,6 +129,20 @@ __global__ void gather_rows_f32_kernel(const float* __restrict__ src, const int3
   for (int i = threadIdx.x; i < d; i += blockDim.x) dst[(int64_t)r * d + i] = src[(int64_t)s * d + i];
 }
 
+__device__ __forceinline__ int lane_id() { return threadIdx.x & 31; }
+// Four consecutive outputs of type T (8 or 16 bytes, aligned) in one store.
+template <typename T>
+__device__ __forceinline__ void store4(T* dst, float a, float b, float c, float d);
+template <>
+__device__ __forceinline__ void store4<float>(float* dst, float a, float b, float c, float d) {
+  *reinterpret_cast<float4*>(dst) = make_float4(a, b, c, d);
+}
+template <>
+__device__ __forceinline__ void store4<bf16>(bf16* dst, float a, float b, float c, float d) {
+  const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+  *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+}
+
 // RMSNorm of the float32 residual stream, one CTA per row, 128-bit accesses (d % 4 == 0):
 //   x[r,:] += sum_s partial[s][r,:]   (optional split-K partial planes of the previous GEMM, summed
 //                                      in plane order; the loads of all planes are independent)
@@ -147,6 +161,36 @@ __global__ void rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ 
   float4* xr = reinterpret_cast<float4*>(x + (int64_t)r * d);
   float4* s4 = reinterpret_cast<float4*>(srow);
   float ss = 0.f;
+  if (d4 <= (int)blockDim.x) {
+    // One float4 per thread (decode-sized rows): the row stays in registers, and the gain is
+    // requested together with the row and the planes, so the kernel makes one round trip to L2.
+    const int i = threadIdx.x;
+    const bool on = i < d4;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f), g = v;
+    if (on) {
+      v = xr[i];
+      g = reinterpret_cast<const float4*>(gain)[i];
+      if (partial) {
+        const float4* p4 = reinterpret_cast<const float4*>(partial + (int64_t)r * d) + i;
+        const int64_t st4 = split_stride >> 2;
+#pragma unroll 4
+        for (int s = 0; s < n_splits; ++s) {
+          const float4 q = p4[s * st4];
+          v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
+        }
+        xr[i] = v;
+      }
+      ss = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = (lane_id() < (int)(blockDim.x >> 5)) ? red[lane_id()] : 0.f;
+    tot = warp_sum(tot);                       // every warp sums the per-warp parts in the same order
+    const float inv = 1.0f / sqrtf(tot / (float)d + eps);
+    if (on) store4<T>(h + (int64_t)r * d + 4 * i, v.x * inv * g.x, v.y * inv * g.y, v.z * inv * g.z, v.w * inv * g.w);
+    return;
+  }
   for (int i = threadIdx.x; i < d4; i += blockDim.x) {
     float4 v = xr[i];
     if (partial) {
