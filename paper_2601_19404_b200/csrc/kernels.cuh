@@ -98,13 +98,33 @@ __global__ void rope_table_kernel(float2* __restrict__ tab, int max_pos, int hal
 // x[r,:] = E[tok[r],:]  (float32 residual stream).
 // step_ctr (decode only): the first kernel of a decode forward advances the device step counter
 // that the sampler at the end of the forward reads, so that every step is the same launch sequence.
+// It also resolves, once per pass, what every layer's RoPE / KV-append kernel needs to know about
+// the row - absolute position and where its K/V go in the paged pool - so that those kernels read
+// one record instead of walking row -> sequence -> block table in every layer.
+struct RowMetaArgs {
+  const int32_t* row_seq; const int32_t* row_t; const SeqDesc* seqs; const int32_t* block_table;
+  int n_blocks, max_pos;
+  int4* row_meta;                     // out: (position, block, slot in block, 0); x = -1: inactive row
+};
 template <typename T>
 __global__ void embed_kernel(const int32_t* __restrict__ tokens, const T* __restrict__ E, float* __restrict__ x,
-                             int rows, int d, int vocab, int* status, int32_t* step_ctr) {
+                             int rows, int d, int vocab, int* status, int32_t* step_ctr, RowMetaArgs m) {
   pdl_prologue();
   const int r = blockIdx.x;
   if (step_ctr && r == 0 && threadIdx.x == 0) *step_ctr += 1;
   if (r >= rows) return;
+  if (threadIdx.x == 32) {            // a thread of the second warp: the first is about to wait on the token
+    int4 out = make_int4(-1, 0, 0, 0);
+    const int t = m.row_t[r];
+    if (t >= 0) {
+      const SeqDesc sd = m.seqs[m.row_seq[r]];
+      const int pos = sd.shared_len + t;
+      const int blk = (pos < m.max_pos) ? m.block_table[sd.priv_tbl + t / KV_BLOCK] : -1;
+      if (blk < 0 || blk >= m.n_blocks) atomicOr(status, STATUS_BAD_BLOCK);
+      else out = make_int4(pos, blk, t % KV_BLOCK, 0);
+    }
+    m.row_meta[r] = out;
+  }
   int tok = tokens[r];
   if (tok < 0 || tok >= vocab) {
     if (threadIdx.x == 0) atomicOr(status, STATUS_BAD_TOKEN);
@@ -288,10 +308,8 @@ __global__ void reduce_partials_kernel(float* __restrict__ x, const float* __res
 // they are summed in plane order and rounded to the storage type first, exactly what the
 // unsplit GEMM epilogue would have stored.
 template <typename T>
-__global__ void rope_kv_kernel(T* __restrict__ qkv, const int32_t* __restrict__ row_seq,
-                               const int32_t* __restrict__ row_t, const SeqDesc* __restrict__ seqs,
-                               const int32_t* __restrict__ block_table, const float2* __restrict__ rope_tab,
-                               KVPool<T> pool, int layer, int rows, int hq, int hkv, int max_pos, int* status,
+__global__ void rope_kv_kernel(T* __restrict__ qkv, const int4* __restrict__ row_meta, const float2* __restrict__ rope_tab,
+                               KVPool<T> pool, int layer, int rows, int hq, int hkv,
                                const float* __restrict__ partial, int n_splits, int64_t split_stride) {
   pdl_prologue();
   const int dh = pool.head_dim, half = dh / 2, tph = dh / 16, heads = hq + 2 * hkv;
@@ -326,18 +344,14 @@ __global__ void rope_kv_kernel(T* __restrict__ qkv, const int32_t* __restrict__ 
 #pragma unroll
     for (int j = 0; j < 8; ++j) { lo[j] = to_f32(tl[j]); hi[j] = to_f32(th[j]); }
   }
-  const int t = row_t[r];
-  if (t < 0) return;
-  const SeqDesc sd = seqs[row_seq[r]];
-  const int pos = sd.shared_len + t;
-  if (pos >= max_pos) { if (i0 == 0) atomicOr(status, STATUS_BAD_BLOCK); return; }
+  const int4 meta = row_meta[r];                        // (position, private KV block, slot in block): resolved once per pass
+  if (meta.x < 0) return;                               // inactive row (or a bad position / block, flagged when resolved)
+  const int pos = meta.x;
   T *dst_lo = src + i0, *dst_hi = src + half + i0;      // q: rotated in place
   if (head >= hq) {
     const int kv = (head - hq) / hkv, kh = (head - hq) % hkv;
-    const int blk = block_table[sd.priv_tbl + t / KV_BLOCK];
-    if (blk < 0 || blk >= pool.n_blocks) { if (i0 == 0) atomicOr(status, STATUS_BAD_BLOCK); return; }
-    dst_lo = pool.chunk(layer, kv, kh, blk, t % KV_BLOCK, i0);
-    dst_hi = pool.chunk(layer, kv, kh, blk, t % KV_BLOCK, half + i0);
+    dst_lo = pool.chunk(layer, kv, kh, meta.y, meta.z, i0);
+    dst_hi = pool.chunk(layer, kv, kh, meta.y, meta.z, half + i0);
   }
   __align__(16) T ol[8], oh[8];
   if (head < hq + hkv) {                                // q or k: rotate

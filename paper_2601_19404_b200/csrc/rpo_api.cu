@@ -94,6 +94,14 @@ static cudaError_t launch_kernel(rpo_ctx* c, void (*kern)(KArgs...), dim3 grid, 
     CUDA_TRY(cudaGetLastError());                                                            \
   } while (0)
 
+// What embed_kernel needs to resolve the rows' positions and KV slots (see RowMetaArgs).
+static RowMetaArgs row_meta_args(rpo_ctx* c) {
+  RowMetaArgs m;
+  m.row_seq = c->ws.row_seq; m.row_t = c->ws.row_t; m.seqs = (const SeqDesc*)c->ws.seqs; m.block_table = c->d_block_table;
+  m.n_blocks = (int)c->lim.kv_pool_blocks; m.max_pos = c->lim.max_positions; m.row_meta = c->ws.row_meta;
+  return m;
+}
+
 static inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
 static inline int grid_for(int64_t n, int block, int cap = 148 * 16) {
   return (int)std::max<int64_t>(1, std::min<int64_t>((n + block - 1) / block, cap));
@@ -269,6 +277,7 @@ extern "C" int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limit
   ALLOC(w.hh, (size_t)w.HR * d * e);
   ALLOC(w.logits, (size_t)w.HR * V * 4);
   ALLOC(w.row_seq, (size_t)w.R * 4);
+  ALLOC(w.row_meta, (size_t)w.R * sizeof(int4));
   ALLOC(w.row_t, (size_t)w.R * 4);
   ALLOC(w.row_tok, (size_t)w.R * 4);
   const int nseq = std::max(lim->max_seqs, lim->max_groups);
@@ -558,10 +567,9 @@ static int run_layers(rpo_ctx* c, int rows, bool flush = true) {
     int qkv_splits = 0;
     RPO_TRY(gemm<T>(c, (const T*)w.h, (const T*)L.wqkv, w.qkv, rows, c->qkv_cols, d, EPI_STORE_T, 0, true, &qkv_splits));
     { ProfScope ps(c, KC_ROPE);
-    LAUNCH(c, rope_kv_kernel<T>, ceil_div((int64_t)rows * (s.n_q_heads + 2 * s.n_kv_heads) * (s.head_dim / 16), 64), 64, 0, (T*)w.qkv, w.row_seq, w.row_t,
-           (const SeqDesc*)w.seqs, c->d_block_table, (const float2*)c->d_rope, kv_pool<T>(c), l, rows, s.n_q_heads,
-           s.n_kv_heads, c->lim.max_positions, c->d_status, qkv_splits > 1 ? (const float*)w.partial : (const float*)nullptr,
-           qkv_splits, (int64_t)rows * c->qkv_cols); }
+    LAUNCH(c, rope_kv_kernel<T>, ceil_div((int64_t)rows * (s.n_q_heads + 2 * s.n_kv_heads) * (s.head_dim / 16), 64), 64, 0, (T*)w.qkv,
+           (const int4*)w.row_meta, (const float2*)c->d_rope, kv_pool<T>(c), l, rows, s.n_q_heads, s.n_kv_heads,
+           qkv_splits > 1 ? (const float*)w.partial : (const float*)nullptr, qkv_splits, (int64_t)rows * c->qkv_cols); }
     RPO_TRY(attention<T>(c, l, rows));
     RPO_TRY(gemm<T>(c, (const T*)w.attn, (const T*)L.wo, w.x, rows, d, qo, EPI_ADD_F32, 0, true));
     RPO_TRY(rmsnorm<T>(c, w.x, L.g2, (T*)w.h, rows));
@@ -629,7 +637,7 @@ static int prefill_chunk(rpo_ctx* c, const int32_t* d_tokens, int tok0, const st
   CUDA_TRY(cudaMemcpyAsync(w.seqs, sd.data(), (size_t)n * sizeof(SeqDesc), cudaMemcpyHostToDevice, c->stream));
   RPO_TRY(upload_row_tiles(c, lens));
   LAUNCH(c, embed_kernel<T>, rows, 128, 0, d_tokens + tok0, (const T*)c->embed, w.x, rows, c->shape.d_model,
-         c->shape.vocab, c->d_status, (int32_t*)nullptr);
+         c->shape.vocab, c->d_status, (int32_t*)nullptr, row_meta_args(c));
   RPO_TRY(run_layers<T>(c, rows));
   // keep the residual stream of every group's last prefix token: step-0 logits come from it
   for (int i = 0; i < n; ++i)
@@ -799,7 +807,7 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
   // the first runs eagerly, the others replay a CUDA graph of it.
   auto enqueue_step = [&]() -> int {
     LAUNCH(c, embed_kernel<T>, B, 128, 0, (const int32_t*)w.cur_tok, (const T*)c->embed, w.x, B, d, c->shape.vocab,
-           c->d_status, w.step_ctr);
+           c->d_status, w.step_ctr, row_meta_args(c));
     // every row is a sequence's last row: the final RMSNorm reads ws.x directly and folds the last
     // layer's split-K partials in (no separate reduction, no copy of the residual rows)
     RPO_TRY(run_layers<T>(c, B, false));
@@ -909,7 +917,7 @@ static int logprobs_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, 
         build_teacher_rows_kernel<<<grid_for(rows, 256), 256, 0, st>>>(d_tokens, d_lens, s0, ns, S, w.row_seq, w.row_t,
                                                                       w.row_tok);
         c->launches++;
-        embed_kernel<T><<<rows, 128, 0, st>>>((const int32_t*)w.row_tok, (const T*)c->embed, w.x, rows, d, V, c->d_status, nullptr);
+        embed_kernel<T><<<rows, 128, 0, st>>>((const int32_t*)w.row_tok, (const T*)c->embed, w.x, rows, d, V, c->d_status, nullptr, row_meta_args(c));
         c->launches++;
         if ((rc = run_layers<T>(c, rows)) != RPO_OK) break;
       }
