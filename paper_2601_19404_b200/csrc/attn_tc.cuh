@@ -36,6 +36,7 @@ struct FlashArgs {
   KVPool<bf16> pool; int layer, hq, hkv; float scale_log2;
   const int2* tiles;      // ROWS: (first row, number of rows)
   int G;                  // SHARED: samples per group
+  const int32_t* pfx_tbl; int pfx_stride;   // SHARED: prefix block ids of the call's groups, dense [group][pfx_stride]
   int* status;
 };
 
@@ -196,6 +197,14 @@ flash_attn_kernel(FlashArgs a) {
       const bool v = qrow < n_rows;
       load_q(qrow, tid % QTPR, v ? grp * a.G + i / rep : -1, kvh * rep + (v ? i % rep : 0));
     }
+    // block ids of this split's prefix keys: one fetch up front instead of one per tile, from the
+    // call's dense table, so the request does not wait for the sequence descriptor (entries past a
+    // short prefix are padding and never used)
+    {
+      const int n_cache = min(BLK_CACHE, a.split_chunk / KV_BLOCK);
+      const int32_t* src = a.pfx_tbl + (int64_t)grp * a.pfx_stride + split * (a.split_chunk / KV_BLOCK);
+      for (int e = tid; e < n_cache; e += THREADS + 32) s_blk[e] = src[e];
+    }
     sd = a.seqs[grp * a.G];
     if (tid < FA_BM) {
       const bool v = tid < n_rows;
@@ -218,11 +227,8 @@ flash_attn_kernel(FlashArgs a) {
       const int j0 = ((split - (sq0 + tid)) % a.n_splits + a.n_splits) % a.n_splits;
       s_pt_sum[tid + 1] = (nt > j0) ? (nt - j0 - 1) / a.n_splits + 1 : 0;      // prefix-summed below
     }
-    // block ids of this split's prefix keys: one fetch up front instead of one per tile
     sh_begin = min(sd.shared_len, split * a.split_chunk);  // a multiple of 16
     sh_end = min(sd.shared_len, sh_begin + a.split_chunk);
-    const int n_blk = min(BLK_CACHE, (sh_end - sh_begin + KV_BLOCK - 1) / KV_BLOCK);
-    for (int e = tid; e < n_blk; e += THREADS + 32) s_blk[e] = a.block_table[sd.shared_tbl + sh_begin / KV_BLOCK + e];
   }
   __syncthreads();
   if (MODE == FA_SHARED) {

@@ -47,6 +47,8 @@ struct Workspace {
   size_t attn_part_elems = 0;
   void* tiles = nullptr;   // int2 (first row, rows) per 64-row attention tile
   int32_t *row_seq = nullptr, *row_t = nullptr, *row_tok = nullptr;
+  int32_t* pfx_tbl = nullptr;          // decode call: the groups' prefix block ids, dense [group][pfx_stride]
+  int pfx_stride = 0;
   int4* row_meta = nullptr;            // per row of the pass: (position, private KV block, slot in block, -) or x < 0: inactive
   void* seqs = nullptr;    // SeqDesc[]
   int32_t *done = nullptr, *lens = nullptr, *cur_tok = nullptr, *logit_row = nullptr, *slot_idx = nullptr;

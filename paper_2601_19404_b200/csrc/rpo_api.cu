@@ -278,6 +278,7 @@ extern "C" int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limit
   ALLOC(w.logits, (size_t)w.HR * V * 4);
   ALLOC(w.row_seq, (size_t)w.R * 4);
   ALLOC(w.row_meta, (size_t)w.R * sizeof(int4));
+  ALLOC(w.pfx_tbl, (size_t)lim->max_groups * (c->tbl_stride + 512 + 8) * 4);
   ALLOC(w.row_t, (size_t)w.R * 4);
   ALLOC(w.row_tok, (size_t)w.R * 4);
   const int nseq = std::max(lim->max_seqs, lim->max_groups);
@@ -483,7 +484,7 @@ static int attention(rpo_ctx* c, int layer, int rows) {
       a.row_seq = w.row_seq; a.row_t = w.row_t; a.seqs = (const SeqDesc*)w.seqs; a.block_table = c->d_block_table;
       a.pool = kv_pool<bf16>(c); a.layer = layer; a.hq = s.n_q_heads; a.hkv = s.n_kv_heads;
       a.scale_log2 = scale * 1.4426950408889634f; a.tiles = (const int2*)w.tiles; a.G = c->attn_G; a.status = c->d_status;
-      a.n_splits = c->attn_splits; a.split_chunk = c->attn_split_chunk;
+      a.n_splits = c->attn_splits; a.split_chunk = c->attn_split_chunk; a.pfx_tbl = w.pfx_tbl; a.pfx_stride = w.pfx_stride;
       if (c->attn_mode == 0 && tc5_attention(c)) {
         // tcgen05 path: 128-row tiles, Q through a tensor map over the fused qkv buffer
         const CUtensorMap* qm = tc_map(c, w.qkv, w.R, c->qkv_cols, T5_BM);
@@ -788,6 +789,17 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
     if (ceil_div(max_p, c->attn_split_chunk) > 32) c->attn_split_chunk = std::max(FA_BN, ceil_div(ceil_div(max_p, 32), FA_BN) * FA_BN);
     c->attn_splits = ceil_div(max_p, c->attn_split_chunk);
     c->attn_mode = 1; c->attn_G = G; c->attn_groups = n_groups;
+    // the groups' prefix block ids, dense and padded to splits x chunk: the attention CTA of
+    // (group, split) fetches its ids without knowing the group's descriptor
+    w.pfx_stride = c->attn_splits * (c->attn_split_chunk / KV_BLOCK);
+    if (w.pfx_stride > c->tbl_stride + 512 + 8) return RPO_ERR_LIMIT;
+    std::vector<int32_t> pfx((size_t)n_groups * w.pfx_stride, 0);
+    for (int g = 0; g < n_groups; ++g) {
+      const std::vector<int32_t>& blocks = c->groups[groups[g].slot].blocks;
+      const int nb = std::min((int)blocks.size(), ceil_div(groups[g].prefix_len, KV_BLOCK));
+      for (int k = 0; k < nb && k < w.pfx_stride; ++k) pfx[(size_t)g * w.pfx_stride + k] = blocks[k];
+    }
+    CUDA_TRY(cudaMemcpyAsync(w.pfx_tbl, pfx.data(), pfx.size() * 4, cudaMemcpyHostToDevice, st));
   }
   SamplerArgs a = sampler_args(c, sp);
   a.seq_ids = w.seq_ids; a.out_stride = S; a.forced = d_forced; a.tokens_out = d_tokens_out;
