@@ -234,3 +234,44 @@ def test_config3_full_size_ragged_prefixes_and_eos():
         assert ctx.device_status() == 0
         ctx.release_groups(groups)
         assert ctx.counters()[1] == ctx.limits.kv_pool_blocks
+
+
+def test_config4_full_size_decode_against_teacher_forced_pass():
+    """Config 4 at full size (7B-class, 28 layers, 32 groups x G=8 = 256 sequences, 4096-token prefixes)
+    with a short suffix: the decode path of this size - weight GEMMs on CTA pairs (256 rows), split-K
+    pair tiles for the down projection, two 2048-key prefix splits per group and KV head - against the
+    teacher-forced pass, which reaches the same log-probabilities through the prefill kernels; the
+    sampler's decisions are exact on the logits it was given."""
+    from oracle import sampler as osampler, philox
+    cfg = workloads.CONFIGS["cfg4_7b_32x8"]
+    shape = workloads.SHAPES[cfg["shape"]]
+    n_g, G, S = cfg["n_groups"], cfg["G"], 12
+    B = n_g * G
+    lens = workloads.prefix_lengths(cfg)
+    sc = cfg["sampler"]
+    with make_ctx(shape, n_g, G, int(lens.max()), S, chunk=16384) as ctx:
+        ctx.init_weights(0, 0.02)
+        toks, off = workloads.prefix_tokens(lens, shape["vocab"], seed=0)
+        groups = ctx.prefill_prefix(dev_i32(toks), off)
+        smp = rpo.Sampler(sc["temperature"], sc["top_p"], sc["greedy"], sc["eos_id"], seed=0)
+        t2, l2, lp2, dbg = run_decode(ctx, groups, G, 2, smp, want_logits=True)
+        for b in range(0, B, 17):                          # a sample of the 256 sequences
+            for j in range(2):
+                u = int(philox.sampler_u24(0, int(b), j))
+                assert t2[b, j] == osampler.sample_token(dbg[b, j], sc["temperature"], sc["top_p"], u), (b, j)
+        del dbg
+        t, l, lp, _ = run_decode(ctx, groups, G, S, smp)
+        ta, la, lpa, _ = run_decode(ctx, groups, G, S, smp)
+        assert np.array_equal(t, ta) and np.array_equal(lp.view(np.uint32), lpa.view(np.uint32))   # same seed, same bytes
+        assert np.array_equal(t[:, :2], t2) and np.all(l == S) and t.min() >= 0 and t.max() < shape["vocab"]
+        assert np.all(lp <= 0) and abs(lp.mean() + np.log(shape["vocab"])) < 1.5
+        pol = torch.zeros((B, S), dtype=torch.float32, device=DEV)
+        ctx.token_logprobs(groups, G, S, dev_i32(t), dev_i32(l), pol)
+        torch.cuda.synchronize()
+        diff = pol.cpu().numpy() - lp
+        # two bf16 passes with different kernels and batching, each within the depth tolerance of the exact value
+        assert np.max(np.abs(diff)) <= 2 * depth_tolerance(2e-2, shape["n_layers"]) * 1.5    # 7B widths: logit spread 1.2 vs 0.78
+        assert np.sqrt(np.mean(diff ** 2)) <= 3e-2
+        assert ctx.device_status() == 0
+        ctx.release_groups(groups)
+        assert ctx.counters()[1] == ctx.limits.kv_pool_blocks
