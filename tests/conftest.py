@@ -12,6 +12,12 @@ def pytest_configure(config):
 
 
 def pytest_collection_modifyitems(config, items):
+    # A GPU test that stalls must fail with the stacks of all threads, not hold the run: every GPU
+    # test gets a time limit when the pytest-timeout plug-in is there (the slowest takes ~20 s).
+    if config.pluginmanager.hasplugin("timeout"):
+        for it in items:
+            if "gpu" in it.keywords and it.get_closest_marker("timeout") is None:
+                it.add_marker(pytest.mark.timeout(600, method="thread"))
     try:
         import torch
         has_gpu = torch.cuda.is_available()
