@@ -1,5 +1,11 @@
 import os
 import sys
+
+# The oracle's numpy code runs on the host next to other jobs: a bounded BLAS thread pool keeps its
+# spin-waiting threads from multiplying the slowdown when the host cores are oversubscribed.
+for _v in ("OMP_NUM_THREADS", "OPENBLAS_NUM_THREADS", "MKL_NUM_THREADS"):
+    os.environ.setdefault(_v, "8")
+
 import pytest
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
