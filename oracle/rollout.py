@@ -24,14 +24,15 @@ class SamplerCfg:
 
 
 def rollout_group(w, shape, prefix_tokens, G, max_new, cfg, group_id=0, dt=np.float64,
-                  forced_tokens=None, want_logits=False):
+                  forced_tokens=None, want_logits=False, rnd=None):
     """Generate (or teacher-force) G suffixes over one shared prefix.
 
     Returns dict(tokens [G,max_new] int32, lens [G] int32, logprobs [G,max_new] float64,
     logits [G,max_new,V] float32 if want_logits).  Logits are rounded to float32 before
-    the sampler, which is the precision the sampler is defined in.
+    the sampler, which is the precision the sampler is defined in.  `rnd` (a
+    `decoder.Rounding`) switches the decoder's optional storage rounding on.
     """
-    sp = decoder.SharedPrefix(w, shape, prefix_tokens, dt)
+    sp = decoder.SharedPrefix(w, shape, prefix_tokens, dt, rnd)
     tokens = np.zeros((G, max_new), dtype=np.int32)
     logprobs = np.zeros((G, max_new), dtype=np.float64)
     lens = np.zeros(G, dtype=np.int32)
@@ -41,7 +42,7 @@ def rollout_group(w, shape, prefix_tokens, G, max_new, cfg, group_id=0, dt=np.fl
         seq = group_id * G + i
         inc_k = [list(k) for k in sp.k]      # private copy of the prefix K/V for this sample
         inc_v = [list(v) for v in sp.v]
-        inc = decoder.Incremental(w, shape, dt)
+        inc = decoder.Incremental(w, shape, dt, rnd)
         inc.k, inc.v, inc.n = inc_k, inc_v, sp.P
         logits = step0
         done = False
@@ -72,9 +73,9 @@ def rollout_group(w, shape, prefix_tokens, G, max_new, cfg, group_id=0, dt=np.fl
 
 
 def token_logprobs(w, shape, prefix_tokens, suffix_tokens, lens, inv_temperature=1.0, dt=np.float64,
-                   want_logits=False):
+                   want_logits=False, rnd=None):
     """log pi(o_j | prefix, o_<j) for j < lens[i]; zeros beyond. suffix_tokens [G, S]."""
-    sp = decoder.SharedPrefix(w, shape, prefix_tokens, dt)
+    sp = decoder.SharedPrefix(w, shape, prefix_tokens, dt, rnd)
     suffix_tokens = np.asarray(suffix_tokens)
     G, S = suffix_tokens.shape
     out = np.zeros((G, S), dtype=np.float64)

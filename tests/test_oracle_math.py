@@ -44,8 +44,8 @@ def test_philox_matches_library_implementation(tmp_path):
     np.save(cin, ctr)
     r = subprocess.run([sys.executable, str(src), str(cin), str(k0), str(k1), str(cout)],
                        capture_output=True, text=True, timeout=600)
-    if r.returncode != 0:
-        pytest.skip("Triton interpreter unavailable: " + r.stderr[-300:])
+    # no skip: without this run the Philox words would be pinned by statistics only
+    assert r.returncode == 0, "the independent Philox (Triton's CPU interpreter) did not run: " + r.stderr[-500:]
     got = np.stack(philox.philox4x32_10(ctr[0], ctr[1], ctr[2], ctr[3], k0, k1))
     assert np.array_equal(got, np.load(cout))
 

@@ -8,11 +8,25 @@ from oracle import sampler, rollout, decoder, init, philox, exactmath as em
 RNG = np.random.default_rng(21)
 
 
+def exact_top_p24(top_p):
+    """floor(float32(top_p) * 2^24) in exact rational arithmetic (no call of the code under test)."""
+    return math.floor(Fraction(float(np.float32(top_p))) * (1 << 24))
+
+
+def test_top_p_fixed_point_is_the_exact_floor():
+    for tp in [0.0, 1.0, 0.5, 0.9, 0.95, 0.3, 1e-9, 2.0 ** -24, 2.0 ** -25, 1.0 - 2.0 ** -24, 0.1, 1 / 3, 0.999999]:
+        assert sampler.top_p_fixed(tp) == exact_top_p24(tp), tp
+    assert sampler.top_p_fixed(0.95) == 15938355 and sampler.top_p_fixed(0.9) == 15099494   # float32(0.95), float32(0.9)
+    assert sampler.top_p_fixed(1.0) == 1 << 24 and sampler.top_p_fixed(0.0) == 0
+    for tp in RNG.uniform(0, 1, 200):
+        assert sampler.top_p_fixed(tp) == exact_top_p24(tp)
+
+
 def brute_sample(w, top_p, u24):
     """Sort-based textbook nucleus on integer weights with python ints."""
     w = [int(x) for x in w]
     total = sum(w)
-    target = (total * sampler.top_p_fixed(top_p)) >> 24
+    target = (total * exact_top_p24(top_p)) >> 24
     order = sorted(range(len(w)), key=lambda i: -w[i])
     acc, n = 0, 0
     while True:                                   # smallest sorted prefix reaching the target ...
@@ -62,7 +76,7 @@ def test_nucleus_mass_is_sufficient_and_minimal():
         top_p = float(RNG.uniform(0.05, 0.99))
         w = sampler.quantised_weights(logits, 1.0)
         tau, mass = sampler.nucleus_threshold(w, top_p)
-        total = int(w.sum()); target = (total * sampler.top_p_fixed(top_p)) >> 24
+        total = int(w.sum()); target = (total * exact_top_p24(top_p)) >> 24
         assert mass >= target
         assert mass - int(w[w == tau].sum()) < target          # dropping the tie class at tau falls short
 
