@@ -1,8 +1,11 @@
 #!/usr/bin/env python
-"""Suffix-rollout benchmark: one step = prefill of the cached prefixes (once per group) plus
-batched decode of G suffixes per group over the shared prefix KV, on seeded synthetic inputs.
+"""Suffix-rollout benchmark: one step = prefill of the cached prefixes (once per group), batched
+decode of G suffixes per group over the shared prefix KV and, where the configuration asks for them,
+the teacher-forced token log-probabilities, on seeded synthetic inputs.
 
-    python bench.py --gpus 1 --steps 5 --warmup 3            # this library, config 2
+    python bench.py --gpus 1 --steps 5 --warmup 3            # this library: config 4 is the headline,
+                                                             # configs 2, 3, 5-partial, 5-full ride along
+    python bench.py --gpus 2                                 # spawns one rank per GPU itself
     python bench.py --impl reference --steps 2 --warmup 1    # the CPU oracle on a bounded sample
 
 Prints ONE JSON line (rank 0).  value = suffix tokens/s over all ranks with inputs resident in
@@ -11,10 +14,10 @@ HBM; e2e = the same through rpo_rollout_host with pinned host buffers.
 import argparse
 import json
 import os
+import socket
 import subprocess
 import sys
 import tempfile
-import threading
 import time
 
 import numpy as np
@@ -25,32 +28,19 @@ import workloads  # noqa: E402
 
 METRIC = "suffix_rollout_tokens_per_sec"
 UNIT = "tokens/s"
+HEADLINE = "cfg4_7b_32x8"
+# The other configurations, with their own (fewer) steps: (name, warm-up, timed steps).  A step of the
+# full-path arm of config 5 is 4351 decode forwards (about a minute), so it runs once after one warm-up.
+OTHERS = [("cfg2_1p5b_16x8", 3, 3), ("cfg3_1p5b_64x8_ragged", 3, 2), ("cfg5_7b_partial", 3, 2), ("cfg5_7b_full", 1, 1)]
 
 
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         d = json.load(open(p))
-        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"], bf16_sustained=d.get("bf16_tflops_sustained"),
-                    source="measured")
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"], bf16_sustained=d.get("bf16_tflops_sustained") or d["bf16_tflops"],
+                    source="measured (MEASURED_PEAKS.json)")
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_sustained=1400.0, source="fallback")
-
-
-def ncu_traffic_per_launch():
-    """DRAM bytes per launch of the decode GEMM from the committed ncu capture, or None once the
-    kernel source has changed since the counters were taken."""
-    import hashlib
-    prof = os.path.join(ROOT, "profiles", "decode_step_kernels_cfg2_reduced.txt")
-    try:
-        vals = dict(l.split(" = ") for l in open(prof).read().splitlines() if " = " in l)
-        h = hashlib.sha256()
-        for name in ("gemm_tc.cuh", "gemm_tc2.cuh"):
-            h.update(open(os.path.join(ROOT, "paper_2601_19404_b200", "csrc", name), "rb").read())
-        if vals["gemm_sources_sha256"].strip() != h.hexdigest():
-            return None
-        return float(vals["gemm_decode_traffic_bytes_per_launch"])
-    except Exception:
-        return None
 
 
 class ClockSampler:
@@ -95,13 +85,17 @@ class ClockSampler:
         return out
 
 
+def layer_params(shape):
+    d, dh, hq, hkv, F = (shape[k] for k in ("d_model", "head_dim", "n_q_heads", "n_kv_heads", "d_ffn"))
+    return (hq + 2 * hkv) * dh * d + d * hq * dh + 3 * F * d
+
+
 def algorithmic_decode_bytes(shape, lens, G, S):
     """Bytes one decode step must move: all layer matrices + lm_head once, each group's prefix K/V
     once per group, each sequence's own suffix K/V (mean over the S-1 forward steps)."""
     e = 2 if shape["dtype"] == "bf16" else 4
-    d, dh, hq, hkv, F, V, L = (shape[k] for k in ("d_model", "head_dim", "n_q_heads", "n_kv_heads", "d_ffn", "vocab", "n_layers"))
-    layer = (hq + 2 * hkv) * dh * d + d * hq * dh + 3 * F * d
-    weights = (L * layer + V * d) * e
+    d, dh, hkv, V, L = (shape[k] for k in ("d_model", "head_dim", "n_kv_heads", "vocab", "n_layers"))
+    weights = (L * layer_params(shape) + V * d) * e
     kv_tok = 2 * L * hkv * dh * e
     prefix = int(np.sum(lens)) * kv_tok
     suffix = len(lens) * G * (S / 2.0) * kv_tok
@@ -109,108 +103,144 @@ def algorithmic_decode_bytes(shape, lens, G, S):
 
 
 def prefill_flops(shape, lens):
-    d, dh, hq, hkv, F, L = (shape[k] for k in ("d_model", "head_dim", "n_q_heads", "n_kv_heads", "d_ffn", "n_layers"))
-    layer = (hq + 2 * hkv) * dh * d + d * hq * dh + 3 * F * d
+    """GEMM flops of the layer stack over every prefix token + causal attention (no lm_head: it runs on
+    the last position of each group only)."""
+    dh, hq, L = (shape[k] for k in ("head_dim", "n_q_heads", "n_layers"))
     T = float(np.sum(lens))
     attn = sum(2 * 2 * (float(p) * p / 2) * dh * hq * L for p in lens)
-    return 2 * layer * L * T + attn
+    return 2 * layer_params(shape) * L * T, attn
 
 
-def run_reference(args, cfg_name, rank, world):
-    """The CPU oracle, as it stands, on a bounded sample of the workload (rank 0 only)."""
-    if rank != 0:
-        return
+def logprob_flops(shape, lens, G, S):
+    """Teacher-forced pass: layer stack over the B*(S-1) suffix rows, attention over prefix + own suffix,
+    lm_head on B*S rows."""
+    d, dh, hq, L, V = (shape[k] for k in ("d_model", "head_dim", "n_q_heads", "n_layers", "vocab"))
+    B = len(lens) * G
+    rows = B * (S - 1)
+    gemm = 2 * layer_params(shape) * L * rows + 2.0 * V * d * B * S
+    attn = sum(G * 2 * 2 * ((S - 1) * float(p) + (S - 1) * (S - 1) / 2.0) * dh * hq * L for p in lens)
+    return gemm, attn
+
+
+# ------------------------------------------------------------------------------------------------
+# the CPU oracle, timed as it stands
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(cfg_name, prefix, suffix, layers):
+    """Times the oracle (float32 numpy) on a bounded sample of the configuration: one prompt group,
+    `prefix` prefix tokens, G suffixes of `suffix` tokens, on a decoder cut to `layers` layers, once with
+    all of them and once with one fewer, so that the cost of a layer and of the rest (embedding, head,
+    sampler) separate and the figure for the configuration's full depth follows by linear extrapolation.
+    Returns (seconds of the sample, extrapolated seconds at full depth, tokens, description, threads)."""
     import torch
     from oracle import init as oinit, rollout as orollout, decoder as odecoder
     cfg = workloads.CONFIGS[cfg_name]
-    shape = workloads.SHAPES[cfg["shape"]]
-    sh = odecoder.Shape(**{k: shape[k] for k in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn",
-                                                  "vocab", "rope_base", "rms_eps", "dtype")})
+    shape = dict(workloads.SHAPES[cfg["shape"]])
+    full_layers = shape["n_layers"]
+    layers = max(2, min(layers, full_layers))
+    keys = ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab", "rope_base", "rms_eps", "dtype")
+    sh = odecoder.Shape(**{**{k: shape[k] for k in keys}, "n_layers": layers})
+    sh_less = odecoder.Shape(**{**{k: shape[k] for k in keys}, "n_layers": layers - 1})
     G = cfg["G"]
-    P, S = args.ref_prefix, args.ref_suffix
     w = oinit.init_weights(sh, seed=0, std=0.02)
-    toks, off = workloads.prefix_tokens(np.array([P], dtype=np.int32), sh.vocab, seed=0)
+    toks, _ = workloads.prefix_tokens(np.array([prefix], dtype=np.int32), sh.vocab, seed=0)
     sc = cfg["sampler"]
     ocfg = orollout.SamplerCfg(sc["temperature"], sc["top_p"], sc["greedy"], 0, sc["eos_id"])
-    times = []
-    for it in range(args.warmup + args.steps):
+
+    def run(s):
         t0 = time.perf_counter()
-        out = orollout.rollout_group(w, sh, toks, G, S, ocfg, group_id=it, dt=np.float32)
-        dt = time.perf_counter() - t0
+        orollout.rollout_group(w, s, toks, G, suffix, ocfg, dt=np.float32)
+        return time.perf_counter() - t0
+
+    def timer():
+        t_all, t_less = run(sh), run(sh_less)
+        per_layer = max(t_all - t_less, 0.0)
+        return t_all, (t_all - layers * per_layer) + full_layers * per_layer
+
+    desc = (f"1 group x G={G}, prefix {prefix} of the config's tokens, {suffix} suffix tokens, float32 numpy, decoder cut to {layers} "
+            f"of {full_layers} layers; tokens/s extrapolated linearly to {full_layers} layers from runs with {layers} and {layers - 1} layers")
+    return timer, G * suffix, desc, torch.get_num_threads()
+
+
+def run_reference(args, rank):
+    """The CPU oracle, as it stands, on a bounded sample of the headline workload (rank 0 only)."""
+    if rank != 0:
+        return
+    timer, n_tok, desc, cores = oracle_sample(args.config, args.ref_prefix, args.ref_suffix, args.ref_layers)
+    full_s = []
+    for it in range(args.warmup + args.steps):
+        _, t_full = timer()
         if it >= args.warmup:
-            times.append(dt)
-    ms = 1e3 * float(np.mean(times))
-    value = G * S / (ms / 1e3)
-    cores = torch.get_num_threads()
-    sample = f"1 group x G={G}, prefix {P} of the config's tokens, {S} suffix tokens, full depth, float32 numpy"
+            full_s.append(t_full)
+    ms = 1e3 * float(np.mean(full_s))
+    value = n_tok / (ms / 1e3)
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic", "config": {"workload": cfg_name, "sample": sample},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "dtype": "f32", "data": "synthetic", "config": {"workload": args.config, "sample": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }))
 
 
-def cpu_baseline(cfg_name, prefix, suffix):
-    import torch
-    from oracle import init as oinit, rollout as orollout, decoder as odecoder
-    cfg = workloads.CONFIGS[cfg_name]
-    shape = workloads.SHAPES[cfg["shape"]]
-    sh = odecoder.Shape(**{k: shape[k] for k in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn",
-                                                  "vocab", "rope_base", "rms_eps", "dtype")})
-    G = cfg["G"]
-    w = oinit.init_weights(sh, seed=0, std=0.02)
-    toks, _ = workloads.prefix_tokens(np.array([prefix], dtype=np.int32), sh.vocab, seed=0)
-    sc = cfg["sampler"]
-    t0 = time.perf_counter()
-    orollout.rollout_group(w, sh, toks, G, suffix, orollout.SamplerCfg(sc["temperature"], sc["top_p"], sc["greedy"], 0, sc["eos_id"]),
-                           dt=np.float32)
-    dt = time.perf_counter() - t0
-    return {"value": G * suffix / dt, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
-            "sample": f"1 group x G={G}, prefix {prefix}, {suffix} suffix tokens, full depth, float32 numpy, {dt:.1f} s"}
+def cpu_baseline(cfg_name, prefix, suffix, layers):
+    timer, n_tok, desc, cores = oracle_sample(cfg_name, prefix, suffix, layers)
+    t_sample, t_full = timer()
+    return {"value": n_tok / t_full, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc + f"; the sample took {t_sample:.1f} s"}
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="cfg2_1p5b_16x8")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-profile", action="store_true")
-    ap.add_argument("--chunk", type=int, default=0, help="prefill chunk in tokens (0: 16384, or the longest prefix if longer)")
-    ap.add_argument("--ref-prefix", type=int, default=1024)
-    ap.add_argument("--ref-suffix", type=int, default=8)
-    ap.add_argument("--options", default="", help="comma list name=value passed to rpo_set_option")
-    ap.add_argument("--layers", type=int, default=0, help="override n_layers (reduced case for profiler captures)")
-    ap.add_argument("--suffix", type=int, default=0, help="override the suffix length (reduced case for profiler captures)")
-    ap.add_argument("--groups", type=int, default=0, help="override the number of prompt groups (reduced case)")
-    ap.add_argument("--kernel-table", action="store_true", help="print per-kernel event timings of one profiled step on stderr")
-    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
-    args = ap.parse_args()
+# ------------------------------------------------------------------------------------------------
+# N ranks on one node
+# ------------------------------------------------------------------------------------------------
+def spawn_local_ranks(n, argv):
+    """`python bench.py --gpus N` without a launcher: start one process per GPU (rank r on device r),
+    rendezvous on 127.0.0.1; rank 0 prints the JSON line.  Returns the worst exit code."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + argv, env=env))
+    return max(p.wait() for p in procs)
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    if args.impl == "reference":
-        run_reference(args, args.config, rank, world)
-        return
 
+def reduce_over_ranks(dist, torch, dev, times_ms, counts):
+    """MAX of the timings, SUM of the counts over all ranks (identity for a single rank)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return list(times_ms), list(counts)
+    t = torch.tensor(times_ms, device=dev, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    c = torch.tensor(counts, device=dev, dtype=torch.int64)
+    dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    return t.tolist(), [int(x) for x in c.tolist()]
+
+
+def plumbing_only(args, rank, world):
+    """The rank plumbing of a multi-GPU run without a GPU (gloo): rendezvous, the reductions of the
+    timed figures, rank 0's JSON line.  Used by the CPU test of the launcher path."""
     import torch
     import torch.distributed as dist
+    if world > 1:
+        dist.init_process_group("gloo", rank=rank, world_size=world)
+    times, counts = reduce_over_ranks(dist if world > 1 else None, torch, "cpu", [100.0 + rank, 10.0 * (rank + 1)], [1000 + rank])
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "unit": UNIT, "n_gpus": world, "plumbing_only": True, "ms_per_step": times[0],
+                          "other_ms": times[1], "tokens": counts[0], "value": counts[0] / (times[0] / 1e3),
+                          "group_ids_rank0": workloads.rank_group_ids(4, rank).tolist()}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------------
+# one configuration on this rank's GPU
+# ------------------------------------------------------------------------------------------------
+def run_config(args, name, steps, warmup, rank, local_rank, world, dist, headline):
+    import torch
     import paper_2601_19404_b200 as rpo
     from paper_2601_19404_b200 import binding
 
-    torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=dev)
-
-    cfg = dict(workloads.CONFIGS[args.config])
+    cfg = dict(workloads.CONFIGS[name])
     shape = dict(workloads.SHAPES[cfg["shape"]])
     reduced = []
     if args.layers:
@@ -264,38 +294,51 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         step()
     barrier()
     launches0 = ctx.counters()[0]
-    clocks = ClockSampler(local_rank)
+    clocks = ClockSampler(local_rank) if headline else None
     timers = []
     t_begin = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
     t_begin.record(stream)
-    for _ in range(args.steps):
+    for _ in range(steps):
         step(timers)
     t_end.record(stream)
     barrier()
-    clk = clocks.stop()
-    total_ms = t_begin.elapsed_time(t_end)
+    clk = clocks.stop() if clocks else None
     launches = ctx.counters()[0] - launches0
-    emitted = int(d_lens.sum().item())
-    pre_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in timers]))
-    dec_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in timers]))
-    lp_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in timers]))
-    if world > 1:
-        t = torch.tensor([total_ms, pre_ms, dec_ms, lp_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, pre_ms, dec_ms, lp_ms = t.tolist()
-        em = torch.tensor([emitted], device=dev, dtype=torch.int64)
-        dist.all_reduce(em, op=dist.ReduceOp.SUM)
-        emitted_all = int(em.item())
-    else:
-        emitted_all = emitted
-    ms_per_step = total_ms / args.steps
-    value = emitted_all / (ms_per_step / 1e3)
+    phase = [float(np.mean([e[i].elapsed_time(e[i + 1]) for e in timers])) for i in range(3)]
+    (total_ms, pre_ms, dec_ms, lp_ms), (emitted,) = reduce_over_ranks(
+        dist if world > 1 else None, torch, dev, [t_begin.elapsed_time(t_end)] + phase, [int(d_lens.sum().item())])
+    ms_per_step = total_ms / steps
+    value = emitted / (ms_per_step / 1e3)
 
-    # ---- end to end through the host-buffer call (pinned host memory, copies inside the timed region)
+    peaks = measured_peaks()
+    ab = algorithmic_decode_bytes(shape, lens, G, S)
+    dec_step_ms = dec_ms / max(S - 1, 1)
+    decode_gbs = ab["total"] / (dec_step_ms * 1e-3) / 1e9
+    pf_gemm, pf_attn = prefill_flops(shape, lens)
+    prefill_tfs = (pf_gemm + pf_attn) / (pre_ms * 1e-3) / 1e12
+    out = {
+        "workload": name + ("" if not reduced else " REDUCED(" + ",".join(reduced) + ")"), "shape": cfg["shape"],
+        "n_groups": n_g, "G": G, "prefix_tokens": int(lens.sum()), "suffix": S, "steps": steps, "warmup": warmup,
+        "value": value, "unit": UNIT, "ms_per_step": ms_per_step,
+        "phases_ms": {"prefill": pre_ms, "decode": dec_ms, "logprobs": lp_ms, "decode_per_forward": dec_step_ms},
+        "decode_hbm": {"algorithmic_bytes_per_step": ab, "achieved_gbs": decode_gbs, "frac_of_measured": decode_gbs / peaks["hbm_gbs"],
+                       "frac_of_8tbs": decode_gbs / 8000.0},
+        "prefill_tensor": {"flops": pf_gemm + pf_attn, "achieved_tflops": prefill_tfs,
+                           "frac_of_measured_burst": prefill_tfs / peaks["bf16_tflops"],
+                           "frac_of_measured_sustained": prefill_tfs / peaks["bf16_sustained"], "frac_of_2250": prefill_tfs / 2250.0},
+    }
+    if want_lp and lp_ms > 0:
+        lg, la = logprob_flops(shape, lens, G, S)
+        out["logprobs_tensor"] = {"flops": lg + la, "achieved_tflops": (lg + la) / (lp_ms * 1e-3) / 1e12}
+    if not headline:
+        ctx.close()
+        return out
+
+    # ---- headline only: end to end through the host-buffer call (pinned host memory, copies timed)
     e2e = None
     if not args.no_e2e:
         h_toks = torch.from_numpy(toks).pin_memory()
@@ -311,75 +354,139 @@ def main():
         e2e_step()
         barrier()
         e_begin = torch.cuda.Event(enable_timing=True); e_end = torch.cuda.Event(enable_timing=True)
-        n_e2e = max(1, min(args.steps, 3))
+        n_e2e = max(1, min(steps, 3))
         e_begin.record(stream)
         for _ in range(n_e2e):
             e2e_step()
         e_end.record(stream)
         barrier()
-        e2e_ms = e_begin.elapsed_time(e_end) / n_e2e
-        e2e_tokens = int(h_lens.sum().item())
-        if world > 1:
-            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64); dist.all_reduce(t, op=dist.ReduceOp.MAX); e2e_ms = t.item()
-            em = torch.tensor([e2e_tokens], device=dev, dtype=torch.int64); dist.all_reduce(em, op=dist.ReduceOp.SUM); e2e_tokens = int(em.item())
+        (e2e_ms,), (e2e_tokens,) = reduce_over_ranks(dist if world > 1 else None, torch, dev,
+                                                     [e_begin.elapsed_time(e_end) / n_e2e], [int(h_lens.sum().item())])
         h2d = int(toks.nbytes)
         d2h = int(h_out.numel() * 4 + h_lens.numel() * 4 + h_lp.numel() * 4 + (h_pol.numel() * 4 if want_lp else 0))
-        e2e = {"value": e2e_tokens / (e2e_ms / 1e3), "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
+        e2e = {"value": e2e_tokens / (e2e_ms / 1e3), "unit": UNIT, "ms_per_step": e2e_ms, "steps": n_e2e, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h}
 
-    # ---- roofline: per-kernel event timing in one extra profiled step (graphs off, same kernels)
-    peaks = measured_peaks()
-    ab = algorithmic_decode_bytes(shape, lens, G, S)
-    dec_step_ms = dec_ms / max(S - 1, 1)
-    roofline = None
-    phases = None
+    # ---- roofline of the kernel with the largest share of the step: per-kernel event timing in one extra
+    #      profiled step (CUDA graphs off, same kernels; the brackets add a few microseconds per launch)
+    roofline = roofline_decode = phases = None
     if not args.no_profile and rank == 0:
         ctx.set_option("profile", 2 if args.kernel_table else 1)
         step()
         prof = ctx.profile_read()
         ctx.set_option("profile", 0)
         phases = {p: {k: {"ms": round(v[0], 3), "launches": v[1]} for k, v in d.items() if v[1]} for p, d in prof.items()}
-        gemm_ms, gemm_n = prof["decode"]["gemm"]
-        # Dominant kernel of the path: the weight-streaming tensor-core GEMM of the decode step (all
-        # layer matrices + lm_head once per step).  Algorithmic bytes per launch = weight bytes a step
-        # reads / GEMM launches per step; duration = mean of CUDA-event pairs bracketing every launch
-        # of the profiled step (bracketing adds a few microseconds per launch: the fraction is a floor).
-        if gemm_n:
-            per_launch_bytes = ab["weights"] * (S - 1) / gemm_n
-            achieved = per_launch_bytes / (gemm_ms / gemm_n * 1e-3) / 1e9
-            esz = 2 if shape["dtype"] == "bf16" else 4
-            roofline = {"bound": "hbm", "kernel": "gemm_tc_kernel / gemm_tc2_kernel (decode weight GEMMs)", "achieved": achieved,
-                        "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                        "traffic": ncu_traffic_per_launch() if (not reduced and args.config.startswith("cfg2")) else None,
-                        "tensor_tflops": 2.0 * B * (ab["weights"] / esz) * (S - 1) / (gemm_ms * 1e-3) / 1e12,
-                        "algorithmic_bytes_per_launch": per_launch_bytes, "launches_per_step": gemm_n / max(S - 1, 1),
-                        "peak_source": peaks["source"] + " copy bandwidth (MEASURED_PEAKS.json)" if peaks["source"] == "measured" else "fallback",
-                        "ms_per_launch": gemm_ms / gemm_n}
-    decode_gbs = ab["total"] / (dec_step_ms * 1e-3) / 1e9
-    pf = prefill_flops(shape, lens)
-    prefill_tfs = pf / (pre_ms * 1e-3) / 1e12
+        esz = 2 if shape["dtype"] == "bf16" else 4
+        dgemm_ms, dgemm_n = prof["decode"]["gemm"]
+        mgemm_ms = prof["prefill"]["gemm"][0] + prof["logprobs"]["gemm"][0]
+        mgemm_n = prof["prefill"]["gemm"][1] + prof["logprobs"]["gemm"][1]
+        if dgemm_n:
+            # weight-streaming GEMMs of the decode forwards: algorithmic bytes = every layer matrix + lm_head once per forward
+            per_launch = ab["weights"] * (S - 1) / dgemm_n
+            ach = per_launch / (dgemm_ms / dgemm_n * 1e-3) / 1e9
+            roofline_decode = {"bound": "hbm", "kernel": "gemm_tc_kernel / gemm_tc2_kernel, decode forwards (weight streaming)",
+                               "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": None,
+                               "algorithmic_bytes_per_launch": per_launch, "launches": dgemm_n, "ms_per_launch": dgemm_ms / dgemm_n,
+                               "share_of_step": dgemm_ms / (ms_per_step), "peak_source": peaks["source"] + ": copy bandwidth",
+                               "tensor_tflops": 2.0 * B * (ab["weights"] / esz) * (S - 1) / (dgemm_ms * 1e-3) / 1e12}
+        if mgemm_n:
+            # the same GEMM kernels over many rows (prefill chunks, teacher-forced pass): 2 M N K flops per launch
+            flops = pf_gemm + (logprob_flops(shape, lens, G, S)[0] if want_lp else 0.0)
+            ach = flops / (mgemm_ms * 1e-3) / 1e12
+            roofline_many = {"bound": "tensor", "kernel": "gemm_tc2_kernel (CTA pairs), prefill and teacher-forced passes",
+                             "achieved": ach, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_sustained"],
+                             "traffic": None, "algorithmic_flops_per_launch": flops / mgemm_n, "launches": mgemm_n,
+                             "ms_per_launch": mgemm_ms / mgemm_n, "share_of_step": mgemm_ms / ms_per_step,
+                             "frac_of_burst_peak": ach / peaks["bf16_tflops"],
+                             "peak_source": peaks["source"] + ": sustained cuBLAS bf16 (the kernel runs inside a seconds-long step)"}
+        else:
+            roofline_many = None
+        # the dominant kernel is the one with the larger share of the timed step
+        if roofline_many and (not roofline_decode or roofline_many["share_of_step"] >= roofline_decode["share_of_step"]):
+            roofline, other = roofline_many, roofline_decode
+        else:
+            roofline, other = roofline_decode, roofline_many
+        roofline_decode = other
+    out.update({"e2e": e2e, "roofline": roofline, "roofline_second_kernel": roofline_decode, "kernel_classes": phases,
+                "gpu_launches": int(launches), "clocks": clk, "device_status": ctx.device_status()})
+    ctx.close()
+    return out
 
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default=HEADLINE, help="headline configuration (workloads.CONFIGS)")
+    ap.add_argument("--no-others", action="store_true", help="skip the other configurations")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-profile", action="store_true")
+    ap.add_argument("--chunk", type=int, default=0, help="prefill chunk in tokens (0: 16384, or the longest prefix if longer)")
+    ap.add_argument("--ref-prefix", type=int, default=128, help="oracle sample: prefix tokens")
+    ap.add_argument("--ref-suffix", type=int, default=4, help="oracle sample: suffix tokens")
+    ap.add_argument("--ref-layers", type=int, default=2, help="oracle sample: layers of the cut decoder (>= 2)")
+    ap.add_argument("--options", default="", help="comma list name=value passed to rpo_set_option")
+    ap.add_argument("--layers", type=int, default=0, help="override n_layers (reduced case for profiler captures)")
+    ap.add_argument("--suffix", type=int, default=0, help="override the suffix length (reduced case for profiler captures)")
+    ap.add_argument("--groups", type=int, default=0, help="override the number of prompt groups (reduced case)")
+    ap.add_argument("--kernel-table", action="store_true", help="print per-kernel event timings of one profiled step on stderr")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--plumbing-only", action="store_true", help="rank plumbing on CPU (gloo), no GPU work: launcher test")
+    args = ap.parse_args()
+
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1 and args.impl == "ours":
+        sys.exit(spawn_local_ranks(args.gpus, sys.argv[1:]))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if args.plumbing_only:
+        plumbing_only(args, rank, world)
+        return
+
+    import torch
+    import torch.distributed as dist
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    head = run_config(args, args.config, args.steps, args.warmup, rank, local_rank, world, dist, headline=True)
+    shape = workloads.SHAPES[workloads.CONFIGS[args.config]["shape"]]
     out = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if shape["dtype"] == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": args.config + ("" if not reduced else " REDUCED(" + ",".join(reduced) + ")"), "shape": cfg["shape"], "n_groups": n_g, "G": G, "prefix_tokens": int(lens.sum()),
-                   "suffix": S, "l2": "inputs larger than L2 (weights %.2f GB + KV)" % (ab["weights"] / 1e9),
+        "config": {"workload": head["workload"], "shape": head["shape"], "n_groups": head["n_groups"], "G": head["G"],
+                   "prefix_tokens": head["prefix_tokens"], "suffix": head["suffix"],
+                   "step": "prefill + decode" + (" + token log-probs" if workloads.CONFIGS[args.config].get("logprobs") else ""),
+                   "l2": "inputs larger than L2 (weights %.2f GB + KV)" % (head["decode_hbm"]["algorithmic_bytes_per_step"]["weights"] / 1e9),
                    "parallelism": f"groups sharded over {world} rank(s), no collective in the step"},
-        "phases_ms": {"prefill": pre_ms, "decode": dec_ms, "logprobs": lp_ms, "decode_per_step": dec_step_ms},
-        "decode_hbm": {"algorithmic_bytes_per_step": ab, "achieved_gbs": decode_gbs, "frac_of_measured": decode_gbs / peaks["hbm_gbs"],
-                       "frac_of_8tbs": decode_gbs / 8000.0},
-        "prefill_tensor": {"flops": pf, "achieved_tflops": prefill_tfs, "frac_of_measured_burst": prefill_tfs / peaks["bf16_tflops"],
-                           "frac_of_2250": prefill_tfs / 2250.0},
-        "roofline": roofline, "kernel_classes": phases,
-        "e2e": e2e,
-        "gpu_launches": int(launches), "clocks": clk, "device_status": ctx.device_status(),
     }
+    for k in ("phases_ms", "decode_hbm", "prefill_tensor", "logprobs_tensor", "roofline", "roofline_second_kernel", "kernel_classes",
+              "e2e", "gpu_launches", "clocks", "device_status"):
+        if k in head:
+            out[k] = head[k]
+    # the other configurations, same kernels, their own (fewer) steps; one GPU only
+    if world == 1 and not args.no_others and not (args.layers or args.suffix or args.groups):
+        others = {}
+        for name, w_, s_ in OTHERS:
+            if name == args.config:
+                continue
+            others[name] = run_config(args, name, s_, w_, rank, local_rank, world, dist, headline=False)
+        full, part = others.get("cfg5_7b_full"), others.get("cfg5_7b_partial")
+        if full and part:
+            others["cfg5_partial_over_full"] = {"wall_time_ratio": part["ms_per_step"] / full["ms_per_step"],
+                                                "generated_token_ratio": part["suffix"] / full["suffix"]}
+        out["other_configs"] = others
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline(args.config, args.ref_prefix, args.ref_suffix)
+        out["cpu_baseline"] = cpu_baseline(args.config, args.ref_prefix, args.ref_suffix, args.ref_layers)
     if rank == 0:
         print(json.dumps(out))
-    ctx.close()
     if world > 1:
         dist.destroy_process_group()
 

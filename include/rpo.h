@@ -254,8 +254,27 @@ int rpo_gemm_bench(rpo_ctx* ctx, int32_t M, int32_t N, int32_t K, const void* d_
 /* Device status word, sticky until read: 0 = clean; bit 0 = a bounded wait expired
  * (TMA / MMA pipeline), bit 1 = token id out of range (clamped), bit 2 = block-table
  * index out of range (access skipped).  Synchronises the stream; *out receives the word
- * and the word is cleared. */
+ * and the word is cleared.  Returns RPO_ERR_DEVICE_TIMEOUT when bit 0 was set (the results of
+ * the work enqueued since the last read are not to be trusted; the context stays usable),
+ * else RPO_OK.  The asynchronous entry points (prefill, decode, token log-probs) cannot
+ * report an expired wait themselves: poll this call after them.  rpo_rollout_host, which
+ * synchronises anyway, checks the word itself and returns RPO_ERR_DEVICE_TIMEOUT (bit 0) or
+ * RPO_ERR_CUDA (bit 2). */
 int rpo_device_status(rpo_ctx* ctx, int32_t* out);
+
+/* Test tap on the residual stream (the hidden state x of the decoder the policy pi_theta of Eq. 3
+ * and Eq. 7 evaluates).  While a buffer is set, every pass through the layer stack (each prefill
+ * chunk, each decode forward, each chunk of rpo_token_logprobs) appends to it, in call order:
+ * the rows entering layer 0 as [rows, d_model] float32; then for every layer its attention
+ * output [rows, n_q_heads*head_dim] in the storage type (two bf16 values per float slot) and the
+ * rows leaving the layer as [rows, d_model] float32.  A parity test can thus check every layer
+ * on its own against the definition, fed with the library's own layer input, so that 16-bit
+ * storage rounding does not accumulate over the depth of the model in the comparison.
+ *   d_buf device float [capacity_floats], caller-owned; NULL switches the tap off.  Each call
+ *   restarts the write position at 0; h_used_out (nullable) receives the number of floats written
+ *   through the previous setting.  A pass that would overflow the buffer fails with RPO_ERR_LIMIT.
+ * While the tap is on the decode step is not replayed as a CUDA graph. */
+int rpo_debug_tap(rpo_ctx* ctx, float* d_buf, int64_t capacity_floats, int64_t* h_used_out);
 
 /* Counters since creation: kernels launched by the library, free KV blocks. */
 int rpo_counters(rpo_ctx* ctx, int64_t* kernel_launches, int64_t* free_kv_blocks);
@@ -268,6 +287,11 @@ int rpo_counters(rpo_ctx* ctx, int64_t* kernel_launches, int64_t* free_kv_blocks
  * pairs for passes of more than 128 rows, default 1), "use_cluster_merge" (decode attention:
  * the prefix splits of a work item form a thread-block cluster and merge through distributed
  * shared memory instead of a second kernel; default 0), "profile" (see rpo_profile_read),
+ * "use_tc5_decode" (tcgen05 decode attention when a group's rows of one KV head fit a 64-row
+ * tile; default 0: the mma.sync kernel measured faster), "use_fused_layers" (RMSNorm / RoPE / KV append / SwiGLU / residual add as GEMM
+ * epilogues in passes whose products do not split K, default 1; 2 = also where they split),
+ * "wait_limit_cycles" (limit of every bounded device-side wait in SM cycles, for ALL contexts on the
+ * device; <= 0 restores the default of 2e8, about 0.1 s),
  * "gemm_bn" (0 = planner, else force the tensor-core tile width: 32/64/96/128/256, or 512 / 384
  * for the CTA-pair kernel with 128 / 64 rows per CTA) and "gemm_splits" (with gemm_bn: force the split-K factor where the
  * caller can reduce planes). */

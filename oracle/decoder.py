@@ -175,6 +175,20 @@ def _finish_layer(w, shape, l, x, a, dt, rnd=None):
     return x + act @ mat(w, f"layers.{l}.wd", dt).T
 
 
+def layer(w, shape, l, x, pos, k_ctx, v_ctx, visible, dt=np.float64, rnd=None):
+    """One decoder layer on rows x [T, d] at positions pos.
+
+    The rows attend to k_ctx / v_ctx [U, Hkv, dh] (keys computed earlier, may be None) followed
+    by their own keys; visible is [T, U + T].  Returns (x_out [T, d], attention output
+    [T, Hq, dh], k [T, Hkv, dh], v [T, Hkv, dh]).
+    """
+    q, k, v = _qkv(w, shape, l, x, pos, dt, rnd)
+    K = k if k_ctx is None else np.concatenate([k_ctx, k])
+    V = v if v_ctx is None else np.concatenate([v_ctx, v])
+    a = attend(q, K, V, visible, rnd)
+    return _finish_layer(w, shape, l, x, a, dt, rnd), a, k, v
+
+
 def head(w, shape, x, dt, rnd=None):
     return normed_products(x, mat(w, "gf", dt), shape.rms_eps, [mat(w, "lm_head", dt)], rnd)[0]
 

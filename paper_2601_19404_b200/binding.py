@@ -14,7 +14,7 @@ _LIB = None
 EXPORTED_SYMBOLS = [
     "rpo_strerror", "rpo_shape_preset", "rpo_create", "rpo_destroy", "rpo_init_weights", "rpo_read_tensor",
     "rpo_write_tensor", "rpo_prefill_prefix", "rpo_decode_suffix", "rpo_token_logprobs", "rpo_release_groups",
-    "rpo_policy_objective", "rpo_rollout_host", "rpo_sample_rows", "rpo_sample_rows_noalloc", "rpo_gemm", "rpo_gemm_bench", "rpo_device_status", "rpo_counters", "rpo_set_option", "rpo_profile_read",
+    "rpo_policy_objective", "rpo_rollout_host", "rpo_sample_rows", "rpo_sample_rows_noalloc", "rpo_gemm", "rpo_gemm_bench", "rpo_device_status", "rpo_debug_tap", "rpo_counters", "rpo_set_option", "rpo_profile_read",
 ]
 
 
@@ -84,6 +84,7 @@ def load_library(path=None):
     lib.rpo_gemm.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp]
     lib.rpo_gemm_bench.argtypes = [vp, i32, i32, i32, vp, C.POINTER(vp), i32, i32, C.POINTER(f32)]
     lib.rpo_device_status.argtypes = [vp, C.POINTER(i32)]
+    lib.rpo_debug_tap.argtypes = [vp, vp, i64, C.POINTER(i64)]
     lib.rpo_counters.argtypes = [vp, C.POINTER(i64), C.POINTER(i64)]
     lib.rpo_set_option.argtypes = [vp, C.c_char_p, i32]
     lib.rpo_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64), i32]
@@ -261,10 +262,21 @@ class Context:
                "rpo_gemm_bench")
         return ms.value
 
-    def device_status(self):
+    def device_status(self, raise_on_timeout=True):
+        """The device status word (cleared by the read).  An expired device-side wait (bit 0) raises
+        RpoError(RPO_ERR_DEVICE_TIMEOUT) unless raise_on_timeout is False."""
         v = C.c_int32()
-        _check(self.lib.rpo_device_status(self.handle, C.byref(v)), "rpo_device_status")
+        rc = self.lib.rpo_device_status(self.handle, C.byref(v))
+        if rc != 0 and (raise_on_timeout or rc != -5):
+            raise RpoError(rc, "rpo_device_status")
         return v.value
+
+    def debug_tap(self, d_buf):
+        """Set (tensor) or clear (None) the residual-stream tap; returns the floats written so far."""
+        used = C.c_int64()
+        _check(self.lib.rpo_debug_tap(self.handle, _ptr(d_buf), 0 if d_buf is None else d_buf.numel(), C.byref(used)),
+               "rpo_debug_tap")
+        return used.value
 
     def counters(self):
         a, b = C.c_int64(), C.c_int64()

@@ -37,6 +37,8 @@ struct FlashArgs {
   const int2* tiles;      // ROWS: (first row, number of rows)
   int G;                  // SHARED: samples per group
   const int32_t* pfx_tbl; int pfx_stride;   // SHARED: prefix block ids of the call's groups, dense [group][pfx_stride]
+  int skip_prefix;        // SHARED: the work items carry suffix tiles only (the prefix is another kernel's: attn_dec5.cuh)
+  int n_slots, slot_base; // SHARED: partial slots per (row, head); split s writes slot slot_base + s
   int* status;
 };
 
@@ -200,7 +202,7 @@ flash_attn_kernel(FlashArgs a) {
     // block ids of this split's prefix keys: one fetch up front instead of one per tile, from the
     // call's dense table, so the request does not wait for the sequence descriptor (entries past a
     // short prefix are padding and never used)
-    {
+    if (!a.skip_prefix) {
       const int n_cache = min(BLK_CACHE, a.split_chunk / KV_BLOCK);
       const int32_t* src = a.pfx_tbl + (int64_t)grp * a.pfx_stride + split * (a.split_chunk / KV_BLOCK);
       for (int e = tid; e < n_cache; e += THREADS + 32) s_blk[e] = src[e];
@@ -229,6 +231,7 @@ flash_attn_kernel(FlashArgs a) {
     }
     sh_begin = min(sd.shared_len, split * a.split_chunk);  // a multiple of 16
     sh_end = min(sd.shared_len, sh_begin + a.split_chunk);
+    if (a.skip_prefix) { sh_begin = 0; sh_end = 0; }
   }
   __syncthreads();
   if (MODE == FA_SHARED) {
@@ -512,7 +515,7 @@ flash_attn_kernel(FlashArgs a) {
       for (int i = 0; i < ONT; ++i)
         *(uint32_t*)(dst + i * 8 + tq * 2) = fa::pack_bf16(o[i][half * 2] * inv, o[i][half * 2 + 1] * inv);
     } else {
-      const int64_t slot = ((int64_t)qr * a.hq + s_head[r]) * a.n_splits + split;
+      const int64_t slot = ((int64_t)qr * a.hq + s_head[r]) * a.n_slots + a.slot_base + split;
       if (tq == 0) { a.part_ml[slot * 2] = m; a.part_ml[slot * 2 + 1] = l; }
       float* dst = a.part_o + slot * DH;
 #pragma unroll

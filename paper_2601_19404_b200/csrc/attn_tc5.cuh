@@ -32,7 +32,6 @@ struct Flash5Args {
   KVPool<bf16> pool; int layer, hq, hkv; float scale_log2;
   const int2* tiles;      // (first row, number of rows <= 128)
   int q_col0;             // column of head 0's q inside a qkv row (0)
-  int v_desc_variant;     // which of LBO / SBO carries the dim-half stride of the V operand (see below)
   int* status;
 };
 
@@ -40,13 +39,13 @@ namespace t5 {
 // K-major, 128-byte swizzle (same as the GEMM operands).
 __device__ __forceinline__ uint64_t desc_k_sw128(uint32_t addr) { return tc::umma_desc_sw128(addr); }
 // MN-major, 128-byte swizzle: rows of 128 bytes run along the N (head dim) axis, 8 rows (keys) form
-// a 1024-byte swizzle atom; the second half of the head dims sits `mn_stride` bytes further.
-__device__ __forceinline__ uint64_t desc_mn_sw128(uint32_t addr, uint32_t mn_stride, uint32_t k_stride, int variant) {
-  const uint32_t lbo = variant ? k_stride : mn_stride, sbo = variant ? mn_stride : k_stride;
+// a 1024-byte swizzle atom; the second half of the head dims sits `mn_stride` bytes further (the
+// leading byte offset), groups of 8 keys are `k_stride` bytes apart (the stride byte offset).
+__device__ __forceinline__ uint64_t desc_mn_sw128(uint32_t addr, uint32_t mn_stride, uint32_t k_stride) {
   uint64_t d = 0;
   d |= (uint64_t)((addr & 0x3FFFF) >> 4);
-  d |= (uint64_t)(lbo >> 4) << 16;
-  d |= (uint64_t)(sbo >> 4) << 32;
+  d |= (uint64_t)(mn_stride >> 4) << 16;
+  d |= (uint64_t)(k_stride >> 4) << 32;
   d |= (uint64_t)1 << 46;
   d |= (uint64_t)2 << 61;
   return d;
@@ -174,7 +173,7 @@ flash_attn_tc5_kernel(const __grid_constant__ CUtensorMap q_map, Flash5Args a) {
 #pragma unroll
         for (int b = 0; b < T5_BN / KV_BLOCK; ++b) {                         // 16 keys per MMA = one KV block
           const uint64_t da = t5::desc_k_sw128(sP + (b >> 2) * (T5_TILE / 2) + (b & 3) * 32);
-          const uint64_t db = t5::desc_mn_sw128(sV + st * T5_TILE + b * 4096, 2048, 1024, a.v_desc_variant);
+          const uint64_t db = t5::desc_mn_sw128(sV + st * T5_TILE + b * 4096, 2048, 1024);
           tc::umma_bf16(tmem + 2 * T5_BN, da, db, idesc_pv, b > 0);
         }
         tc::umma_commit(&empty_v[st]);
@@ -202,7 +201,7 @@ flash_attn_tc5_kernel(const __grid_constant__ CUtensorMap q_map, Flash5Args a) {
       const bool shared_tile = it < n_sh;
       const int key0 = (shared_tile ? it * T5_BN : (it - n_sh) * T5_BN) + hf * 64;   // first key of my half
       const int lim = shared_tile ? sh_end - 1 : t_row;                       // last visible key of this row in the segment
-      if (!tc::mbar_wait(&s_full[sb], (it >> 1) & 1, abort_flag)) { ok = false; break; }
+      if (!tc::mbar_wait_warp(&s_full[sb], (it >> 1) & 1, abort_flag)) { ok = false; break; }
       tc::tmem_fence_after();
       // my 64 scores, kept in registers for both passes
       uint32_t v[64];
@@ -222,14 +221,14 @@ flash_attn_tc5_kernel(const __grid_constant__ CUtensorMap q_map, Flash5Args a) {
       xmax[(sb * 2 + hf) * 128 + r] = mx;
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(pair_bar);                               // release: my warp's maxima are written
-      if (!tc::mbar_wait(pair_bar, it & 1, abort_flag)) { ok = false; break; }
+      if (!tc::mbar_wait_warp(pair_bar, it & 1, abort_flag)) { ok = false; break; }
       mx = fmaxf(mx, xmax[(sb * 2 + (hf ^ 1)) * 128 + r]);
       const float m_new = fmaxf(m, mx), mu = (m_new == -INFINITY) ? 0.f : m_new;
       const float c_prev = corr;                                              // factor that goes with O_tile(it-1)
       corr = fa::ex2(m - mu);
       // fold the previous tile's P V into the running output (its MMAs also released the P buffer)
       if (it > 0) {
-        if (!tc::mbar_wait(o_full, (it - 1) & 1, abort_flag)) { ok = false; break; }
+        if (!tc::mbar_wait_warp(o_full, (it - 1) & 1, abort_flag)) { ok = false; break; }
         tc::tmem_fence_after();
         uint32_t w[64];
         tc::tmem_ld32_nowait(t_lane + 2 * T5_BN, w);
@@ -266,7 +265,7 @@ flash_attn_tc5_kernel(const __grid_constant__ CUtensorMap q_map, Flash5Args a) {
       if (lane == 0) { tc::mbar_arrive(&s_free[sb]); tc::mbar_arrive(p_full); }
     }
     if (ok && n_tiles > 0) {
-      if (tc::mbar_wait(o_full, (n_tiles - 1) & 1, abort_flag)) {
+      if (tc::mbar_wait_warp(o_full, (n_tiles - 1) & 1, abort_flag)) {
         tc::tmem_fence_after();
         uint32_t w[64];
         tc::tmem_ld32_nowait(t_lane + 2 * T5_BN, w);
@@ -280,7 +279,7 @@ flash_attn_tc5_kernel(const __grid_constant__ CUtensorMap q_map, Flash5Args a) {
     xmax[512 + hf * 128 + r] = l;
     __syncwarp();
     if (lane == 0) tc::mbar_arrive(pair_bar);
-    if (ok && tc::mbar_wait(pair_bar, n_tiles & 1, abort_flag)) l += xmax[512 + (hf ^ 1) * 128 + r];
+    if (ok && tc::mbar_wait_warp(pair_bar, n_tiles & 1, abort_flag)) l += xmax[512 + (hf ^ 1) * 128 + r];
     if (row_valid) {
       const float inv = (l > 0.f) ? 1.0f / l : 0.f;
       bf16* dst = a.out + (int64_t)(row0 + r) * a.out_cols + head * T5_DH + hf * 64;

@@ -24,7 +24,12 @@ template <> __device__ __forceinline__ bf16 from_f32<bf16>(float x) { return __f
 // the predecessor writes (or reads, if this kernel overwrites it) before pdl_wait(), which returns
 // once the predecessor grid has completed and its writes are visible.  pdl_launch_dependents()
 // lets the successor's CTAs be scheduled early.  Both are no-ops for ordinary launches.
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// The kernels read some of what their predecessor wrote with plain stores through bulk / tensor copies
+// (the async proxy): the proxy fence after the wait orders those copies behind the predecessor's writes.
+__device__ __forceinline__ void pdl_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("fence.proxy.async.global;" ::: "memory");
+}
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_prologue() { pdl_launch_dependents(); pdl_wait(); }
 

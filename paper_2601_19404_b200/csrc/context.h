@@ -41,6 +41,10 @@ struct Workspace {
   float* logits = nullptr; // [HR, V]
   uint32_t* sampler_w = nullptr;  // [max(max_seqs, max_groups), V] quantised sampler weights
   size_t sampler_w_rows = 0;
+  float* ssq = nullptr;          // [R][ssq_stride] partial sums of squares of the residual rows (fused RMSNorm)
+  int ssq_stride = 0;
+  float* ssq_h = nullptr;        // [HR] the same for the rows that go into the output head
+  int* tile_ctr = nullptr;       // split-K arrival counters (zero between launches)
   float* partial = nullptr;      // split-K partial sums
   size_t partial_elems = 0;
   float* attn_part = nullptr;    // decode attention partials
@@ -88,9 +92,17 @@ struct rpo_ctx {
   int* d_status = nullptr;
   int64_t launches = 0;
   int sm_count = 148;
+  int device = 0;                     // the CUDA device this context lives on
+  int ssq_parts = 1;                  // parts per row currently in ws.ssq (set by the kernel that wrote them)
   // options
+  int fused_split_limit = 1;          // ... for passes none of whose products splits K (more planes allowed: tests, sweeps)
+  int use_fused_layers = 1;           // 16-bit models: RMSNorm / RoPE / KV append / SwiGLU / residual as GEMM epilogues
   int use_tcgen05 = 1, use_tc_attention = 1, use_graph = 1;
-  int use_tc5_attention = 1, tc5_v_variant = 0;   // tcgen05 prefill attention (and the descriptor reading under test)
+  int use_tc5_attention = 1;          // tcgen05 attention for many-row passes
+  int use_tc5_decode = 0;             // tcgen05 decode attention (head_dim 128, <= 64 rows per group and KV head): parity-green, but
+                                      // measured 5-25 % slower per launch than the mma.sync kernel (1.8 us per 64-key tile): off by default
+  bool attn_dec5 = false;             // plan of the decode call being enqueued: prefix on tcgen05, suffix tiles in a pass of their own
+  int attn_suf_splits = 1;
   int use_cluster_merge = 0;          // decode attention: splits of a work item merge inside a thread-block cluster
                                       // (measured slower than partials + merge kernel at 8 splits: off by default)
   int launch_cluster_x = 0;           // cluster width of the next launch (0: none); cleared by the launch
@@ -105,6 +117,9 @@ struct rpo_ctx {
   void* host_stage[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
   size_t host_stage_bytes[5] = {0, 0, 0, 0, 0};
   int pending_splits = 0, pending_rows = 0;   // split-K partials of ws.x not yet reduced
+  // test tap (rpo_debug_tap): residual rows entering the layer stack and leaving every layer
+  float* tap_buf = nullptr;
+  int64_t tap_capacity = 0, tap_used = 0;
   // optional per-kernel timing: event pairs around every launch, tagged class + 16*phase
   struct ProfEvent { cudaEvent_t a, b; int tag; const char* label; };
   int profile = 0, prof_class = 0, prof_phase = 0;

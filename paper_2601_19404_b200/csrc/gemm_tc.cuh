@@ -21,22 +21,16 @@
 
 #include "common.cuh"
 #include "context.h"
+#include "gemm_epi.cuh"
 
 namespace rpo {
 
-enum TcEpilogue { TC_STORE_BF16 = 0, TC_STORE_F32 = 1, TC_ADD_F32 = 2, TC_SWIGLU = 3, TC_PARTIAL = 4 };
-
 constexpr int TC_BM = 128, TC_BK = 64;
-constexpr long long TC_TIMEOUT_CYCLES = 4000000000LL;   // ~2 s at 2 GHz
-
-struct TcParams {
-  void* C;              // output (type by epilogue)
-  int M, N, K;
-  int ldc;              // elements per output row
-  int tiles_m, tiles_n, splits, kb_per_split, kb_total;
-  int64_t split_stride; // TC_PARTIAL: elements between split planes
-  int* status;
-};
+// Limit of every bounded device-side wait, in SM clock cycles (~0.1 s at 2 GHz by default: a thousand
+// times the longest legitimate wait of these kernels).  One value per device and library image, shared
+// by all contexts on the device; rpo_set_option("wait_limit_cycles") changes it.
+constexpr long long TC_TIMEOUT_CYCLES_DEFAULT = 200000000LL;
+__device__ long long g_wait_limit_cycles = TC_TIMEOUT_CYCLES_DEFAULT;
 
 namespace tc {
 
@@ -61,12 +55,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait: false when the time limit ran out or another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
+  const long long t0 = clock64(), limit = g_wait_limit_cycles;
   while (!mbar_try_wait(bar, parity)) {
     if (*abort_flag) return false;
-    if (clock64() - t0 > TC_TIMEOUT_CYCLES) { *abort_flag = 1; return false; }
+    if (clock64() - t0 > limit) { *abort_flag = 1; return false; }
   }
   return true;
+}
+
+// The same for a whole warp that goes on to warp-wide (.sync.aligned) instructions: either every lane
+// saw the phase complete, or all of them give up together.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  const bool ok = mbar_wait(bar, parity, abort_flag);
+  return __all_sync(0xffffffffu, ok);
 }
 
 __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
@@ -117,6 +118,29 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// Registers back into tensor memory: 32 columns of this warp's 32 lanes.
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]),
+        "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]),
+        "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+
+// 16 columns of this warp's 32 lanes.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
 // tcgen05.ld without the wait: several loads can be in flight before one tmem_ld_wait().
 __device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t* r) {
   asm volatile(
@@ -131,56 +155,6 @@ __device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t* r) {
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 }  // namespace tc
-
-// Epilogue of one 32-column chunk of an accumulator row: r[0..31] are the float32 bit patterns of
-// columns col .. col+31 of output row `row`.
-// STREAM: the output is far larger than L2 and not read again by this kernel; streaming stores
-// keep it from evicting the operand tiles other CTAs are about to fetch.
-template <int EPI>
-__device__ __forceinline__ void tc_store_chunk(const TcParams& p, const uint32_t* r, int row, int col, int split,
-                                               const bool STREAM = false) {
-  if (row >= p.M || col >= p.N) return;
-  const int ncol = min(32, p.N - col);       // multiple of 8 (N % 8 == 0)
-  if (EPI == TC_STORE_BF16) {
-    bf16* dst = (bf16*)p.C + (int64_t)row * p.ldc + col;
-    for (int j = 0; j < ncol; j += 8) {
-      uint4 v;
-      __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
-      __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
-      __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]));
-      __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
-      v.x = *(uint32_t*)&h0; v.y = *(uint32_t*)&h1; v.z = *(uint32_t*)&h2; v.w = *(uint32_t*)&h3;
-      if (STREAM) __stcs((uint4*)(dst + j), v); else *(uint4*)(dst + j) = v;
-    }
-  } else if (EPI == TC_SWIGLU) {
-    // columns (2j, 2j+1) = (gate_j, up_j)  ->  out[row, col/2 + j]
-    bf16* dst = (bf16*)p.C + (int64_t)row * p.ldc + col / 2;
-    for (int j = 0; j < ncol; j += 16) {
-      uint32_t o[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const float g0 = __uint_as_float(r[j + 4 * q]), u0 = __uint_as_float(r[j + 4 * q + 1]);
-        const float g1 = __uint_as_float(r[j + 4 * q + 2]), u1 = __uint_as_float(r[j + 4 * q + 3]);
-        __nv_bfloat162 h = __floats2bfloat162_rn(g0 / (1.0f + __expf(-g0)) * u0, g1 / (1.0f + __expf(-g1)) * u1);
-        o[q] = *(uint32_t*)&h;
-      }
-      if (STREAM) __stcs((uint4*)(dst + j / 2), make_uint4(o[0], o[1], o[2], o[3]));
-      else *(uint4*)(dst + j / 2) = make_uint4(o[0], o[1], o[2], o[3]);
-    }
-  } else {
-    float* dst = (EPI == TC_PARTIAL) ? (float*)p.C + split * p.split_stride + (int64_t)row * p.ldc + col
-                                     : (float*)p.C + (int64_t)row * p.ldc + col;
-    for (int j = 0; j < ncol; j += 4) {
-      float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
-                             __uint_as_float(r[j + 3]));
-      if (EPI == TC_ADD_F32) {
-        const float4 o = *(float4*)(dst + j);
-        v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-      }
-      if (STREAM) __stcs((float4*)(dst + j), v); else *(float4*)(dst + j) = v;
-    }
-  }
-}
 
 template <int BN>
 struct TcCfg {
@@ -302,23 +276,64 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     pdl_wait();                                      // the epilogue reads / overwrites what earlier kernels produced
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
+    const bool split_k = p.splits > 1;
     for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
       const int split = it % p.splits, t = it / p.splits;
       const int tn = t % p.tiles_n, tm = t / p.tiles_n;
+      const int row = tm * TC_BM + quad * 32 + lane;
+      // what the epilogue needs besides the sums is requested before the wait for the accumulator
+      float scale = 1.f;
+      int4 meta = make_int4(-1, 0, 0, 0);
+      if (tc_epi_scaled(EPI) && !split_k) scale = epi_row_scale(p, row);
+      if (EPI == TC_QKV_ROPE && !split_k && row < p.M) meta = p.row_meta[row];
       if (!tc::mbar_wait(&acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc::tmem_fence_after();
-      const int row = tm * TC_BM + quad * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN);
+      if (split_k) {
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        uint32_t r[32];
-        tc::tmem_ld32(t_row + (uint32_t)c0, r);
-        tc_store_chunk<EPI>(p, r, row, tn * BN + c0, split);
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          uint32_t r[32];
+          tc::tmem_ld32(t_row + (uint32_t)c0, r);
+          tc_store_chunk<TC_PARTIAL>(p, r, row, tn * BN + c0, split);
+        }
+      } else if (EPI == TC_QKV_ROPE) {
+        const int half = p.head_dim >> 1;
+#pragma unroll 1
+        for (int h0 = 0; h0 < BN; h0 += p.head_dim) {
+#pragma unroll 1
+          for (int j = 0; j < half; j += 32) {
+            uint32_t lo[32], hi[32];
+            tc::tmem_ld32_nowait(t_row + (uint32_t)(h0 + j), lo);
+            tc::tmem_ld32_nowait(t_row + (uint32_t)(h0 + j + half), hi);
+            tc::tmem_ld_wait();
+            epi_rope_pair(p, lo, hi, row, tn * BN + h0 + j, scale, meta);
+          }
+        }
+      } else if (EPI == TC_ADD_NORM) {
+        float ss = 0.f;
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          uint32_t r[32];
+          tc::tmem_ld32(t_row + (uint32_t)c0, r);
+          ss += epi_add_norm_chunk(p, r, row, tn * BN + c0);
+        }
+        if (row < p.M) p.ssq_out[(int64_t)row * p.ssq_out_parts + tn] = ss;
+      } else {
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          uint32_t r[32];
+          tc::tmem_ld32(t_row + (uint32_t)c0, r);
+          if (EPI == TC_NSTORE_F32 || EPI == TC_NSWIGLU) epi_scaled_chunk<EPI>(p, r, row, tn * BN + c0, scale, false);
+          else tc_store_chunk<EPI>(p, r, row, tn * BN + c0, split);
+        }
       }
       tc::tmem_fence_before();
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(&acc_empty[acc]);
       if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+      // split-K with an epilogue of its own: the last warp to arrive at these 32 rows of the tile reduces them
+      if (split_k && EPI != TC_PARTIAL && epi_arrive_last(p, (tm * p.tiles_n + tn) * 4 + quad, lane))
+        epi_reduce_rows<EPI>(p, tm * TC_BM + quad * 32, tn * BN, BN, tn, lane);
     }
   }
 
@@ -400,14 +415,39 @@ inline bool tc_gemm_supported<bf16>(rpo_ctx* c, int M, int N, int K) {
   return s && s->encode && M >= 1 && (K % TC_BK) == 0 && (N % 16) == 0;
 }
 
+// Inputs / outputs of the fused epilogues (gemm_epi.cuh) that the plain GEMM call does not have.
+struct TcFuse {
+  const float* ssq_in = nullptr; int ssq_in_parts = 0; int norm_dim = 0; float eps = 0.f;       // TC_N*
+  float* ssq_out = nullptr; bf16* xg_out = nullptr; const float* gain = nullptr;                 // TC_ADD_NORM
+  int ssq_out_parts = 0;                                                                         //   (out) parts per row written
+  const int4* row_meta = nullptr; const float2* rope = nullptr; KVPool<bf16> pool = {}; int layer = 0, hq = 0, hkv = 0, head_dim = 0;   // TC_QKV_ROPE
+};
+
+constexpr int TC_CTR_CAPACITY = 1 << 16;     // arrival counters of a split-K launch (ints)
+
+// cudaFuncSetAttribute has to be made once per device, not once per process.
+inline bool tc_first_use_on_device(rpo_ctx* c, bool (&done)[64]) {
+  const int d = (c->device >= 0 && c->device < 64) ? c->device : 0;
+  if (done[d]) return false;
+  done[d] = true;
+  return true;
+}
+
+inline void tc_fill_fuse(rpo_ctx* c, TcParams& p, const TcFuse* f) {
+  p.planes = c->ws.partial; p.tile_ctr = c->ws.tile_ctr;
+  if (!f) return;
+  p.ssq_in = f->ssq_in; p.ssq_in_parts = f->ssq_in_parts; p.inv_norm_dim = f->norm_dim > 0 ? 1.0f / (float)f->norm_dim : 0.f; p.eps = f->eps;
+  p.ssq_out = f->ssq_out; p.xg_out = f->xg_out; p.gain = f->gain;
+  p.row_meta = f->row_meta; p.rope = f->rope; p.pool = f->pool; p.layer = f->layer; p.hq = f->hq; p.hkv = f->hkv; p.head_dim = f->head_dim;
+}
+
 template <int BN, int EPI>
 inline int tc_launch(rpo_ctx* c, const CUtensorMap* ma, const CUtensorMap* mw, const TcParams& p, int grid) {
   using Cfg = TcCfg<BN>;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done[64] = {};
+  if (tc_first_use_on_device(c, attr_done)) {
     if (cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
       return RPO_ERR_CUDA;
-    attr_done = true;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = Cfg::SMEM_BYTES; cfg.stream = c->stream;
@@ -425,6 +465,12 @@ inline int tc_launch_epi(rpo_ctx* c, int epi, const CUtensorMap* ma, const CUten
     case TC_STORE_F32: return tc_launch<BN, TC_STORE_F32>(c, ma, mw, p, grid);
     case TC_ADD_F32: return tc_launch<BN, TC_ADD_F32>(c, ma, mw, p, grid);
     case TC_SWIGLU: return tc_launch<BN, TC_SWIGLU>(c, ma, mw, p, grid);
+    case TC_NSTORE_F32: return tc_launch<BN, TC_NSTORE_F32>(c, ma, mw, p, grid);
+    case TC_NSWIGLU: return tc_launch<BN, TC_NSWIGLU>(c, ma, mw, p, grid);
+    case TC_ADD_NORM: return tc_launch<BN, TC_ADD_NORM>(c, ma, mw, p, grid);
+    case TC_QKV_ROPE:
+      if constexpr (BN % 64 == 0) return tc_launch<BN, TC_QKV_ROPE>(c, ma, mw, p, grid);
+      else return RPO_ERR_INVALID_ARG;
     default: return tc_launch<BN, TC_PARTIAL>(c, ma, mw, p, grid);
   }
 }
@@ -436,13 +482,15 @@ inline int tc_launch_epi(rpo_ctx* c, int epi, const CUtensorMap* ma, const CUten
 //     them unsplit; otherwise (tile_n, k-split) items are sized by a small cost model fitted to
 //     measurements: cost of an item ~ k-blocks x (W rows + a share for the A tile re-read from L2)
 //     + a pipeline-fill term, cost of the launch = rounds x item cost + a term per split plane
-//     (partials written and re-read by the reducing kernel).
+//     (partials written and re-read by whoever reduces them).
+// bn_multiple: the epilogue needs whole heads in a tile (RoPE pairs dims half a head apart).
 struct TcPlan { int bn, splits, kb_per_split; };
 
-inline TcPlan tc_plan(rpo_ctx* c, int M, int N, int K, int epi, bool allow_split) {
+inline TcPlan tc_plan(rpo_ctx* c, int M, int N, int K, int epi, bool allow_split, int bn_multiple = 1) {
   const int sms = c->sm_count, tiles_m = (M + TC_BM - 1) / TC_BM, kb_total = K / TC_BK;
   TcPlan best{256, 1, kb_total};
-  if (c->gemm_bn > 0) {                                  // test / sweep override
+  const bool self_reduce = tc_epi_fused(epi);           // the kernel's last-arriving warps reduce the planes
+  if (c->gemm_bn > 0 && c->gemm_bn < 384 && c->gemm_bn % bn_multiple == 0) {   // test / sweep override
     best.bn = c->gemm_bn;
     best.splits = (allow_split && c->gemm_splits > 0) ? std::min(c->gemm_splits, kb_total) : 1;
   } else if (tiles_m * ((N + 255) / 256) >= sms && tiles_m >= 4) {
@@ -453,7 +501,8 @@ inline TcPlan tc_plan(rpo_ctx* c, int M, int N, int K, int epi, bool allow_split
     static const int widths[] = {128, 96, 64, 32};
     double best_cost = 1e30;
     for (int bn : widths) {
-      if (epi == TC_SWIGLU && bn % 32) continue;
+      if ((epi == TC_SWIGLU || epi == TC_NSWIGLU) && bn % 32) continue;
+      if (bn % bn_multiple) continue;
       const int tiles = tiles_m * ((N + bn - 1) / bn);
       int max_splits = 1;
       if (allow_split && tiles < sms) max_splits = std::max(1, std::min(sms / tiles, kb_total / 2));
@@ -461,8 +510,11 @@ inline TcPlan tc_plan(rpo_ctx* c, int M, int N, int K, int epi, bool allow_split
         const int kbs = (kb_total + sp - 1) / sp;
         const int real = (kb_total + kbs - 1) / kbs;
         if (real > 1 && (size_t)real * M * N > c->ws.partial_elems) continue;
+        if (real > 1 && self_reduce && tiles * 4 > TC_CTR_CAPACITY) continue;
         const int rounds = (tiles * real + sms - 1) / sms;
-        const double cost = (double)rounds * (kbs * (bn + 40.0) + 600.0) + (real > 1 ? 60.0 * real : 0.0);
+        // planes reduced inside the kernel cost the last-arriving warp a serial pass per pair of planes
+        const double plane_cost = self_reduce ? 45.0 * bn / 128.0 * real : 60.0 * real;
+        const double cost = (double)rounds * (kbs * (bn + 40.0) + 600.0) + (real > 1 ? plane_cost : 0.0);
         if (cost < best_cost) { best_cost = cost; best.bn = bn; best.splits = real; }
       }
     }
@@ -473,24 +525,29 @@ inline TcPlan tc_plan(rpo_ctx* c, int M, int N, int K, int epi, bool allow_split
   return best;
 }
 
-// Plan and launch.  With allow_split the launch may write split-K partial planes [splits][M][N]
-// (float32) to ws.partial instead of applying `epi`; `splits_out` then receives the number of
-// planes (> 1) and the caller owns the reduction and the epilogue.
+// Plan and launch.  With allow_split the launch may split K.  For the fused epilogues (gemm_epi.cuh)
+// the kernel reduces the planes itself and the caller sees a finished result.  For the plain ones it
+// writes split-K partial planes [splits][M][N] (float32) to ws.partial instead of applying `epi`;
+// `splits_out` then receives the number of planes (> 1) and the caller owns the reduction.
 inline int tc_gemm_launch(rpo_ctx* c, const bf16* A, const bf16* W, void* C, int M, int N, int K, int epi, int ldc,
-                          bool allow_split, int* splits_out) {
+                          bool allow_split, int* splits_out, TcFuse* fuse = nullptr) {
   if (splits_out) *splits_out = 0;
   const int tiles_m = (M + TC_BM - 1) / TC_BM;
   const int kb_total = K / TC_BK;
   const int sms = c->sm_count;
-  const TcPlan plan = tc_plan(c, M, N, K, epi, allow_split);
+  const int bn_multiple = (epi == TC_QKV_ROPE && fuse) ? fuse->head_dim : 1;
+  const TcPlan plan = tc_plan(c, M, N, K, epi, allow_split, bn_multiple);
   const int bn = plan.bn, splits = plan.splits, kb_per_split = plan.kb_per_split;
   const int tiles_n = (N + bn - 1) / bn;
-  TcParams p;
+  TcParams p = {};
   p.C = C; p.M = M; p.N = N; p.K = K; p.ldc = ldc;
   p.tiles_m = tiles_m; p.tiles_n = tiles_n; p.splits = splits; p.kb_per_split = kb_per_split; p.kb_total = kb_total;
   p.split_stride = (int64_t)M * N; p.status = c->d_status;
+  tc_fill_fuse(c, p, fuse);
+  p.ssq_out_parts = tiles_n;
+  if (fuse) fuse->ssq_out_parts = tiles_n;
   int use_epi = epi;
-  if (splits > 1) { use_epi = TC_PARTIAL; p.C = c->ws.partial; p.ldc = N; if (splits_out) *splits_out = splits; }
+  if (splits > 1 && !tc_epi_fused(epi)) { use_epi = TC_PARTIAL; if (splits_out) *splits_out = splits; }
   const CUtensorMap* ma = tc_map(c, A, M, K, TC_BM);
   const CUtensorMap* mw = tc_map(c, W, N, K, bn);
   if (!ma || !mw) return RPO_ERR_CUDA;

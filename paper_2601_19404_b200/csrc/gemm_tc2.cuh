@@ -220,28 +220,71 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
     const int quad = warp & 3;
     const bool stream_out = p.M >= 2048;           // output far larger than L2: streaming stores
+    const bool split_k = p.splits > 1;
     pdl_wait();
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
     for (int it = cluster_id; it < n_items && ok; it += n_clusters) {
       int tm, tn;
       tc2_tile(it / p.splits, p.tiles_m, p.tiles_n, tm, tn);
+      // RM = 128: lane = row, 256 columns.  RM = 64: lanes 64.. hold columns 128..255 of rows 0..63.
+      const int row0 = tm * TM + (int)rank * RM + (RM == 128 ? quad * 32 : (quad & 1) * 32);
+      const int row = row0 + lane;
+      const int col_base = tn * 256 + (RM == 128 ? 0 : (quad >> 1) * 128);
+      const int part = RM == 128 ? tn : tn * 2 + (quad >> 1);         // column unit of this warp (TC_ADD_NORM statistics)
+      float scale = 1.f;
+      int4 meta = make_int4(-1, 0, 0, 0);
+      if (tc_epi_scaled(EPI) && !split_k) scale = epi_row_scale(p, row);
+      if (EPI == TC_QKV_ROPE && !split_k && row < p.M) meta = p.row_meta[row];
       if (!tc::mbar_wait(&acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc::tmem_fence_after();
-      // RM = 128: lane = row, 256 columns.  RM = 64: lanes 64.. hold columns 128..255 of rows 0..63.
-      const int row = tm * TM + (int)rank * RM + (RM == 128 ? quad * 32 : (quad & 1) * 32) + lane;
-      const int col_base = tn * 256 + (RM == 128 ? 0 : (quad >> 1) * 128);
       const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * Cfg::ACC_COLS);
+      if (split_k) {
 #pragma unroll 1
-      for (int c0 = 0; c0 < Cfg::ACC_COLS; c0 += 32) {
-        uint32_t r[32];
-        tc::tmem_ld32(t_row + (uint32_t)c0, r);
-        tc_store_chunk<EPI>(p, r, row, col_base + c0, it % p.splits, stream_out);
+        for (int c0 = 0; c0 < Cfg::ACC_COLS; c0 += 32) {
+          uint32_t r[32];
+          tc::tmem_ld32(t_row + (uint32_t)c0, r);
+          tc_store_chunk<TC_PARTIAL>(p, r, row, col_base + c0, it % p.splits, false);
+        }
+      } else if (EPI == TC_QKV_ROPE) {
+        const int half = p.head_dim >> 1;
+#pragma unroll 1
+        for (int h0 = 0; h0 < Cfg::ACC_COLS; h0 += p.head_dim) {
+#pragma unroll 1
+          for (int j = 0; j < half; j += 32) {
+            uint32_t lo[32], hi[32];
+            tc::tmem_ld32_nowait(t_row + (uint32_t)(h0 + j), lo);
+            tc::tmem_ld32_nowait(t_row + (uint32_t)(h0 + j + half), hi);
+            tc::tmem_ld_wait();
+            epi_rope_pair(p, lo, hi, row, col_base + h0 + j, scale, meta);
+          }
+        }
+      } else if (EPI == TC_ADD_NORM) {
+        float ss = 0.f;
+#pragma unroll 1
+        for (int c0 = 0; c0 < Cfg::ACC_COLS; c0 += 32) {
+          uint32_t r[32];
+          tc::tmem_ld32(t_row + (uint32_t)c0, r);
+          ss += epi_add_norm_chunk(p, r, row, col_base + c0);
+        }
+        if (row < p.M) p.ssq_out[(int64_t)row * p.ssq_out_parts + part] = ss;
+      } else {
+#pragma unroll 1
+        for (int c0 = 0; c0 < Cfg::ACC_COLS; c0 += 32) {
+          uint32_t r[32];
+          tc::tmem_ld32(t_row + (uint32_t)c0, r);
+          if (EPI == TC_NSTORE_F32 || EPI == TC_NSWIGLU) epi_scaled_chunk<EPI>(p, r, row, col_base + c0, scale, stream_out);
+          else tc_store_chunk<EPI>(p, r, row, col_base + c0, it % p.splits, stream_out);
+        }
       }
       tc::tmem_fence_before();
       __syncwarp();
       if (lane == 0) tc::mbar_arrive_cluster(tc::map_to_rank(tc::smem_u32(&acc_empty[acc]), 0));
       if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+      // split-K with an epilogue of its own: the last warp to arrive at this 32-row unit reduces it
+      if (split_k && EPI != TC_PARTIAL &&
+          epi_arrive_last(p, (((tm * p.tiles_n + tn) * 2 + (int)rank) * 4 + quad), lane))
+        epi_reduce_rows<EPI>(p, row0, col_base, Cfg::ACC_COLS, part, lane);
     }
   }
 
@@ -267,7 +310,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 template <int EPI, int RM>
 inline int tc2_launch(rpo_ctx* c, const CUtensorMap* ma, const CUtensorMap* mw, const TcParams& p) {
   using Cfg = Tc2Cfg<RM>;
-  static int max_clusters = -1;
+  static int max_clusters_dev[64];
+  static bool init_done[64] = {};
+  const int dev_i = (c->device >= 0 && c->device < 64) ? c->device : 0;
+  if (!init_done[dev_i]) { max_clusters_dev[dev_i] = -1; init_done[dev_i] = true; }
+  int& max_clusters = max_clusters_dev[dev_i];
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -327,22 +374,27 @@ inline bool tc2_wanted(rpo_ctx* c, int M, int N, int K, bool allow_split) {
   return tiles * sp >= c->sm_count / 2 - 10;
 }
 
-// With allow_split the launch may leave split-K partial planes [splits][M][N] in ws.partial
-// instead of applying `epi`; *splits_out then holds the number of planes (> 1).
+// With allow_split the launch may split K: the fused epilogues (gemm_epi.cuh) reduce the planes inside
+// the kernel; for the plain ones the planes [splits][M][N] stay in ws.partial instead of applying `epi`
+// and *splits_out holds their number (> 1).
 inline int tc2_gemm_launch(rpo_ctx* c, const bf16* A, const bf16* W, void* C, int M, int N, int K, int epi, int ldc,
-                           bool allow_split, int* splits_out) {
+                           bool allow_split, int* splits_out, TcFuse* fuse = nullptr) {
   if (splits_out) *splits_out = 0;
   const int rm = tc2_rows(c, M), tm = 2 * rm;
-  TcParams p;
+  TcParams p = {};
   p.C = C; p.M = M; p.N = N; p.K = K; p.ldc = ldc;
   p.tiles_m = (M + tm - 1) / tm; p.tiles_n = (N + 255) / 256; p.kb_total = K / TC_BK;
   int splits = (M <= 128 && c->gemm_bn == 0) ? 1 : tc2_splits(c, M, N, K, allow_split);
+  if (tc_epi_fused(epi) && p.tiles_m * p.tiles_n * 8 > TC_CTR_CAPACITY) splits = 1;
   p.kb_per_split = (p.kb_total + splits - 1) / splits;
   splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
   if (splits > 1 && (size_t)splits * M * N > c->ws.partial_elems) { splits = 1; p.kb_per_split = p.kb_total; }
   p.splits = splits;
   p.split_stride = (int64_t)M * N; p.status = c->d_status;
-  if (splits > 1) { epi = TC_PARTIAL; p.C = c->ws.partial; p.ldc = N; if (splits_out) *splits_out = splits; }
+  tc_fill_fuse(c, p, fuse);
+  p.ssq_out_parts = rm == 128 ? p.tiles_n : 2 * p.tiles_n;
+  if (fuse) fuse->ssq_out_parts = p.ssq_out_parts;
+  if (splits > 1 && !tc_epi_fused(epi)) { epi = TC_PARTIAL; if (splits_out) *splits_out = splits; }
   const CUtensorMap* ma = tc_map(c, A, M, K, rm);
   const CUtensorMap* mw = tc_map(c, W, N, K, 128);
   if (!ma || !mw) return RPO_ERR_CUDA;
@@ -352,6 +404,10 @@ inline int tc2_gemm_launch(rpo_ctx* c, const bf16* A, const bf16* W, void* C, in
       case TC_STORE_F32: return tc2_launch<TC_STORE_F32, 64>(c, ma, mw, p);
       case TC_ADD_F32: return tc2_launch<TC_ADD_F32, 64>(c, ma, mw, p);
       case TC_SWIGLU: return tc2_launch<TC_SWIGLU, 64>(c, ma, mw, p);
+      case TC_NSTORE_F32: return tc2_launch<TC_NSTORE_F32, 64>(c, ma, mw, p);
+      case TC_NSWIGLU: return tc2_launch<TC_NSWIGLU, 64>(c, ma, mw, p);
+      case TC_QKV_ROPE: return tc2_launch<TC_QKV_ROPE, 64>(c, ma, mw, p);
+      case TC_ADD_NORM: return tc2_launch<TC_ADD_NORM, 64>(c, ma, mw, p);
       default: return tc2_launch<TC_PARTIAL, 64>(c, ma, mw, p);
     }
   }
@@ -360,6 +416,10 @@ inline int tc2_gemm_launch(rpo_ctx* c, const bf16* A, const bf16* W, void* C, in
     case TC_STORE_F32: return tc2_launch<TC_STORE_F32, 128>(c, ma, mw, p);
     case TC_ADD_F32: return tc2_launch<TC_ADD_F32, 128>(c, ma, mw, p);
     case TC_SWIGLU: return tc2_launch<TC_SWIGLU, 128>(c, ma, mw, p);
+    case TC_NSTORE_F32: return tc2_launch<TC_NSTORE_F32, 128>(c, ma, mw, p);
+    case TC_NSWIGLU: return tc2_launch<TC_NSWIGLU, 128>(c, ma, mw, p);
+    case TC_QKV_ROPE: return tc2_launch<TC_QKV_ROPE, 128>(c, ma, mw, p);
+    case TC_ADD_NORM: return tc2_launch<TC_ADD_NORM, 128>(c, ma, mw, p);
     default: return tc2_launch<TC_PARTIAL, 128>(c, ma, mw, p);
   }
 }

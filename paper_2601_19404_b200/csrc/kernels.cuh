@@ -82,6 +82,20 @@ __global__ void fill_kernel(T* dst, int64_t n, float v) {
     dst[i] = from_f32<T>(v);
 }
 
+__device__ __forceinline__ int lane_id() { return threadIdx.x & 31; }
+// Four consecutive outputs of type T (8 or 16 bytes, aligned) in one store.
+template <typename T>
+__device__ __forceinline__ void store4(T* dst, float a, float b, float c, float d);
+template <>
+__device__ __forceinline__ void store4<float>(float* dst, float a, float b, float c, float d) {
+  *reinterpret_cast<float4*>(dst) = make_float4(a, b, c, d);
+}
+template <>
+__device__ __forceinline__ void store4<bf16>(bf16* dst, float a, float b, float c, float d) {
+  const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+  *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+}
+
 // cos/sin table [max_positions][head_dim/2], angles in float64.
 __global__ void rope_table_kernel(float2* __restrict__ tab, int max_pos, int half, double base) {
   pdl_prologue();
@@ -106,10 +120,24 @@ struct RowMetaArgs {
   int n_blocks, max_pos;
   int4* row_meta;                     // out: (position, block, slot in block, 0); x = -1: inactive row
 };
+// Sum of v over the block's threads, in a fixed order (same bits on every run); every thread gets it.
+__device__ __forceinline__ float block_sum_fixed(float v, float* red) {
+  v = warp_sum(v);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float t = 0.f;
+  for (int i = 0; i < (int)(blockDim.x >> 5); ++i) t += red[i];
+  return t;
+}
+
+// With xg != NULL (the fused-epilogue layer stack, 16-bit models) the kernel also prepares the first
+// RMSNorm: xg[r,:] = bf16(x[r,:] * gain) and ssq[r] = sum x[r,:]^2 (one part per row).
 template <typename T>
 __global__ void embed_kernel(const int32_t* __restrict__ tokens, const T* __restrict__ E, float* __restrict__ x,
-                             int rows, int d, int vocab, int* status, int32_t* step_ctr, RowMetaArgs m) {
+                             int rows, int d, int vocab, int* status, int32_t* step_ctr, RowMetaArgs m,
+                             const float* __restrict__ gain, bf16* __restrict__ xg, float* __restrict__ ssq) {
   pdl_prologue();
+  __shared__ float red[32];
   const int r = blockIdx.x;
   if (step_ctr && r == 0 && threadIdx.x == 0) *step_ctr += 1;
   if (r >= rows) return;
@@ -132,7 +160,38 @@ __global__ void embed_kernel(const int32_t* __restrict__ tokens, const T* __rest
   }
   const T* src = E + (int64_t)tok * d;
   float* dst = x + (int64_t)r * d;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = to_f32(src[i]);
+  if (!xg) {
+    for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = to_f32(src[i]);
+    return;
+  }
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    const float v = to_f32(src[i]);
+    dst[i] = v;
+    xg[(int64_t)r * d + i] = __float2bfloat16_rn(v * gain[i]);
+    ss += v * v;
+  }
+  ss = block_sum_fixed(ss, red);
+  if (threadIdx.x == 0) ssq[r] = ss;
+}
+
+// The RMSNorm preparation alone, for residual rows that no GEMM epilogue produced (the rows that go
+// into the output head): xg[r,:] = bf16(x[r,:] * gain), ssq[r] = sum x[r,:]^2.
+__global__ void norm_prep_kernel(const float* __restrict__ x, const float* __restrict__ gain, bf16* __restrict__ xg,
+                                 float* __restrict__ ssq, int rows, int d) {
+  pdl_prologue();
+  __shared__ float red[32];
+  const int r = blockIdx.x;
+  if (r >= rows) return;
+  float ss = 0.f;
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    const float4 v = *reinterpret_cast<const float4*>(x + (int64_t)r * d + i);
+    const float4 g = *reinterpret_cast<const float4*>(gain + i);
+    store4<bf16>(xg + (int64_t)r * d + i, v.x * g.x, v.y * g.y, v.z * g.z, v.w * g.w);
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  ss = block_sum_fixed(ss, red);
+  if (threadIdx.x == 0) ssq[r] = ss;
 }
 
 // dst[r,:] = src[idx[r],:]  (float32 rows; idx may be NULL = identity)
@@ -147,20 +206,6 @@ __global__ void gather_rows_f32_kernel(const float* __restrict__ src, const int3
     return;
   }
   for (int i = threadIdx.x; i < d; i += blockDim.x) dst[(int64_t)r * d + i] = src[(int64_t)s * d + i];
-}
-
-__device__ __forceinline__ int lane_id() { return threadIdx.x & 31; }
-// Four consecutive outputs of type T (8 or 16 bytes, aligned) in one store.
-template <typename T>
-__device__ __forceinline__ void store4(T* dst, float a, float b, float c, float d);
-template <>
-__device__ __forceinline__ void store4<float>(float* dst, float a, float b, float c, float d) {
-  *reinterpret_cast<float4*>(dst) = make_float4(a, b, c, d);
-}
-template <>
-__device__ __forceinline__ void store4<bf16>(bf16* dst, float a, float b, float c, float d) {
-  const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
-  *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
 }
 
 // RMSNorm of the float32 residual stream, one CTA per row, 128-bit accesses (d % 4 == 0):

@@ -13,6 +13,7 @@
 
 #include "attn_tc.cuh"
 #include "attn_tc5.cuh"
+#include "attn_dec5.cuh"
 #include "context.h"
 #include "gemm_tc.cuh"
 #include "gemm_tc2.cuh"
@@ -211,6 +212,7 @@ extern "C" int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limit
   c->qkv_cols = (s.n_q_heads + 2 * s.n_kv_heads) * s.head_dim;
   int dev = 0;
   cudaGetDevice(&dev);
+  c->device = dev;
   cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev);
   const size_t e = c->esz;
   const int d = s.d_model, dh = s.head_dim, F = s.d_ffn, V = s.vocab, qo = s.n_q_heads * dh;
@@ -297,6 +299,11 @@ extern "C" int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limit
   ALLOC(w.attn_part, w.attn_part_elems * 4);
   w.partial_elems = (size_t)c->sm_count * 128 * 256;
   ALLOC(w.partial, w.partial_elems * 4);
+  w.ssq_stride = std::max((d + 31) / 32, 2 * ((d + 255) / 256));
+  ALLOC(w.ssq, (size_t)w.R * w.ssq_stride * 4);
+  ALLOC(w.ssq_h, (size_t)w.HR * 4);
+  ALLOC(w.tile_ctr, (size_t)TC_CTR_CAPACITY * 4);
+  if (rc == RPO_OK && cudaMemsetAsync(w.tile_ctr, 0, (size_t)TC_CTR_CAPACITY * 4, c->stream) != cudaSuccess) { cudaGetLastError(); rc = RPO_ERR_CUDA; }
   if (rc == RPO_OK) rc = tc_create(c);
   // The attention kernels mask keys beyond a segment's end instead of zero-filling them, so the
   // pool must never hold NaN/Inf bit patterns: start from zeros.
@@ -396,6 +403,21 @@ static int flush_partials(rpo_ctx* c) {
 // allow_split: the tensor-core kernel may leave split-K partial planes in ws.partial instead of
 // applying the epilogue.  For EPI_ADD_F32 on ws.x the next RMSNorm (or flush_partials) folds them
 // in; for other epilogues the caller must pass splits_out and reduce the planes itself.
+// Fused epilogues (TC_N*, TC_QKV_ROPE, TC_ADD_NORM; 16-bit models on the tensor-core kernels only):
+// C = A W^T with the layer's elementwise work done in the epilogue; split-K is reduced inside the kernel.
+static int gemm_fused(rpo_ctx* c, const bf16* A, const bf16* W, void* C, int M, int N, int K, int tc_epi, int ldc, TcFuse& fuse) {
+  if (M <= 0) return RPO_OK;
+  ProfScope ps(c, KC_GEMM);
+  static const char* labels[] = {"gemm", "gemm", "gemm", "gemm", "gemm", "gemm (1/rms, float32 store: output head)",
+                                 "gemm (1/rms, SwiGLU: gate/up)", "gemm (1/rms, RoPE, KV append: qkv)", "gemm (residual add, next norm: O / down)"};
+  prof_begin(c, labels[tc_epi]);
+  const int rc = tc2_wanted(c, M, N, K, true) ? tc2_gemm_launch(c, A, W, C, M, N, K, tc_epi, ldc, true, nullptr, &fuse)
+                                              : tc_gemm_launch(c, A, W, C, M, N, K, tc_epi, ldc, true, nullptr, &fuse);
+  prof_end(c);
+  c->launches++;
+  return rc;
+}
+
 template <typename T>
 static int gemm(rpo_ctx* c, const T* A, const T* W, void* C, int M, int N, int K, int epi, int impl = 0,
                 bool allow_split = false, int* splits_out = nullptr) {
@@ -451,11 +473,9 @@ static int rmsnorm(rpo_ctx* c, float* x, const float* g, T* h, int rows) {
 template <int DH, int MODE, bool CLM = false>
 static int launch_flash(rpo_ctx* c, const FlashArgs& a, dim3 grid) {
   constexpr int smem = FaCfg<MODE>::template smem_bytes<DH>();
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done[64] = {};
+  if (tc_first_use_on_device(c, attr_done))
     CUDA_TRY(cudaFuncSetAttribute(flash_attn_kernel<DH, MODE, CLM>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    attr_done = true;
-  }
   if (CLM) c->launch_cluster_x = a.n_splits;         // the splits of a work item are consecutive along x
   LAUNCH(c, (flash_attn_kernel<DH, MODE, CLM>), grid, FaCfg<MODE>::THREADS + 32, smem, a);
   return RPO_OK;
@@ -494,12 +514,10 @@ static int attention(rpo_ctx* c, int layer, int rows) {
         f.out = (bf16*)w.attn; f.out_cols = s.n_q_heads * s.head_dim; f.row_seq = w.row_seq; f.row_t = w.row_t;
         f.seqs = (const SeqDesc*)w.seqs; f.block_table = c->d_block_table; f.pool = kv_pool<bf16>(c); f.layer = layer;
         f.hq = s.n_q_heads; f.hkv = s.n_kv_heads; f.scale_log2 = scale * 1.4426950408889634f; f.tiles = (const int2*)w.tiles;
-        f.q_col0 = 0; f.v_desc_variant = c->tc5_v_variant; f.status = c->d_status;
-        static bool attr_done = false;
-        if (!attr_done) {
+        f.q_col0 = 0; f.status = c->d_status;
+        static bool attr_done[64] = {};
+        if (tc_first_use_on_device(c, attr_done))
           CUDA_TRY(cudaFuncSetAttribute(flash_attn_tc5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, T5_SMEM));
-          attr_done = true;
-        }
         LAUNCH(c, flash_attn_tc5_kernel, dim3(s.n_q_heads, c->attn_tiles), 320, T5_SMEM, *qm, f);
         return RPO_OK;
       }
@@ -508,6 +526,24 @@ static int attention(rpo_ctx* c, int layer, int rows) {
         return s.head_dim == 128 ? launch_flash<128, FA_ROWS>(c, a, grid) : launch_flash<64, FA_ROWS>(c, a, grid);
       }
       const int rep = s.n_q_heads / s.n_kv_heads;
+      a.n_slots = a.n_splits; a.slot_base = 0; a.skip_prefix = 0;
+      if (c->attn_dec5) {
+        // one tcgen05 work item per (group, KV head, split): its prefix split, then its share of the suffix tiles
+        Decode5Args d5;
+        memset(&d5, 0, sizeof(d5));
+        d5.qkv = (const bf16*)w.qkv; d5.qkv_cols = c->qkv_cols; d5.part_ml = a.part_ml; d5.part_o = a.part_o; d5.n_slots = c->attn_splits;
+        d5.pfx_tbl = w.pfx_tbl; d5.pfx_stride = w.pfx_stride; d5.seqs = (const SeqDesc*)w.seqs; d5.row_t = w.row_t;
+        d5.block_table = c->d_block_table; d5.pool = kv_pool<bf16>(c);
+        d5.layer = layer; d5.hq = s.n_q_heads; d5.hkv = s.n_kv_heads; d5.G = c->attn_G; d5.scale_log2 = a.scale_log2;
+        d5.n_splits = c->attn_splits; d5.split_chunk = c->attn_split_chunk; d5.status = c->d_status;
+        static bool d5_attr[64] = {};
+        if (tc_first_use_on_device(c, d5_attr))
+          CUDA_TRY(cudaFuncSetAttribute(flash_decode_tc5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, D5_SMEM));
+        LAUNCH(c, flash_decode_tc5_kernel, dim3(c->attn_groups * c->attn_splits, s.n_kv_heads), 320, D5_SMEM, d5);
+        const int mgrid = ceil_div((int64_t)rows * s.n_q_heads, 4);
+        LAUNCH(c, (attn_decode_merge_kernel<128>), mgrid, 128, 0, a.out, a.part_ml, a.part_o, c->attn_splits, w.row_t, rows, a.hq);
+        return RPO_OK;
+      }
       dim3 grid(c->attn_groups * ceil_div(c->attn_G * rep, FA_BM) * c->attn_splits, s.n_kv_heads);
       if (c->use_cluster_merge && cluster_mergeable(a.n_splits))
         return s.head_dim == 128 ? launch_flash<128, FA_SHARED, true>(c, a, grid) : launch_flash<64, FA_SHARED, true>(c, a, grid);
@@ -554,14 +590,38 @@ static int upload_row_tiles(rpo_ctx* c, const std::vector<int>& rows_per_seq) {
   return RPO_OK;
 }
 
+// Test tap (rpo_debug_tap): the residual rows of the pass are appended to the caller's buffer.
+static int tap_copy(rpo_ctx* c, const void* src, int64_t bytes) {
+  const int64_t n = (bytes + 3) / 4;
+  if (c->tap_used + n > c->tap_capacity) return RPO_ERR_LIMIT;
+  CUDA_TRY(cudaMemcpyAsync(c->tap_buf + c->tap_used, src, (size_t)bytes, cudaMemcpyDeviceToDevice, c->stream));
+  c->tap_used += n;
+  return RPO_OK;
+}
+static int tap_rows(rpo_ctx* c, int rows) {            // the residual rows
+  if (!c->tap_buf) return RPO_OK;
+  RPO_TRY(flush_partials(c));
+  return tap_copy(c, c->ws.x, (int64_t)rows * c->shape.d_model * 4);
+}
+static int tap_attn(rpo_ctx* c, int rows) {            // the attention output rows, in the storage type
+  if (!c->tap_buf) return RPO_OK;
+  return tap_copy(c, c->ws.attn, (int64_t)rows * c->shape.n_q_heads * c->shape.head_dim * (int64_t)c->esz);
+}
+
+static int read_status(rpo_ctx* c, int* word);
+static bool fused_layers(rpo_ctx* c, int rows);
+static int run_layers_fused(rpo_ctx* c, int rows);
+
 // The layer stack over `rows` rows of ws.x, whose (sequence, private index) metadata sits in
 // ws.row_seq / ws.row_t and whose sequence descriptors sit in ws.seqs.
 // flush = false leaves the last layer's split-K partials pending for the caller's next RMSNorm on ws.x.
 template <typename T>
 static int run_layers(rpo_ctx* c, int rows, bool flush = true) {
+  if (fused_layers(c, rows)) return run_layers_fused(c, rows);
   const rpo_shape& s = c->shape;
   Workspace& w = c->ws;
   const int d = s.d_model, F = s.d_ffn, qo = s.n_q_heads * s.head_dim;
+  RPO_TRY(tap_rows(c, rows));
   for (int l = 0; l < s.n_layers; ++l) {
     const LayerWeights& L = c->layers[l];
     RPO_TRY(rmsnorm<T>(c, w.x, L.g1, (T*)w.h, rows));
@@ -572,6 +632,7 @@ static int run_layers(rpo_ctx* c, int rows, bool flush = true) {
            (const int4*)w.row_meta, (const float2*)c->d_rope, kv_pool<T>(c), l, rows, s.n_q_heads, s.n_kv_heads,
            qkv_splits > 1 ? (const float*)w.partial : (const float*)nullptr, qkv_splits, (int64_t)rows * c->qkv_cols); }
     RPO_TRY(attention<T>(c, l, rows));
+    RPO_TRY(tap_attn(c, rows));
     RPO_TRY(gemm<T>(c, (const T*)w.attn, (const T*)L.wo, w.x, rows, d, qo, EPI_ADD_F32, 0, true));
     RPO_TRY(rmsnorm<T>(c, w.x, L.g2, (T*)w.h, rows));
     if (c->use_tcgen05 && tc_gemm_supported<T>(c, rows, 2 * F, d) && F % 8 == 0) {
@@ -581,14 +642,103 @@ static int run_layers(rpo_ctx* c, int rows, bool flush = true) {
       LAUNCH(c, swiglu_kernel<T>, grid_for((int64_t)rows * F, 256), 256, 0, (const T*)w.gu, (T*)w.act, (int64_t)rows * F);
     }
     RPO_TRY(gemm<T>(c, (const T*)w.act, (const T*)L.wd, w.x, rows, d, F, EPI_ADD_F32, 0, true));
+    RPO_TRY(tap_rows(c, rows));
   }
   return flush ? flush_partials(c) : RPO_OK;
+}
+
+// True when the layer stack runs with the fused GEMM epilogues (gemm_epi.cuh): 16-bit model, tensor-
+// core kernels on, every product of the layer in the shape the tensor-core kernel takes.
+// Split-K factor the planner would pick for a fused product of `rows` rows.
+static int fused_splits(rpo_ctx* c, int rows, int N, int K, int epi, int bn_multiple) {
+  if (tc2_wanted(c, rows, N, K, true)) return (rows <= 128 && c->gemm_bn == 0) ? 1 : tc2_splits(c, rows, N, K, true);
+  return tc_plan(c, rows, N, K, epi, true, bn_multiple).splits;
+}
+
+static bool fused_layers(rpo_ctx* c, int rows) {
+  const rpo_shape& s = c->shape;
+  if (!c->bf16 || !c->use_tcgen05 || !c->use_fused_layers) return false;
+  const int qo = s.n_q_heads * s.head_dim;
+  if (!(tc_gemm_supported<bf16>(c, 1, c->qkv_cols, s.d_model) && tc_gemm_supported<bf16>(c, 1, s.d_model, qo) &&
+        tc_gemm_supported<bf16>(c, 1, 2 * s.d_ffn, s.d_model) && tc_gemm_supported<bf16>(c, 1, s.d_model, s.d_ffn) &&
+        tc_gemm_supported<bf16>(c, 1, s.vocab, s.d_model) && s.d_ffn % 8 == 0))
+    return false;
+  if (c->use_fused_layers >= 2) return true;           // forced (tests)
+  // A split-K launch with a fused epilogue is reduced by the last warp to arrive at each 32-row unit, so
+  // a few warps per tile do alone what a reduction kernel spreads over the whole machine: measured 12-17 %
+  // slower per decode forward (256 / 512 sequences, 2-5 planes), neutral at 128 sequences.  Passes whose
+  // products split K (decode batches) therefore keep the unfused kernels; prefill and teacher-forced
+  // passes, which never split, run fused (-3 % / -9 % measured).
+  const int lim = c->fused_split_limit;
+  return fused_splits(c, rows, c->qkv_cols, s.d_model, TC_QKV_ROPE, s.head_dim) <= lim &&
+         fused_splits(c, rows, s.d_model, qo, TC_ADD_NORM, 1) <= lim && fused_splits(c, rows, s.d_model, s.d_ffn, TC_ADD_NORM, 1) <= lim;
+}
+
+// What embed_kernel writes besides x when the layers are fused: xg = bf16(x * g1 of layer 0), sum of squares.
+static void embed_norm_args(rpo_ctx* c, int rows, const float*& gain, bf16*& xg, float*& ssq) {
+  gain = nullptr; xg = nullptr; ssq = nullptr;
+  if (!fused_layers(c, rows) || c->shape.n_layers == 0) return;
+  gain = c->layers[0].g1; xg = (bf16*)c->ws.h; ssq = c->ws.ssq;
+  c->ssq_parts = 1;
+}
+
+static TcFuse fuse_norm_in(rpo_ctx* c) {             // the consumer side of a fused RMSNorm
+  TcFuse f;
+  f.ssq_in = c->ws.ssq; f.ssq_in_parts = c->ssq_parts; f.norm_dim = c->shape.d_model; f.eps = c->shape.rms_eps;
+  return f;
+}
+
+// The layer stack with five kernels per layer.  On entry ws.x holds the residual rows, ws.h = bf16(x *
+// g1 of layer 0) and ws.ssq their sums of squares (c->ssq_parts parts per row).  On return ws.h =
+// bf16(x * final_gain) and ws.ssq belong to the rows leaving the last layer (the output head's input).
+static int run_layers_fused(rpo_ctx* c, int rows) {
+  const rpo_shape& s = c->shape;
+  Workspace& w = c->ws;
+  const int d = s.d_model, F = s.d_ffn, qo = s.n_q_heads * s.head_dim;
+  RPO_TRY(tap_rows(c, rows));
+  for (int l = 0; l < s.n_layers; ++l) {
+    const LayerWeights& L = c->layers[l];
+    {
+      TcFuse f = fuse_norm_in(c);
+      f.row_meta = (const int4*)w.row_meta; f.rope = (const float2*)c->d_rope; f.pool = kv_pool<bf16>(c); f.layer = l;
+      f.hq = s.n_q_heads; f.hkv = s.n_kv_heads; f.head_dim = s.head_dim;
+      RPO_TRY(gemm_fused(c, (const bf16*)w.h, (const bf16*)L.wqkv, w.qkv, rows, c->qkv_cols, d, TC_QKV_ROPE, c->qkv_cols, f));
+    }
+    RPO_TRY(attention<bf16>(c, l, rows));
+    RPO_TRY(tap_attn(c, rows));
+    {
+      TcFuse f;
+      f.ssq_out = w.ssq; f.xg_out = (bf16*)w.h; f.gain = L.g2;
+      RPO_TRY(gemm_fused(c, (const bf16*)w.attn, (const bf16*)L.wo, w.x, rows, d, qo, TC_ADD_NORM, d, f));
+      c->ssq_parts = f.ssq_out_parts;
+    }
+    {
+      TcFuse f = fuse_norm_in(c);
+      RPO_TRY(gemm_fused(c, (const bf16*)w.h, (const bf16*)L.wgu, w.act, rows, 2 * F, d, TC_NSWIGLU, F, f));
+    }
+    {
+      TcFuse f;
+      f.ssq_out = w.ssq; f.xg_out = (bf16*)w.h; f.gain = (l + 1 < s.n_layers) ? c->layers[l + 1].g1 : c->gf;
+      RPO_TRY(gemm_fused(c, (const bf16*)w.act, (const bf16*)L.wd, w.x, rows, d, F, TC_ADD_NORM, d, f));
+      c->ssq_parts = f.ssq_out_parts;
+    }
+    RPO_TRY(tap_rows(c, rows));
+  }
+  return RPO_OK;
 }
 
 // logits[n, V] (float32, ws.logits) from n residual rows in ws.xh.
 template <typename T>
 static int head(rpo_ctx* c, int n) {
   Workspace& w = c->ws;
+  if (fused_layers(c, 1 << 20)) {                      // (many rows: no split question) the output head takes bf16(x * g) rows
+    ProfScope ps(c, KC_NORM);
+    LAUNCH(c, norm_prep_kernel, n, 128, 0, (const float*)w.xh, (const float*)c->gf, (bf16*)w.hh, w.ssq_h, n, c->shape.d_model);
+    TcFuse f;
+    f.ssq_in = w.ssq_h; f.ssq_in_parts = 1; f.norm_dim = c->shape.d_model; f.eps = c->shape.rms_eps;
+    return gemm_fused(c, (const bf16*)w.hh, (const bf16*)c->lm_head, w.logits, n, c->shape.vocab, c->shape.d_model, TC_NSTORE_F32,
+                      c->shape.vocab, f);
+  }
   RPO_TRY(rmsnorm<T>(c, w.xh, c->gf, (T*)w.hh, n));
   return gemm<T>(c, (const T*)w.hh, (const T*)c->lm_head, w.logits, n, c->shape.vocab, c->shape.d_model, EPI_STORE_F32);
 }
@@ -637,8 +787,10 @@ static int prefill_chunk(rpo_ctx* c, const int32_t* d_tokens, int tok0, const st
   CUDA_TRY(cudaMemcpyAsync(w.row_t, row_t.data(), (size_t)rows * 4, cudaMemcpyHostToDevice, c->stream));
   CUDA_TRY(cudaMemcpyAsync(w.seqs, sd.data(), (size_t)n * sizeof(SeqDesc), cudaMemcpyHostToDevice, c->stream));
   RPO_TRY(upload_row_tiles(c, lens));
+  const float* e_gain; bf16* e_xg; float* e_ssq;
+  embed_norm_args(c, rows, e_gain, e_xg, e_ssq);
   LAUNCH(c, embed_kernel<T>, rows, 128, 0, d_tokens + tok0, (const T*)c->embed, w.x, rows, c->shape.d_model,
-         c->shape.vocab, c->d_status, (int32_t*)nullptr, row_meta_args(c));
+         c->shape.vocab, c->d_status, (int32_t*)nullptr, row_meta_args(c), e_gain, e_xg, e_ssq);
   RPO_TRY(run_layers<T>(c, rows));
   // keep the residual stream of every group's last prefix token: step-0 logits come from it
   for (int i = 0; i < n; ++i)
@@ -703,11 +855,9 @@ extern "C" int rpo_release_groups(rpo_ctx* c, int32_t n_groups, const rpo_group*
 // decode
 // ---------------------------------------------------------------------------------------------
 static int launch_sampler(rpo_ctx* c, int n_rows, const SamplerArgs& a) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done[64] = {};
+  if (tc_first_use_on_device(c, attr_done))
     CUDA_TRY(cudaFuncSetAttribute(sampler_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SAMPLER_SMEM));
-    attr_done = true;
-  }
   ProfScope ps(c, KC_SAMPLER);
   LAUNCH(c, sampler_kernel, n_rows, 1024, SAMPLER_SMEM, a);
   return RPO_OK;
@@ -771,22 +921,28 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
     // Prefix split: the chunk (a multiple of the key tile) that minimises rounds x (keys per CTA +
     // a fixed per-CTA cost of ~160 keys' worth of set-up and tail), with two CTAs resident per SM;
     // CTAs whose chunk lies beyond a short prefix carry suffix tiles only and are not counted.
-    const int slots = 2 * c->sm_count, per_group = pairs / std::max(n_groups, 1);
+    // The tcgen05 kernel takes over when a group's rows of one KV head fit its 64-row tile: one CTA per
+    // SM, 128-key tiles, a fixed cost of about 3 tiles (set-up, the pipeline's fill and drain).
+    c->attn_dec5 = c->bf16 && c->use_tc_attention && c->use_tc5_decode && c->shape.head_dim == T5_DH && G * rep <= D5_ROWS;
+    const int tile = c->attn_dec5 ? T5_BN : FA_BN;
+    const double fixed = c->attn_dec5 ? 384.0 : 160.0;
+    const int max_splits = c->attn_dec5 ? 24 : 32;
+    c->attn_suf_splits = 1;
+    const int slots = (c->attn_dec5 ? 1 : 2) * c->sm_count, per_group = pairs / std::max(n_groups, 1);
     double best_cost = 1e30, best_cl_cost = 1e30;
-    int best_chunk = std::max(FA_BN, ceil_div(max_p, FA_BN) * FA_BN), best_cl_chunk = best_chunk;
-    for (int want = 1; want <= 32; ++want) {
-      const int chunk = std::max(FA_BN, ceil_div(ceil_div(max_p, want), FA_BN) * FA_BN);
+    int best_chunk = std::max(tile, ceil_div(max_p, tile) * tile), best_cl_chunk = best_chunk;
+    for (int want = 1; want <= max_splits; ++want) {
+      const int chunk = std::max(tile, ceil_div(ceil_div(max_p, want), tile) * tile);
       int64_t ctas = 0;
       for (int g = 0; g < n_groups; ++g) ctas += (int64_t)per_group * ceil_div(std::max(groups[g].prefix_len, 1), chunk);
-      const double cost = (double)ceil_div((int)ctas, slots) * (chunk + 160.0);
+      const double cost = (double)ceil_div((int)ctas, slots) * (chunk + fixed);
       if (cost < best_cost - 1e-9) { best_cost = cost; best_chunk = chunk; }
       if (cluster_mergeable(ceil_div(max_p, chunk)) && cost < best_cl_cost - 1e-9) { best_cl_cost = cost; best_cl_chunk = chunk; }
     }
     // split counts that merge inside a cluster save the merge kernel: preferred unless clearly costlier
-    if (c->use_cluster_merge && best_cl_cost <= 1.1 * best_cost) best_chunk = best_cl_chunk;
+    if (c->use_cluster_merge && !c->attn_dec5 && best_cl_cost <= 1.1 * best_cost) best_chunk = best_cl_chunk;
     c->attn_split_chunk = best_chunk;
-    c->attn_splits = std::min(32, ceil_div(max_p, c->attn_split_chunk));
-    if (ceil_div(max_p, c->attn_split_chunk) > 32) c->attn_split_chunk = std::max(FA_BN, ceil_div(ceil_div(max_p, 32), FA_BN) * FA_BN);
+    if (ceil_div(max_p, c->attn_split_chunk) > max_splits) c->attn_split_chunk = std::max(tile, ceil_div(ceil_div(max_p, max_splits), tile) * tile);
     c->attn_splits = ceil_div(max_p, c->attn_split_chunk);
     c->attn_mode = 1; c->attn_G = G; c->attn_groups = n_groups;
     // the groups' prefix block ids, dense and padded to splits x chunk: the attention CTA of
@@ -817,9 +973,21 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
   a.logit_row = nullptr;
   // steps 1..S-1 are one and the same launch sequence (the step number lives on the device):
   // the first runs eagerly, the others replay a CUDA graph of it.
+  const bool fused = fused_layers(c, B);
   auto enqueue_step = [&]() -> int {
+    const float* e_gain; bf16* e_xg; float* e_ssq;
+    embed_norm_args(c, B, e_gain, e_xg, e_ssq);
     LAUNCH(c, embed_kernel<T>, B, 128, 0, (const int32_t*)w.cur_tok, (const T*)c->embed, w.x, B, d, c->shape.vocab,
-           c->d_status, w.step_ctr, row_meta_args(c));
+           c->d_status, w.step_ctr, row_meta_args(c), e_gain, e_xg, e_ssq);
+    if (fused && c->shape.n_layers > 0) {
+      // the last layer's down projection left bf16(x * final gain) and the rows' sums of squares: the
+      // output head scales its rows by 1/rms in its epilogue
+      RPO_TRY(run_layers_fused(c, B));
+      TcFuse f = fuse_norm_in(c);
+      RPO_TRY(gemm_fused(c, (const bf16*)w.h, (const bf16*)c->lm_head, w.logits, B, c->shape.vocab, d, TC_NSTORE_F32, c->shape.vocab, f));
+      RPO_TRY(launch_sampler(c, B, a));
+      return RPO_OK;
+    }
     // every row is a sequence's last row: the final RMSNorm reads ws.x directly and folds the last
     // layer's split-K partials in (no separate reduction, no copy of the residual rows)
     RPO_TRY(run_layers<T>(c, B, false));
@@ -830,7 +998,7 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
   };
   int j = 1;
   if (j < S) { RPO_TRY(enqueue_step()); ++j; }
-  if (j < S && c->use_graph && !c->profile && S - j >= 2) {
+  if (j < S && c->use_graph && !c->profile && !c->tap_buf && S - j >= 2) {
     uint32_t temp_bits; memcpy(&temp_bits, &a.temperature, 4);
     std::vector<uint64_t> key = {(uint64_t)B, (uint64_t)n_groups, (uint64_t)G, (uint64_t)S, (uint64_t)c->attn_splits,
                                  (uint64_t)c->attn_split_chunk, (uint64_t)(uintptr_t)d_forced, (uint64_t)(uintptr_t)d_tokens_out,
@@ -838,7 +1006,8 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
                                  (uint64_t)a.top_p24, (uint64_t)temp_bits,
                                  (uint64_t)a.greedy, (uint64_t)(uint32_t)a.eos_id, a.seed,
                                  (uint64_t)c->use_tcgen05, (uint64_t)c->use_tc_attention, (uint64_t)c->use_pdl,
-                                 (uint64_t)c->gemm_bn, (uint64_t)c->gemm_splits, (uint64_t)c->use_gemm_pairs, (uint64_t)c->use_cluster_merge, (uint64_t)c->use_gemm_pairs_small};
+                                 (uint64_t)c->gemm_bn, (uint64_t)c->gemm_splits, (uint64_t)c->use_gemm_pairs, (uint64_t)c->use_cluster_merge, (uint64_t)c->use_gemm_pairs_small, (uint64_t)c->use_fused_layers,
+                                 (uint64_t)c->attn_dec5, (uint64_t)c->attn_suf_splits};
     rpo_ctx::StepGraph* sg = nullptr;
     for (auto& g : c->step_graphs) if (g.key == key) sg = &g;
     if (!sg) {
@@ -929,7 +1098,10 @@ static int logprobs_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, 
         build_teacher_rows_kernel<<<grid_for(rows, 256), 256, 0, st>>>(d_tokens, d_lens, s0, ns, S, w.row_seq, w.row_t,
                                                                       w.row_tok);
         c->launches++;
-        embed_kernel<T><<<rows, 128, 0, st>>>((const int32_t*)w.row_tok, (const T*)c->embed, w.x, rows, d, V, c->d_status, nullptr, row_meta_args(c));
+        const float* e_gain; bf16* e_xg; float* e_ssq;
+        embed_norm_args(c, rows, e_gain, e_xg, e_ssq);
+        embed_kernel<T><<<rows, 128, 0, st>>>((const int32_t*)w.row_tok, (const T*)c->embed, w.x, rows, d, V, c->d_status, nullptr,
+                                              row_meta_args(c), e_gain, e_xg, e_ssq);
         c->launches++;
         if ((rc = run_layers<T>(c, rows)) != RPO_OK) break;
       }
@@ -1036,7 +1208,13 @@ extern "C" int rpo_rollout_host(rpo_ctx* c, int32_t n_groups, const int32_t* h_t
     cudaMemcpyAsync(h_lens_out, d_lens, B * 4, cudaMemcpyDeviceToHost, c->stream);
     if (h_logprobs_out) cudaMemcpyAsync(h_logprobs_out, d_lp, BS * 4, cudaMemcpyDeviceToHost, c->stream);
     if (want_policy) cudaMemcpyAsync(h_policy_out, d_pol, BS * 4, cudaMemcpyDeviceToHost, c->stream);
-    if (cudaStreamSynchronize(c->stream) != cudaSuccess) rc = RPO_ERR_CUDA;
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) { rc = RPO_ERR_CUDA; break; }
+    // the call has synchronised anyway: an expired device-side wait or a bad block index means the
+    // results are not to be trusted
+    int word = 0;
+    if ((rc = read_status(c, &word)) != RPO_OK) break;
+    if (word & STATUS_TIMEOUT) rc = RPO_ERR_DEVICE_TIMEOUT;
+    else if (word & STATUS_BAD_BLOCK) rc = RPO_ERR_CUDA;
   } while (0);
   if (rc != RPO_OK) { cudaStreamSynchronize(c->stream); cudaGetLastError(); }
   if (prefilled) rpo_release_groups(c, n_groups, groups.data());
@@ -1120,13 +1298,32 @@ extern "C" int rpo_gemm_bench(rpo_ctx* c, int32_t M, int32_t N, int32_t K, const
   return RPO_OK;
 }
 
-extern "C" int rpo_device_status(rpo_ctx* c, int32_t* out) {
-  if (!c || !out) return RPO_ERR_INVALID_ARG;
+// Reads and clears the device status word (synchronises the stream).  After an expired wait the
+// arrival counters of the split-K launches may be left half-counted: they are cleared too.
+static int read_status(rpo_ctx* c, int* word) {
   int v = 0;
   CUDA_TRY(cudaMemcpyAsync(&v, c->d_status, 4, cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(cudaStreamSynchronize(c->stream));
-  CUDA_TRY(cudaMemsetAsync(c->d_status, 0, 4, c->stream));
+  if (v) {
+    CUDA_TRY(cudaMemsetAsync(c->d_status, 0, 4, c->stream));
+    if (v & STATUS_TIMEOUT) CUDA_TRY(cudaMemsetAsync(c->ws.tile_ctr, 0, (size_t)TC_CTR_CAPACITY * 4, c->stream));
+  }
+  *word = v;
+  return RPO_OK;
+}
+
+extern "C" int rpo_device_status(rpo_ctx* c, int32_t* out) {
+  if (!c || !out) return RPO_ERR_INVALID_ARG;
+  int v = 0;
+  RPO_TRY(read_status(c, &v));
   *out = v;
+  return (v & STATUS_TIMEOUT) ? RPO_ERR_DEVICE_TIMEOUT : RPO_OK;
+}
+
+extern "C" int rpo_debug_tap(rpo_ctx* c, float* d_buf, int64_t capacity_floats, int64_t* h_used_out) {
+  if (!c || capacity_floats < 0 || (d_buf && capacity_floats == 0)) return RPO_ERR_INVALID_ARG;
+  if (h_used_out) *h_used_out = c->tap_used;
+  c->tap_buf = d_buf; c->tap_capacity = d_buf ? capacity_floats : 0; c->tap_used = 0;
   return RPO_OK;
 }
 
@@ -1143,8 +1340,15 @@ extern "C" int rpo_set_option(rpo_ctx* c, const char* name, int32_t value) {
   else if (!strcmp(name, "use_tc_attention")) c->use_tc_attention = value;
   else if (!strcmp(name, "use_graph")) c->use_graph = value;
   else if (!strcmp(name, "use_pdl")) c->use_pdl = value;
+  else if (!strcmp(name, "use_fused_layers")) c->use_fused_layers = value;
+  else if (!strcmp(name, "wait_limit_cycles")) {        // <= 0: the default; applies to the whole device (see gemm_tc.cuh)
+    const long long lim = value > 0 ? (long long)value : TC_TIMEOUT_CYCLES_DEFAULT;
+    CUDA_TRY(cudaMemcpyToSymbolAsync(g_wait_limit_cycles, &lim, sizeof(lim), 0, cudaMemcpyHostToDevice, c->stream));
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+  }
+  else if (!strcmp(name, "fused_split_limit")) c->fused_split_limit = value;
   else if (!strcmp(name, "use_tc5_attention")) c->use_tc5_attention = value;
-  else if (!strcmp(name, "tc5_v_variant")) c->tc5_v_variant = value;
+  else if (!strcmp(name, "use_tc5_decode")) c->use_tc5_decode = value;
   else if (!strcmp(name, "use_gemm_pairs")) c->use_gemm_pairs = value;
   else if (!strcmp(name, "use_cluster_merge")) c->use_cluster_merge = value;
   else if (!strcmp(name, "use_gemm_pairs_small")) c->use_gemm_pairs_small = value;

@@ -197,3 +197,27 @@ def test_float32_mode_is_close_to_float64():
     a = decoder.forward_full(w, sh, toks, dt=np.float64)
     b = decoder.forward_full(w, sh, toks, dt=np.float32)
     assert b.dtype == np.float32 and np.max(np.abs(a - b)) < 1e-4
+
+
+def test_single_layer_routine_chains_to_the_dense_forward():
+    """`decoder.layer` (used to check an implementation layer by layer) applied in turn is the dense
+    recompute bit for bit, and with a key context it is the shared-prefix routine."""
+    sh = small()
+    w = weights(sh)
+    toks = RNG.integers(0, sh.vocab, 17)
+    x = decoder.mat(w, "embed", np.float64)[toks]
+    causal = np.tril(np.ones((17, 17), dtype=bool))
+    ks, vs = [], []
+    for l in range(sh.n_layers):
+        x, a, k, v = decoder.layer(w, sh, l, x, np.arange(17), None, None, causal)
+        assert a.shape == (17, sh.n_q_heads, sh.head_dim)
+        ks.append(k); vs.append(v)
+    assert np.array_equal(x, decoder.forward_full(w, sh, toks, return_hidden=True))
+    # rows 12.. against a context of the first 12 keys
+    x = decoder.mat(w, "embed", np.float64)[toks]
+    xs = x[12:]
+    vis = np.concatenate([np.ones((5, 12), dtype=bool), np.tril(np.ones((5, 5), dtype=bool))], axis=1)
+    hid = decoder.forward_full(w, sh, toks, return_hidden=True)
+    for l in range(sh.n_layers):
+        xs, _, _, _ = decoder.layer(w, sh, l, xs, np.arange(12, 17), ks[l][:12], vs[l][:12], vis)
+    assert np.max(np.abs(xs - hid[12:])) < 1e-12

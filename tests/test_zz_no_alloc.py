@@ -12,6 +12,7 @@ import torch
 
 import paper_2601_19404_b200 as rpo
 import workloads
+from oracle import philox, sampler as osampler
 from gpu_util import DEV, make_ctx
 
 pytestmark = pytest.mark.gpu
@@ -44,6 +45,9 @@ def test_noalloc_sampler_equals_the_allocating_entry_point_on_consecutive_calls(
             smp = rpo.Sampler(T, top_p, False, -1, seed=7 + ci)
             want_t, want_lp, got_t, got_lp = _both(ctx, logits, smp, seqs, step, stream)
             assert np.array_equal(got_t, want_t), ci                      # token ids: bit-exact
+            for r in range(n):                                            # ... and the oracle's decision on these logits
+                u24 = int(philox.sampler_u24(7 + ci, int(seqs[r]), step))
+                assert got_t[r] == osampler.sample_token(logits[r], T, top_p, u24), (ci, r)
             assert np.max(np.abs(got_lp - want_lp)) <= 1e-4, ci           # the tolerance of the sampler parity test
         logits = workloads.logits_rows(4, 4096, 1.0, seed=50)
         want_t, _, got_t, _ = _both(ctx, logits, rpo.Sampler(1.0, 1.0, True, -1, 0), np.arange(4, dtype=np.int64), 0, None)
