@@ -298,7 +298,7 @@ def run_config(args, name, steps, warmup, rank, local_rank, world, dist, headlin
         step()
     barrier()
     launches0 = ctx.counters()[0]
-    clocks = ClockSampler(local_rank) if headline else None
+    clocks = ClockSampler(local_rank)
     timers = []
     t_begin = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
     t_begin.record(stream)
@@ -306,7 +306,7 @@ def run_config(args, name, steps, warmup, rank, local_rank, world, dist, headlin
         step(timers)
     t_end.record(stream)
     barrier()
-    clk = clocks.stop() if clocks else None
+    clk = clocks.stop()
     launches = ctx.counters()[0] - launches0
     phase = [float(np.mean([e[i].elapsed_time(e[i + 1]) for e in timers])) for i in range(3)]
     (total_ms, pre_ms, dec_ms, lp_ms), (emitted,) = reduce_over_ranks(
@@ -323,7 +323,7 @@ def run_config(args, name, steps, warmup, rank, local_rank, world, dist, headlin
     out = {
         "workload": name + ("" if not reduced else " REDUCED(" + ",".join(reduced) + ")"), "shape": cfg["shape"],
         "n_groups": n_g, "G": G, "prefix_tokens": int(lens.sum()), "suffix": S, "steps": steps, "warmup": warmup,
-        "value": value, "unit": UNIT, "ms_per_step": ms_per_step,
+        "value": value, "unit": UNIT, "ms_per_step": ms_per_step, "clocks": clk,
         "phases_ms": {"prefill": pre_ms, "decode": dec_ms, "logprobs": lp_ms, "decode_per_forward": dec_step_ms},
         "decode_hbm": {"algorithmic_bytes_per_step": ab, "achieved_gbs": decode_gbs, "frac_of_measured": decode_gbs / peaks["hbm_gbs"],
                        "frac_of_8tbs": decode_gbs / 8000.0},

@@ -116,8 +116,8 @@ int rpo_read_tensor(rpo_ctx* ctx, const char* name, void* h_dst, size_t bytes);
 int rpo_write_tensor(rpo_ctx* ctx, const char* name, const void* h_src, size_t bytes);
 
 /* Prefill: run the decoder over the cached prefix q_k || a_k^{[0:-m]} of each group ONCE
- * and keep its K/V in KV blocks that all G samples of the group will read (Eq. 3; "the
- * same response prefix is shared during the sampling phase", Section 3.4).
+ * and keep its K/V in KV blocks that all G samples of the group will read (Eq. 3; Section 3.4
+ * notes that the G samples of a group start from one and the same prefix).
  *   d_tokens   device int32, the n_groups prefixes concatenated
  *   h_offsets  host int32 [n_groups+1], prefix g = d_tokens[h_offsets[g] .. h_offsets[g+1])
  *   h_group_ids host int32 [n_groups] or NULL (ids 0..n_groups-1)

@@ -103,6 +103,15 @@ static RowMetaArgs row_meta_args(rpo_ctx* c) {
   return m;
 }
 
+// A context lives on the device that was current at rpo_create: calls made with another device current
+// switch to it (and leave it current, like the CUDA runtime's own stream calls would require).
+static int enter(rpo_ctx* c) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return RPO_ERR_CUDA; }
+  if (dev != c->device && cudaSetDevice(c->device) != cudaSuccess) { cudaGetLastError(); return RPO_ERR_CUDA; }
+  return RPO_OK;
+}
+
 static inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
 static inline int grid_for(int64_t n, int block, int cap = 148 * 16) {
   return (int)std::max<int64_t>(1, std::min<int64_t>((n + block - 1) / block, cap));
@@ -346,6 +355,7 @@ static int init_weights_t(rpo_ctx* c, uint64_t seed, float stdv) {
 
 extern "C" int rpo_init_weights(rpo_ctx* c, uint64_t seed, float stdv) {
   if (!c || !(stdv >= 0.f)) return RPO_ERR_INVALID_ARG;
+  RPO_TRY(enter(c));
   RPO_TRY(c->bf16 ? init_weights_t<bf16>(c, seed, stdv) : init_weights_t<float>(c, seed, stdv));
   c->weights_ready = true;
   return RPO_OK;
@@ -754,7 +764,13 @@ static void give_blocks(rpo_ctx* c, std::vector<int32_t>& b) {
 }
 
 static int check_groups(rpo_ctx* c, int n_groups, const rpo_group* g) {
+  if (n_groups > c->lim.max_groups) return RPO_ERR_LIMIT;      // (a handle given twice would also exceed the per-call tables)
+  std::vector<char> seen(c->lim.max_groups, 0);
   for (int i = 0; i < n_groups; ++i) {
+    if (g[i].slot >= 0 && g[i].slot < c->lim.max_groups) {
+      if (seen[g[i].slot]) return RPO_ERR_INVALID_ARG;
+      seen[g[i].slot] = 1;
+    }
     if (g[i].slot < 0 || g[i].slot >= c->lim.max_groups) return RPO_ERR_NOT_INITIALISED;
     const GroupState& gs = c->groups[g[i].slot];
     if (!gs.live || gs.group_id != g[i].group_id || gs.prefix_len != g[i].prefix_len) return RPO_ERR_NOT_INITIALISED;
@@ -803,6 +819,7 @@ extern "C" int rpo_prefill_prefix(rpo_ctx* c, int32_t n_groups, const int32_t* d
                                   const int32_t* h_group_ids, rpo_group* h_groups_out) {
   if (!c || n_groups < 0 || (n_groups > 0 && (!d_tokens || !h_offsets || !h_groups_out))) return RPO_ERR_INVALID_ARG;
   if (!c->weights_ready) return RPO_ERR_NOT_INITIALISED;
+  RPO_TRY(enter(c));
   c->prof_phase = 0;
   int64_t need_blocks = 0;
   for (int g = 0; g < n_groups; ++g) {
@@ -1044,6 +1061,7 @@ extern "C" int rpo_decode_suffix(rpo_ctx* c, int32_t n_groups, const rpo_group* 
   if (!c || n_groups <= 0 || !h_groups || G <= 0 || max_new <= 0 || !d_tokens_out || !d_lens_out) return RPO_ERR_INVALID_ARG;
   RPO_TRY(check_sampler(sp));
   if (!c->weights_ready) return RPO_ERR_NOT_INITIALISED;
+  RPO_TRY(enter(c));
   RPO_TRY(check_groups(c, n_groups, h_groups));
   if ((int64_t)n_groups * G > c->lim.max_seqs) return RPO_ERR_LIMIT;
   for (int g = 0; g < n_groups; ++g)
@@ -1129,6 +1147,7 @@ extern "C" int rpo_token_logprobs(rpo_ctx* c, int32_t n_groups, const rpo_group*
       !(inv_temperature > 0.f))
     return RPO_ERR_INVALID_ARG;
   if (!c->weights_ready) return RPO_ERR_NOT_INITIALISED;
+  RPO_TRY(enter(c));
   RPO_TRY(check_groups(c, n_groups, h_groups));
   for (int g = 0; g < n_groups; ++g)
     if (h_groups[g].prefix_len + max_new > c->lim.max_positions) return RPO_ERR_LIMIT;
