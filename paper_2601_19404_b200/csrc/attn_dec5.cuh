@@ -138,18 +138,24 @@ __global__ void __launch_bounds__(320, 1) flash_decode_tc5_kernel(Decode5Args a)
     bool ok = true;
     const int32_t* ptbl = a.pfx_tbl + (int64_t)grp * a.pfx_stride;
     int cur = 0;
-    for (int it = 0; it < n_tiles && ok; ++it) {
-      const int sk = it % D5_NSK, sv = it % D5_NSV;
-      const uint32_t par_k = ((it / D5_NSK) & 1) ^ 1, par_v = ((it / D5_NSV) & 1) ^ 1;
+    // Lane b < 4 looks up the KV block of keys key0 + 16 b .. of tile `it` (past the end of the segment: the last
+    // valid block, finite data that the softmax masks).  The look-up of tile it + 1 is requested before tile it is
+    // waited for and sent, so the round trip to the table never sits between two tiles.
+    auto lookup = [&](int it) -> int {
       int seq, key0, limit;
       tile_info(it, cur, seq, key0, limit);                     // key0 is a multiple of 64: whole KV blocks
       const int nb = max(1, min(D5_BN / KV_BLOCK, (limit - key0 + KV_BLOCK - 1) / KV_BLOCK));
-      int blk = 0;
-      if (lane < D5_BN / KV_BLOCK) {          // lane b: block of keys key0 + 16 b .. (past the end: the last valid one)
-        const int e = key0 / KV_BLOCK + min(lane, nb - 1);
-        blk = (seq < 0) ? ptbl[e] : a.block_table[s_tbl[seq] + e];
-        if (blk < 0 || blk >= a.pool.n_blocks) { atomicOr(a.status, STATUS_BAD_BLOCK); blk = 0; }
-      }
+      if (lane >= D5_BN / KV_BLOCK) return 0;
+      const int e = key0 / KV_BLOCK + min(lane, nb - 1);
+      return (seq < 0) ? ptbl[e] : a.block_table[s_tbl[seq] + e];
+    };
+    int blk_next = (n_tiles > 0) ? lookup(0) : 0;
+    for (int it = 0; it < n_tiles && ok; ++it) {
+      const int sk = it % D5_NSK, sv = it % D5_NSV;
+      const uint32_t par_k = ((it / D5_NSK) & 1) ^ 1, par_v = ((it / D5_NSV) & 1) ^ 1;
+      int blk = blk_next;
+      if (it + 1 < n_tiles) blk_next = lookup(it + 1);
+      if (blk < 0 || blk >= a.pool.n_blocks) { atomicOr(a.status, STATUS_BAD_BLOCK); blk = 0; }
       if (lane == 0) { ok = tc::mbar_wait(&empty_k[sk], par_k, abort_flag); if (ok) tc::mbar_expect_tx(&full_k[sk], D5_KV_TILE); }
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
@@ -170,36 +176,43 @@ __global__ void __launch_bounds__(320, 1) flash_decode_tc5_kernel(Decode5Args a)
     if (lane == 0) {
       constexpr uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(D5_BN >> 3) << 17) | ((uint32_t)(T5_BM >> 4) << 24);
       constexpr uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(T5_DH >> 3) << 17) | ((uint32_t)(T5_BM >> 4) << 24);   // B operand (V) is MN-major, N = 128 dims
+      // One thread issues every MMA of the CTA, so its instruction stream is on the critical path of every tile:
+      // the operand descriptors are built once; inside the loop a descriptor is a base plus a constant (the
+      // address field counts 16-byte units and never carries out of its 14 bits within 227 KB of shared memory).
+      const uint64_t dq = t5::desc_k_sw128(sQ), dk = t5::desc_k_sw128(sK), dp = t5::desc_k_sw128(sP);
+      const uint64_t dv = t5::desc_mn_sw128(sV, 2048, 1024);
       bool ok = tc::mbar_wait(q_full, 0, abort_flag);
+      int sk_n = 0, sv_n = 0;                                                // ring stages of the next Q K^T / P V
+      uint32_t phk = 0, phv = 0;                                             // and their phases
       auto issue_qk = [&](int it) -> bool {
-        const int sk = it % D5_NSK, sb = it & 1;
-        if (!tc::mbar_wait(&full_k[sk], (it / D5_NSK) & 1, abort_flag)) return false;
+        const int sb = it & 1;
+        if (!tc::mbar_wait(&full_k[sk_n], phk, abort_flag)) return false;
         if (!tc::mbar_wait(&s_free[sb], ((it >> 1) & 1) ^ 1, abort_flag)) return false;
         tc::tmem_fence_after();
+        const uint64_t dks = dk + (uint64_t)(sk_n * (D5_KV_TILE >> 4));
 #pragma unroll
-        for (int k = 0; k < T5_DH / 16; ++k) {                               // dim half plane (k / 4), 32 bytes per 16 dims
-          tc::umma_bf16(tmem + sb * D5_BN, t5::desc_k_sw128(sQ + (k >> 2) * (D5_Q_TILE / 2) + (k & 3) * 32),
-                        t5::desc_k_sw128(sK + sk * D5_KV_TILE + (k >> 2) * (D5_KV_TILE / 2) + (k & 3) * 32), idesc_qk, k > 0);
-        }
-        tc::umma_commit(&empty_k[sk]);
+        for (int k = 0; k < T5_DH / 16; ++k)                                 // dim half plane (k / 4), 32 bytes per 16 dims
+          tc::umma_bf16(tmem + sb * D5_BN, dq + (uint64_t)((k >> 2) * (D5_Q_TILE >> 5) + (k & 3) * 2),
+                        dks + (uint64_t)((k >> 2) * (D5_KV_TILE >> 5) + (k & 3) * 2), idesc_qk, k > 0);
+        tc::umma_commit(&empty_k[sk_n]);
         tc::umma_commit(&s_full[sb]);
+        if (++sk_n == D5_NSK) { sk_n = 0; phk ^= 1; }
         return true;
       };
       if (ok && n_tiles > 0) ok = issue_qk(0);
       for (int it = 0; it < n_tiles && ok; ++it) {
         if (it + 1 < n_tiles) { ok = issue_qk(it + 1); if (!ok) break; }      // S(it+1) overlaps the softmax of tile it
-        const int sv = it % D5_NSV, pb = it & 1;
+        const int pb = it & 1;
         if (!tc::mbar_wait(&p_full[pb], (it >> 1) & 1, abort_flag)) { ok = false; break; }
-        if (!tc::mbar_wait(&full_v[sv], (it / D5_NSV) & 1, abort_flag)) { ok = false; break; }
+        if (!tc::mbar_wait(&full_v[sv_n], phv, abort_flag)) { ok = false; break; }
         tc::tmem_fence_after();
+        const uint64_t dps = dp + (uint64_t)(pb * (D5_KV_TILE >> 4)), dvs = dv + (uint64_t)(sv_n * (D5_KV_TILE >> 4));
 #pragma unroll
-        for (int b = 0; b < D5_BN / KV_BLOCK; ++b) {                         // 16 keys per MMA = one KV block
-          const uint64_t da = t5::desc_k_sw128(sP + pb * D5_KV_TILE + b * 32);   // P: one 128-byte row of 64 keys per query row
-          const uint64_t db = t5::desc_mn_sw128(sV + sv * D5_KV_TILE + b * 4096, 2048, 1024);
-          tc::umma_bf16(tmem + 2 * D5_BN, da, db, idesc_pv, (it > 0 || b > 0) ? 1u : 0u);   // O accumulates over all tiles
-        }
-        tc::umma_commit(&empty_v[sv]);
+        for (int b = 0; b < D5_BN / KV_BLOCK; ++b)                           // 16 keys per MMA = one KV block: P advances 32 bytes, V 4096
+          tc::umma_bf16(tmem + 2 * D5_BN, dps + (uint64_t)(b * 2), dvs + (uint64_t)(b * 256), idesc_pv, (it > 0 || b > 0) ? 1u : 0u);
+        tc::umma_commit(&empty_v[sv_n]);
         tc::umma_commit(&p_free[pb]);                                        // every MMA up to P V of tile it is done
+        if (++sv_n == D5_NSV) { sv_n = 0; phv ^= 1; }
       }
     }
   } else {

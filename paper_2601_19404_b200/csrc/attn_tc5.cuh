@@ -115,18 +115,22 @@ flash_attn_tc5_kernel(const __grid_constant__ CUtensorMap q_map, Flash5Args a) {
       tc::tma_load_2d((void*)(sm + T5_TILE / 2), &q_map, a.q_col0 + head * T5_DH + 64, row0, q_full);
     }
     bool ok = true;
-    for (int it = 0; it < n_tiles && ok; ++it) {
-      const int st = it & 1;
-      const uint32_t par = ((it >> 1) & 1) ^ 1;
+    // lane b < 8: block of keys key0 + 16 b .. of tile `it` (past the end: the last valid one).  The look-up of
+    // tile it + 1 is requested before tile it is waited for and sent.
+    auto lookup = [&](int it) -> int {
       const bool shared_tile = it < n_sh;
       const int tbl = shared_tile ? sd.shared_tbl : sd.priv_tbl;
       const int key0 = shared_tile ? it * T5_BN : (it - n_sh) * T5_BN, limit = shared_tile ? sh_end : pr_end;
       const int nb = max(1, min(T5_BN / KV_BLOCK, (limit - key0 + KV_BLOCK - 1) / KV_BLOCK));
-      int blk = 0;
-      if (lane < T5_BN / KV_BLOCK) {          // lane b: block of keys key0 + 16 b .. (past the end: the last valid one)
-        blk = a.block_table[tbl + (key0 + min(lane, nb - 1) * KV_BLOCK) / KV_BLOCK];
-        if (blk < 0 || blk >= a.pool.n_blocks) { atomicOr(a.status, STATUS_BAD_BLOCK); blk = 0; }
-      }
+      return (lane < T5_BN / KV_BLOCK) ? a.block_table[tbl + (key0 + min(lane, nb - 1) * KV_BLOCK) / KV_BLOCK] : 0;
+    };
+    int blk_next = (n_tiles > 0) ? lookup(0) : 0;
+    for (int it = 0; it < n_tiles && ok; ++it) {
+      const int st = it & 1;
+      const uint32_t par = ((it >> 1) & 1) ^ 1;
+      int blk = blk_next;
+      if (it + 1 < n_tiles) blk_next = lookup(it + 1);
+      if (blk < 0 || blk >= a.pool.n_blocks) { atomicOr(a.status, STATUS_BAD_BLOCK); blk = 0; }
       if (lane == 0) { ok = tc::mbar_wait(&empty_k[st], par, abort_flag); if (ok) tc::mbar_expect_tx(&full_k[st], T5_TILE); }
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
@@ -147,16 +151,20 @@ flash_attn_tc5_kernel(const __grid_constant__ CUtensorMap q_map, Flash5Args a) {
     if (lane == 0) {
       constexpr uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(T5_BN >> 3) << 17) | ((uint32_t)(T5_BM >> 4) << 24);
       constexpr uint32_t idesc_pv = idesc_qk | (1u << 16);                 // B operand (V) is MN-major
+      // operand descriptors built once: inside the loop a descriptor is a base plus a constant number of 16-byte units
+      const uint64_t dq = t5::desc_k_sw128(sQ), dk = t5::desc_k_sw128(sK), dp = t5::desc_k_sw128(sP);
+      const uint64_t dv = t5::desc_mn_sw128(sV, 2048, 1024);
       bool ok = tc::mbar_wait(q_full, 0, abort_flag);
       auto issue_qk = [&](int it) -> bool {
         const int st = it & 1, sb = it & 1;
         if (!tc::mbar_wait(&full_k[st], (it >> 1) & 1, abort_flag)) return false;
         if (!tc::mbar_wait(&s_free[sb], ((it >> 1) & 1) ^ 1, abort_flag)) return false;
         tc::tmem_fence_after();
+        const uint64_t dks = dk + (uint64_t)(st * (T5_TILE >> 4));
 #pragma unroll
-        for (int k = 0; k < T5_DH / 16; ++k) {
-          const uint32_t off = (k >> 2) * (T5_TILE / 2) + (k & 3) * 32;    // dim half plane, 32 bytes per 16 dims
-          tc::umma_bf16(tmem + sb * T5_BN, t5::desc_k_sw128(sQ + off), t5::desc_k_sw128(sK + st * T5_TILE + off), idesc_qk, k > 0);
+        for (int k = 0; k < T5_DH / 16; ++k) {                             // dim half plane (k / 4), 32 bytes per 16 dims
+          const uint64_t off = (uint64_t)((k >> 2) * (T5_TILE >> 5) + (k & 3) * 2);
+          tc::umma_bf16(tmem + sb * T5_BN, dq + off, dks + off, idesc_qk, k > 0);
         }
         tc::umma_commit(&empty_k[st]);
         tc::umma_commit(&s_full[sb]);
@@ -170,12 +178,10 @@ flash_attn_tc5_kernel(const __grid_constant__ CUtensorMap q_map, Flash5Args a) {
         if (!tc::mbar_wait(&full_v[st], (it >> 1) & 1, abort_flag)) { ok = false; break; }
         if (!tc::mbar_wait(o_free, (it & 1) ^ 1, abort_flag)) { ok = false; break; }
         tc::tmem_fence_after();
+        const uint64_t dvs = dv + (uint64_t)(st * (T5_TILE >> 4));
 #pragma unroll
-        for (int b = 0; b < T5_BN / KV_BLOCK; ++b) {                         // 16 keys per MMA = one KV block
-          const uint64_t da = t5::desc_k_sw128(sP + (b >> 2) * (T5_TILE / 2) + (b & 3) * 32);
-          const uint64_t db = t5::desc_mn_sw128(sV + st * T5_TILE + b * 4096, 2048, 1024);
-          tc::umma_bf16(tmem + 2 * T5_BN, da, db, idesc_pv, b > 0);
-        }
+        for (int b = 0; b < T5_BN / KV_BLOCK; ++b)                           // 16 keys per MMA = one KV block
+          tc::umma_bf16(tmem + 2 * T5_BN, dp + (uint64_t)((b >> 2) * (T5_TILE >> 5) + (b & 3) * 2), dvs + (uint64_t)(b * 256), idesc_pv, b > 0);
         tc::umma_commit(&empty_v[st]);
         tc::umma_commit(o_full);
       }
