@@ -149,6 +149,31 @@ int rpo_decode_suffix(rpo_ctx* ctx, int32_t n_groups, const rpo_group* h_groups,
                       const rpo_sampler* sampler, const int32_t* d_forced_tokens, int32_t* d_tokens_out,
                       int32_t* d_lens_out, float* d_logprobs_out, float* d_logits_dbg);
 
+/* Decode in waves: the NEXT max_new suffix tokens of each group's G sequences.  Generating the
+ * cache's full-path responses (Section 3.1, Eq. 1: one response per question, sampled before
+ * training) proceeds in waves so that finished sequences can leave the batch and waiting
+ * questions take their place; this call keeps what a sequence needs to go on, so that a wave
+ * does not run the decoder over prompt + generated tokens again:
+ *   - the first call on a group reserves private KV blocks for max_total suffix tokens per
+ *     sequence and one state row per sequence; later calls on the group must pass the same G
+ *     and stay within max_total (RPO_ERR_LIMIT otherwise; max_total is read on the first call);
+ *   - every token of a wave, the last one included, is run through the decoder before the
+ *     call's work ends: its K/V joins the private blocks, and the logits its successor will
+ *     be drawn from are parked in the state row (vocab floats) with the finished flag;
+ *   - draw number j of a sequence is its absolute suffix position, so W calls of max_new
+ *     tokens produce the tokens and log-probs of ONE rpo_decode_suffix call of W*max_new
+ *     tokens on the same groups, bit for bit;
+ *   - blocks and state rows return to the pool with rpo_release_groups.
+ * Groups at different stages may share a call.  Outputs are relative to the wave:
+ * d_tokens_out [B*max_new], d_lens_out [B] = tokens of this wave up to and including EOS
+ * (0 for a sequence that had finished before), d_logprobs_out NULL or [B*max_new];
+ * d_forced_tokens NULL or [B*max_new] as in rpo_decode_suffix.
+ * Errors: RPO_ERR_KV_POOL (blocks or state rows exhausted; nothing is reserved),
+ * RPO_ERR_LIMIT, RPO_ERR_NOT_INITIALISED, RPO_ERR_INVALID_ARG. */
+int rpo_decode_wave(rpo_ctx* ctx, int32_t n_groups, const rpo_group* h_groups, int32_t G, int32_t max_new,
+                    int32_t max_total, const rpo_sampler* sampler, const int32_t* d_forced_tokens,
+                    int32_t* d_tokens_out, int32_t* d_lens_out, float* d_logprobs_out);
+
 /* Token log-probabilities log pi_theta(o_{i,j} | q, o_{i,<j}) of given suffixes (numerator
  * and denominator of r_{i,j}, Eq. 7), teacher-forced over the shared prefix KV:
  *   d_tokens [B*max_new], d_lens [B] as written by rpo_decode_suffix

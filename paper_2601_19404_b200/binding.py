@@ -13,7 +13,7 @@ _LIB = None
 
 EXPORTED_SYMBOLS = [
     "rpo_strerror", "rpo_shape_preset", "rpo_create", "rpo_destroy", "rpo_init_weights", "rpo_read_tensor",
-    "rpo_write_tensor", "rpo_prefill_prefix", "rpo_decode_suffix", "rpo_token_logprobs", "rpo_release_groups",
+    "rpo_write_tensor", "rpo_prefill_prefix", "rpo_decode_suffix", "rpo_decode_wave", "rpo_token_logprobs", "rpo_release_groups",
     "rpo_policy_objective", "rpo_rollout_host", "rpo_sample_rows", "rpo_sample_rows_noalloc", "rpo_gemm", "rpo_gemm_bench", "rpo_device_status", "rpo_debug_tap", "rpo_counters", "rpo_set_option", "rpo_profile_read",
 ]
 
@@ -75,6 +75,7 @@ def load_library(path=None):
     lib.rpo_write_tensor.argtypes = [vp, C.c_char_p, vp, C.c_size_t]
     lib.rpo_prefill_prefix.argtypes = [vp, i32, vp, vp, vp, C.POINTER(Group)]
     lib.rpo_decode_suffix.argtypes = [vp, i32, C.POINTER(Group), i32, i32, C.POINTER(Sampler), vp, vp, vp, vp, vp]
+    lib.rpo_decode_wave.argtypes = [vp, i32, C.POINTER(Group), i32, i32, i32, C.POINTER(Sampler), vp, vp, vp, vp]
     lib.rpo_token_logprobs.argtypes = [vp, i32, C.POINTER(Group), i32, i32, vp, vp, f32, vp, vp]
     lib.rpo_policy_objective.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, C.POINTER(ObjectiveCfg), vp, vp, vp, vp, vp]
     lib.rpo_release_groups.argtypes = [vp, i32, C.POINTER(Group)]
@@ -214,6 +215,12 @@ class Context:
         _check(self.lib.rpo_decode_suffix(self.handle, len(groups), groups, int(G), int(max_new), C.byref(sampler),
                                           _ptr(d_forced_tokens), _ptr(d_tokens_out), _ptr(d_lens_out),
                                           _ptr(d_logprobs_out), _ptr(d_logits_dbg)), "rpo_decode_suffix")
+
+    def decode_wave(self, groups, G, max_new, max_total, sampler, d_tokens_out, d_lens_out, d_logprobs_out=None,
+                    d_forced_tokens=None):
+        _check(self.lib.rpo_decode_wave(self.handle, len(groups), groups, int(G), int(max_new), int(max_total),
+                                        C.byref(sampler), _ptr(d_forced_tokens), _ptr(d_tokens_out), _ptr(d_lens_out),
+                                        _ptr(d_logprobs_out)), "rpo_decode_wave")
 
     def token_logprobs(self, groups, G, max_new, d_tokens, d_lens, d_logprobs_out, inv_temperature=1.0, d_logits_dbg=None):
         _check(self.lib.rpo_token_logprobs(self.handle, len(groups), groups, int(G), int(max_new), _ptr(d_tokens),

@@ -27,6 +27,11 @@ struct GroupState {
   bool live = false;
   int32_t group_id = 0, prefix_len = 0;
   std::vector<int32_t> blocks;
+  // a decode that proceeds in waves (rpo_decode_wave): the private suffix blocks and the state rows of the group's
+  // sequences stay with the group between calls
+  int wave_G = 0, wave_total = 0, wave_t = 0;      // sequences, reserved suffix positions, positions generated so far
+  std::vector<int32_t> wave_blocks;                // wave_G x ceil(wave_total / 16) private blocks
+  std::vector<int32_t> wave_rows;                  // wave_G rows of the sequence-state pool
 };
 
 struct Workspace {
@@ -38,7 +43,7 @@ struct Workspace {
   void* act = nullptr;     // [R, F]
   float* xh = nullptr;     // [HR, d] head input rows
   void* hh = nullptr;      // [HR, d]
-  float* logits = nullptr; // [HR, V]
+  float* logits = nullptr; // [HR + max_seqs, V]: HR work rows, then the rows parked by a decode in waves
   uint32_t* sampler_w = nullptr;  // [max(max_seqs, max_groups), V] quantised sampler weights
   size_t sampler_w_rows = 0;
   float* ssq = nullptr;          // [R][ssq_stride] partial sums of squares of the residual rows (fused RMSNorm)
@@ -56,6 +61,8 @@ struct Workspace {
   int4* row_meta = nullptr;            // per row of the pass: (position, private KV block, slot in block, -) or x < 0: inactive
   void* seqs = nullptr;    // SeqDesc[]
   int32_t *done = nullptr, *lens = nullptr, *cur_tok = nullptr, *logit_row = nullptr, *slot_idx = nullptr;
+  int32_t *t_base = nullptr, *state_idx = nullptr;      // resumed decode: positions generated before the call; state row per sequence
+  int32_t *done_idx = nullptr;                          // resumed decode: where the finished flags are read from (-1: fresh)
   int32_t* step_ctr = nullptr;   // device counter of the decode step being computed
   int64_t* seq_ids = nullptr;
   int R = 0, HR = 0;
@@ -87,6 +94,8 @@ struct rpo_ctx {
   std::vector<int32_t> free_slots;
   std::vector<rpo::GroupState> groups;
   float* d_x_last = nullptr;   // [max_groups, d]
+  int32_t* d_seq_done = nullptr;           // [max_seqs] finished flag per state row (decode in waves)
+  std::vector<int32_t> free_state_rows;
   void* d_rope = nullptr;      // float2 [max_positions, dh/2]
   rpo::Workspace ws;
   int* d_status = nullptr;

@@ -194,6 +194,17 @@ __global__ void norm_prep_kernel(const float* __restrict__ x, const float* __res
   if (threadIdx.x == 0) ssq[r] = ss;
 }
 
+// dst[idx[r],:] = src[r,:]  (32-bit words; rows whose idx is negative are skipped)
+__global__ void scatter_rows_u32_kernel(const uint32_t* __restrict__ src, const int32_t* __restrict__ idx,
+                                        uint32_t* __restrict__ dst, int rows, int d) {
+  pdl_prologue();
+  const int r = blockIdx.x;
+  if (r >= rows) return;
+  const int s = idx[r];
+  if (s < 0) return;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) dst[(int64_t)s * d + i] = src[(int64_t)r * d + i];
+}
+
 // dst[r,:] = src[idx[r],:]  (float32 rows; idx may be NULL = identity)
 __global__ void gather_rows_f32_kernel(const float* __restrict__ src, const int32_t* __restrict__ idx,
                                        float* __restrict__ dst, int rows, int d) {

@@ -272,6 +272,8 @@ extern "C" int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limit
   c->groups.resize(lim->max_groups);
   for (int i = lim->max_groups - 1; i >= 0; --i) c->free_slots.push_back(i);
   ALLOC(c->d_x_last, (size_t)lim->max_groups * d * 4);
+  ALLOC(c->d_seq_done, (size_t)std::max(lim->max_seqs, 1) * 4);
+  for (int i = lim->max_seqs - 1; i >= 0; --i) c->free_state_rows.push_back(i);
   ALLOC(c->d_rope, (size_t)lim->max_positions * (dh / 2) * sizeof(float2));
   ALLOC(c->d_status, 16);
   // ---- workspaces
@@ -286,7 +288,7 @@ extern "C" int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limit
   ALLOC(w.act, (size_t)w.R * F * e);
   ALLOC(w.xh, (size_t)w.HR * d * 4);
   ALLOC(w.hh, (size_t)w.HR * d * e);
-  ALLOC(w.logits, (size_t)w.HR * V * 4);
+  ALLOC(w.logits, (size_t)(w.HR + lim->max_seqs) * V * 4);   // HR work rows, then one parked row per state row (decode in waves)
   ALLOC(w.row_seq, (size_t)w.R * 4);
   ALLOC(w.row_meta, (size_t)w.R * sizeof(int4));
   ALLOC(w.pfx_tbl, (size_t)lim->max_groups * (c->tbl_stride + 512 + 8) * 4);
@@ -300,6 +302,9 @@ extern "C" int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limit
   ALLOC(w.lens, (size_t)nseq * 4);
   ALLOC(w.cur_tok, (size_t)nseq * 4);
   ALLOC(w.logit_row, (size_t)nseq * 4);
+  ALLOC(w.t_base, (size_t)nseq * 4);
+  ALLOC(w.state_idx, (size_t)nseq * 4);
+  ALLOC(w.done_idx, (size_t)nseq * 4);
   ALLOC(w.slot_idx, (size_t)nseq * 4);
   ALLOC(w.step_ctr, 16);
   ALLOC(w.seq_ids, (size_t)nseq * 8);
@@ -862,6 +867,10 @@ extern "C" int rpo_release_groups(rpo_ctx* c, int32_t n_groups, const rpo_group*
     if (g[i].slot < 0 || g[i].slot >= c->lim.max_groups || !c->groups[g[i].slot].live) { rc = RPO_ERR_NOT_INITIALISED; continue; }
     GroupState& gs = c->groups[g[i].slot];
     give_blocks(c, gs.blocks);
+    give_blocks(c, gs.wave_blocks);
+    for (auto it = gs.wave_rows.rbegin(); it != gs.wave_rows.rend(); ++it) c->free_state_rows.push_back(*it);
+    gs.wave_rows.clear();
+    gs.wave_G = gs.wave_total = gs.wave_t = 0;
     gs.live = false;
     c->free_slots.push_back(g[i].slot);
   }
@@ -899,24 +908,42 @@ static int check_sampler(const rpo_sampler* sp) {
 template <typename T>
 static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, int S, const rpo_sampler* sp,
                     const int32_t* d_forced, int32_t* d_tokens_out, int32_t* d_lens_out, float* d_logprobs_out,
-                    float* d_logits_dbg, std::vector<int32_t>& priv_blocks) {
+                    float* d_logits_dbg, std::vector<int32_t>& priv_blocks, bool wave = false) {
+  // wave: the call continues the groups' sequences where their last rpo_decode_wave call stopped; blocks and state
+  // rows were reserved by the caller and stay with the groups
   Workspace& w = c->ws;
   const int B = n_groups * G, d = c->shape.d_model;
   const int per_seq = ceil_div(std::max(S - 1, 0), KV_BLOCK);
-  RPO_TRY(take_blocks(c, B * per_seq, priv_blocks));
+  if (!wave) RPO_TRY(take_blocks(c, B * per_seq, priv_blocks));
   std::vector<SeqDesc> sd(B);
   std::vector<int32_t> tbl((size_t)B * c->tbl_stride, -1), logit_row(B), slot_idx(n_groups), zero(B, 0), seq_of_row(B);
+  std::vector<int32_t> t_base(B, 0), state_idx(B, -1), done_idx(B, -1);
   std::vector<int64_t> seq_ids(B);
+  int n_fresh = 0;                                       // wave: groups that start with this call, in call order
   for (int g = 0; g < n_groups; ++g) {
     slot_idx[g] = groups[g].slot;
+    const GroupState& gs = c->groups[groups[g].slot];
+    if (wave && gs.wave_t == 0) slot_idx[n_fresh] = groups[g].slot;
     for (int i = 0; i < G; ++i) {
       const int b = g * G + i;
       sd[b].shared_tbl = groups[g].slot * c->tbl_stride; sd[b].shared_len = groups[g].prefix_len;
       sd[b].priv_tbl = (c->lim.max_groups + b) * c->tbl_stride; sd[b].reserved = 0;
-      for (int k = 0; k < per_seq; ++k) tbl[(size_t)b * c->tbl_stride + k] = priv_blocks[(size_t)b * per_seq + k];
-      logit_row[b] = g; seq_of_row[b] = b;
+      if (wave) {
+        const int per = ceil_div(gs.wave_total, KV_BLOCK);
+        for (int k = 0; k < per; ++k) tbl[(size_t)b * c->tbl_stride + k] = gs.wave_blocks[(size_t)i * per + k];
+        t_base[b] = gs.wave_t;
+        state_idx[b] = gs.wave_rows[i];                                // where the sequence's state is parked
+        done_idx[b] = gs.wave_t > 0 ? gs.wave_rows[i] : -1;            // a fresh sequence starts unfinished
+        // the row its first logits of this call come from: the parked row, or the row of its (fresh) group
+        logit_row[b] = gs.wave_t > 0 ? w.HR + gs.wave_rows[i] : n_fresh;
+      } else {
+        for (int k = 0; k < per_seq; ++k) tbl[(size_t)b * c->tbl_stride + k] = priv_blocks[(size_t)b * per_seq + k];
+        logit_row[b] = g;
+      }
+      seq_of_row[b] = b;
       seq_ids[b] = (int64_t)groups[g].group_id * G + i;
     }
+    if (wave && gs.wave_t == 0) ++n_fresh;
   }
   cudaStream_t st = c->stream;
   CUDA_TRY(cudaMemcpyAsync(w.seqs, sd.data(), (size_t)B * sizeof(SeqDesc), cudaMemcpyHostToDevice, st));
@@ -929,6 +956,13 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
   CUDA_TRY(cudaMemsetAsync(w.done, 0, (size_t)B * 4, st));
   CUDA_TRY(cudaMemsetAsync(w.lens, 0, (size_t)B * 4, st));
   CUDA_TRY(cudaMemsetAsync(w.row_t, 0xFF, (size_t)B * 4, st));
+  if (wave) {
+    CUDA_TRY(cudaMemcpyAsync(w.t_base, t_base.data(), (size_t)B * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaMemcpyAsync(w.state_idx, state_idx.data(), (size_t)B * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaMemcpyAsync(w.done_idx, done_idx.data(), (size_t)B * 4, cudaMemcpyHostToDevice, st));
+    // finished flags of the continuing sequences (a negative index yields 0)
+    LAUNCH(c, gather_rows_f32_kernel, B, 32, 0, (const float*)c->d_seq_done, (const int32_t*)w.done_idx, (float*)w.done, B, 1);
+  }
 
   {
     int max_p = 1;
@@ -982,16 +1016,29 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
   // step 0: the G samples of a group draw from the logits of the group's last prefix token
   CUDA_TRY(cudaMemsetAsync(w.step_ctr, 0, 4, st));
   a.step_ptr = w.step_ctr; a.n_steps = S;
-  LAUNCH(c, gather_rows_f32_kernel, n_groups, 128, 0, (const float*)c->d_x_last, (const int32_t*)w.slot_idx, w.xh,
-         n_groups, d);
-  RPO_TRY(head<T>(c, n_groups));
-  a.logit_row = w.logit_row;
-  RPO_TRY(launch_sampler(c, B, a));
-  a.logit_row = nullptr;
+  if (wave) {
+    // a fresh group's sequences draw from the logits of its last prefix token, a continuing sequence from the
+    // logits parked by its last call; the call's last token is fed too (below), so no step of it is the last one
+    a.t_base = w.t_base; a.n_steps = S + 1;
+    if (n_fresh > 0) {
+      LAUNCH(c, gather_rows_f32_kernel, n_fresh, 128, 0, (const float*)c->d_x_last, (const int32_t*)w.slot_idx, w.xh, n_fresh, d);
+      RPO_TRY(head<T>(c, n_fresh));
+    }
+    a.logit_row = w.logit_row;
+    RPO_TRY(launch_sampler(c, B, a));
+    a.logit_row = nullptr;
+  } else {
+    LAUNCH(c, gather_rows_f32_kernel, n_groups, 128, 0, (const float*)c->d_x_last, (const int32_t*)w.slot_idx, w.xh,
+           n_groups, d);
+    RPO_TRY(head<T>(c, n_groups));
+    a.logit_row = w.logit_row;
+    RPO_TRY(launch_sampler(c, B, a));
+    a.logit_row = nullptr;
+  }
   // steps 1..S-1 are one and the same launch sequence (the step number lives on the device):
   // the first runs eagerly, the others replay a CUDA graph of it.
   const bool fused = fused_layers(c, B);
-  auto enqueue_step = [&]() -> int {
+  auto enqueue_step = [&](bool sample = true) -> int {
     const float* e_gain; bf16* e_xg; float* e_ssq;
     embed_norm_args(c, B, e_gain, e_xg, e_ssq);
     LAUNCH(c, embed_kernel<T>, B, 128, 0, (const int32_t*)w.cur_tok, (const T*)c->embed, w.x, B, d, c->shape.vocab,
@@ -1002,7 +1049,7 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
       RPO_TRY(run_layers_fused(c, B));
       TcFuse f = fuse_norm_in(c);
       RPO_TRY(gemm_fused(c, (const bf16*)w.h, (const bf16*)c->lm_head, w.logits, B, c->shape.vocab, d, TC_NSTORE_F32, c->shape.vocab, f));
-      RPO_TRY(launch_sampler(c, B, a));
+      if (sample) RPO_TRY(launch_sampler(c, B, a));
       return RPO_OK;
     }
     // every row is a sequence's last row: the final RMSNorm reads ws.x directly and folds the last
@@ -1010,7 +1057,7 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
     RPO_TRY(run_layers<T>(c, B, false));
     RPO_TRY(rmsnorm<T>(c, w.x, c->gf, (T*)w.hh, B));
     RPO_TRY(gemm<T>(c, (const T*)w.hh, (const T*)c->lm_head, w.logits, B, c->shape.vocab, d, EPI_STORE_F32));
-    RPO_TRY(launch_sampler(c, B, a));
+    if (sample) RPO_TRY(launch_sampler(c, B, a));
     return RPO_OK;
   };
   int j = 1;
@@ -1024,7 +1071,7 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
                                  (uint64_t)a.greedy, (uint64_t)(uint32_t)a.eos_id, a.seed,
                                  (uint64_t)c->use_tcgen05, (uint64_t)c->use_tc_attention, (uint64_t)c->use_pdl,
                                  (uint64_t)c->gemm_bn, (uint64_t)c->gemm_splits, (uint64_t)c->use_gemm_pairs, (uint64_t)c->use_cluster_merge, (uint64_t)c->use_gemm_pairs_small, (uint64_t)c->use_fused_layers,
-                                 (uint64_t)c->attn_dec5, (uint64_t)c->attn_suf_splits};
+                                 (uint64_t)c->attn_dec5, (uint64_t)c->attn_suf_splits, (uint64_t)wave};
     rpo_ctx::StepGraph* sg = nullptr;
     for (auto& g : c->step_graphs) if (g.key == key) sg = &g;
     if (!sg) {
@@ -1052,6 +1099,14 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
   }
   for (; j < S; ++j) RPO_TRY(enqueue_step());
   CUDA_TRY(cudaMemcpyAsync(d_lens_out, w.lens, (size_t)B * 4, cudaMemcpyDeviceToDevice, st));
+  if (wave) {
+    // feed the call's last token: its K/V joins the private blocks, and the logits its successor will be drawn from
+    // are parked in the sequence's state row together with the finished flag
+    RPO_TRY(enqueue_step(false));
+    LAUNCH(c, scatter_rows_u32_kernel, B, 256, 0, (const uint32_t*)w.logits, (const int32_t*)w.state_idx,
+           (uint32_t*)(w.logits + (size_t)w.HR * c->shape.vocab), B, c->shape.vocab);
+    LAUNCH(c, scatter_rows_u32_kernel, B, 32, 0, (const uint32_t*)w.done, (const int32_t*)w.state_idx, (uint32_t*)c->d_seq_done, B, 1);
+  }
   return RPO_OK;
 }
 
@@ -1073,6 +1128,47 @@ extern "C" int rpo_decode_suffix(rpo_ctx* c, int32_t n_groups, const rpo_group* 
                    : decode_t<float>(c, n_groups, h_groups, G, max_new, sp, d_forced, d_tokens_out, d_lens_out,
                                      d_logprobs_out, d_logits_dbg, priv);
   give_blocks(c, priv);   // stream order protects the blocks until the enqueued work is done
+  return rc;
+}
+
+extern "C" int rpo_decode_wave(rpo_ctx* c, int32_t n_groups, const rpo_group* h_groups, int32_t G, int32_t max_new,
+                               int32_t max_total, const rpo_sampler* sp, const int32_t* d_forced, int32_t* d_tokens_out,
+                               int32_t* d_lens_out, float* d_logprobs_out) {
+  if (!c || n_groups <= 0 || !h_groups || G <= 0 || max_new <= 0 || max_total < max_new || !d_tokens_out || !d_lens_out)
+    return RPO_ERR_INVALID_ARG;
+  RPO_TRY(check_sampler(sp));
+  if (!c->weights_ready) return RPO_ERR_NOT_INITIALISED;
+  RPO_TRY(enter(c));
+  RPO_TRY(check_groups(c, n_groups, h_groups));
+  if ((int64_t)n_groups * G > c->lim.max_seqs) return RPO_ERR_LIMIT;
+  // first pass: every group must be able to take the wave; nothing is reserved before all of them have been checked
+  int64_t need_blocks = 0, need_rows = 0;
+  for (int g = 0; g < n_groups; ++g) {
+    const GroupState& gs = c->groups[h_groups[g].slot];
+    if (gs.wave_G == 0) {
+      if (h_groups[g].prefix_len + max_total > c->lim.max_positions) return RPO_ERR_LIMIT;
+      need_blocks += (int64_t)G * ceil_div(max_total, KV_BLOCK);
+      need_rows += G;
+    } else if (gs.wave_G != G || gs.wave_t + max_new > gs.wave_total) {
+      return RPO_ERR_LIMIT;                      // another G than the group began with, or past the reserved positions
+    }
+  }
+  if (need_blocks > (int64_t)c->free_blocks.size() || need_rows > (int64_t)c->free_state_rows.size()) return RPO_ERR_KV_POOL;
+  for (int g = 0; g < n_groups; ++g) {
+    GroupState& gs = c->groups[h_groups[g].slot];
+    if (gs.wave_G != 0) continue;
+    RPO_TRY(take_blocks(c, G * ceil_div(max_total, KV_BLOCK), gs.wave_blocks));
+    for (int i = 0; i < G; ++i) { gs.wave_rows.push_back(c->free_state_rows.back()); c->free_state_rows.pop_back(); }
+    gs.wave_G = G; gs.wave_total = max_total; gs.wave_t = 0;
+  }
+  std::vector<int32_t> none;
+  c->prof_phase = 1;
+  const int rc = c->bf16 ? decode_t<bf16>(c, n_groups, h_groups, G, max_new, sp, d_forced, d_tokens_out, d_lens_out,
+                                          d_logprobs_out, nullptr, none, true)
+                         : decode_t<float>(c, n_groups, h_groups, G, max_new, sp, d_forced, d_tokens_out, d_lens_out,
+                                           d_logprobs_out, nullptr, none, true);
+  if (rc == RPO_OK)
+    for (int g = 0; g < n_groups; ++g) c->groups[h_groups[g].slot].wave_t += max_new;
   return rc;
 }
 
