@@ -315,6 +315,10 @@ int rpo_counters(rpo_ctx* ctx, int64_t* kernel_launches, int64_t* free_kv_blocks
  * "use_tc5_decode" (tcgen05 decode attention when a group's rows of one KV head fit a 64-row
  * tile; default 0: the mma.sync kernel measured faster), "use_fused_layers" (RMSNorm / RoPE / KV append / SwiGLU / residual add as GEMM
  * epilogues in passes whose products do not split K, default 1; 2 = also where they split),
+ * "use_fused_lse" (rpo_token_logprobs: the output head keeps, per row and tile, the running maximum,
+ * the sum of exponentials and the target's logit instead of writing the logits; default 1 = where the
+ * CTA-pair kernel serves the output head, 2 = always, 0 = never; calls that ask for d_logits_dbg always
+ * write the logits),
  * "wait_limit_cycles" (limit of every bounded device-side wait in SM cycles, for ALL contexts on the
  * device; <= 0 restores the default of 2e8, about 0.1 s),
  * "gemm_bn" (0 = planner, else force the tensor-core tile width: 32/64/96/128/256, or 512 / 384

@@ -62,6 +62,8 @@ struct Workspace {
   void* seqs = nullptr;    // SeqDesc[]
   int32_t *done = nullptr, *lens = nullptr, *cur_tok = nullptr, *logit_row = nullptr, *slot_idx = nullptr;
   int32_t *t_base = nullptr, *state_idx = nullptr;      // resumed decode: positions generated before the call; state row per sequence
+  void* lse_parts = nullptr;                            // float2 [HR][2 ceil(V / 256)]: the output head's per-unit (max, sum of exponentials)
+  float* lse_tgt = nullptr; int32_t* lse_target = nullptr;   // [HR]
   int32_t *done_idx = nullptr;                          // resumed decode: where the finished flags are read from (-1: fresh)
   int32_t* step_ctr = nullptr;   // device counter of the decode step being computed
   int64_t* seq_ids = nullptr;
@@ -108,6 +110,7 @@ struct rpo_ctx {
   int use_fused_layers = 1;           // 16-bit models: RMSNorm / RoPE / KV append / SwiGLU / residual as GEMM epilogues
   int use_tcgen05 = 1, use_tc_attention = 1, use_graph = 1;
   int use_tc5_attention = 1;          // tcgen05 attention for many-row passes
+  int use_fused_lse = 1;              // token log-probs: the output head keeps (max, sum exp, target) per tile instead of writing logits
   int use_tc5_decode = 0;             // tcgen05 decode attention (head_dim 128, <= 64 rows per group and KV head): parity-green, but
                                       // measured 5-25 % slower per launch than the mma.sync kernel (1.8 us per 64-key tile): off by default
   bool attn_dec5 = false;             // plan of the decode call being enqueued: prefix on tcgen05, suffix tiles in a pass of their own

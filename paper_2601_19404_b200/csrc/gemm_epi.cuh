@@ -27,9 +27,12 @@ enum TcEpilogue {
   TC_NSWIGLU = 6,      // rows scaled by 1/rms, SwiGLU on interleaved gate/up columns, bf16 store
   TC_QKV_ROPE = 7,     // rows scaled by 1/rms, RoPE on q and k heads, q -> qkv buffer, k / v -> paged pool
   TC_ADD_NORM = 8,     // x += C; xg = bf16(x * gain); partial sums of x^2 per (row, column tile)
+  TC_NLSE = 9,         // rows scaled by 1/rms and 1/T; nothing is stored but, per (row, column unit), the running
+                       // maximum and the sum of exponentials, and the logit of the row's target token (Eq. 7's
+                       // log pi(o_j | ...) without writing the logits out); pair kernel, no split-K
 };
 
-__host__ __device__ constexpr bool tc_epi_scaled(int epi) { return epi == TC_NSTORE_F32 || epi == TC_NSWIGLU || epi == TC_QKV_ROPE; }
+__host__ __device__ constexpr bool tc_epi_scaled(int epi) { return epi == TC_NSTORE_F32 || epi == TC_NSWIGLU || epi == TC_QKV_ROPE || epi == TC_NLSE; }
 __host__ __device__ constexpr bool tc_epi_fused(int epi) { return epi >= TC_NSTORE_F32; }
 
 struct TcParams {
@@ -53,6 +56,11 @@ struct TcParams {
   const float2* rope;   // TC_QKV_ROPE: [positions][head_dim / 2] (cos, sin)
   KVPool<bf16> pool;    // TC_QKV_ROPE
   int layer, hq, hkv, head_dim;
+  float2* lse_parts;    // TC_NLSE: [M][lse_stride] (max, sum of exp(z - max)) over the unit's columns, z = logit / T
+  int lse_stride;       //   column units per row (as ssq_out_parts)
+  float* lse_tgt;       // TC_NLSE: [M] z of the row's target token
+  const int32_t* lse_target;   // TC_NLSE: [M] target token id per row, negative = none
+  float lse_inv_T;
 };
 
 // Epilogue of one 32-column chunk of an accumulator row: r[0..31] are the float32 bit patterns of
@@ -142,6 +150,32 @@ __device__ __forceinline__ void epi_scaled_chunk(const TcParams& p, uint32_t* r,
   for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * scale);
   if (EPI == TC_NSTORE_F32) tc_store_chunk<TC_STORE_F32>(p, r, row, col, 0, STREAM);
   else tc_store_chunk<TC_SWIGLU>(p, r, row, col, 0, STREAM);
+}
+
+// TC_NLSE on one chunk: z = C * (1/rms) * (1/T); folds the chunk into the row's running (m, s) with
+// s = sum exp(z - m), and picks up the target's z when it lies in the chunk.
+__device__ __forceinline__ void epi_lse_chunk(const TcParams& p, const uint32_t* r, int col, float scale, int tgt,
+                                              float& m, float& s, float& zt) {
+  if (col >= p.N) return;
+  float z[32];
+  float cm = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    z[j] = (__uint_as_float(r[j]) * scale) * p.lse_inv_T;
+    if (col + j < p.N) cm = fmaxf(cm, z[j]);
+  }
+  const float mn = fmaxf(m, cm);
+  float acc = 0.f;
+#pragma unroll
+  for (int j = 0; j < 32; ++j)
+    if (col + j < p.N) acc += __expf(z[j] - mn);
+  s = s * __expf(m - mn) + acc;                 // m = -inf at the start: s = 0 * 0
+  m = mn;
+  if (tgt >= col && tgt < col + 32) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (tgt - col == j) zt = z[j];
+  }
 }
 
 // TC_QKV_ROPE on the chunk pair (lo, hi): columns col_lo .. +31 and col_lo + head_dim/2 .. +31 of one head.

@@ -419,7 +419,8 @@ inline bool tc_gemm_supported<bf16>(rpo_ctx* c, int M, int N, int K) {
 struct TcFuse {
   const float* ssq_in = nullptr; int ssq_in_parts = 0; int norm_dim = 0; float eps = 0.f;       // TC_N*
   float* ssq_out = nullptr; bf16* xg_out = nullptr; const float* gain = nullptr;                 // TC_ADD_NORM
-  int ssq_out_parts = 0;                                                                         //   (out) parts per row written
+  int ssq_out_parts = 0;                                                                         //   (out) parts per row written (TC_NLSE: units per row)
+  float2* lse_parts = nullptr; float* lse_tgt = nullptr; const int32_t* lse_target = nullptr; float lse_inv_T = 1.f;   // TC_NLSE
   const int4* row_meta = nullptr; const float2* rope = nullptr; KVPool<bf16> pool = {}; int layer = 0, hq = 0, hkv = 0, head_dim = 0;   // TC_QKV_ROPE
 };
 
@@ -439,6 +440,7 @@ inline void tc_fill_fuse(rpo_ctx* c, TcParams& p, const TcFuse* f) {
   p.ssq_in = f->ssq_in; p.ssq_in_parts = f->ssq_in_parts; p.inv_norm_dim = f->norm_dim > 0 ? 1.0f / (float)f->norm_dim : 0.f; p.eps = f->eps;
   p.ssq_out = f->ssq_out; p.xg_out = f->xg_out; p.gain = f->gain;
   p.row_meta = f->row_meta; p.rope = f->rope; p.pool = f->pool; p.layer = f->layer; p.hq = f->hq; p.hkv = f->hkv; p.head_dim = f->head_dim;
+  p.lse_parts = f->lse_parts; p.lse_tgt = f->lse_tgt; p.lse_target = f->lse_target; p.lse_inv_T = f->lse_inv_T;
 }
 
 template <int BN, int EPI>
@@ -468,6 +470,7 @@ inline int tc_launch_epi(rpo_ctx* c, int epi, const CUtensorMap* ma, const CUten
     case TC_NSTORE_F32: return tc_launch<BN, TC_NSTORE_F32>(c, ma, mw, p, grid);
     case TC_NSWIGLU: return tc_launch<BN, TC_NSWIGLU>(c, ma, mw, p, grid);
     case TC_ADD_NORM: return tc_launch<BN, TC_ADD_NORM>(c, ma, mw, p, grid);
+    case TC_NLSE: return RPO_ERR_INVALID_ARG;            // pair kernel only
     case TC_QKV_ROPE:
       if constexpr (BN % 64 == 0) return tc_launch<BN, TC_QKV_ROPE>(c, ma, mw, p, grid);
       else return RPO_ERR_INVALID_ARG;

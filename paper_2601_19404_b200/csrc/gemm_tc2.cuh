@@ -268,6 +268,19 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           ss += epi_add_norm_chunk(p, r, row, col_base + c0);
         }
         if (row < p.M) p.ssq_out[(int64_t)row * p.ssq_out_parts + part] = ss;
+      } else if (EPI == TC_NLSE) {
+        float m = -INFINITY, s = 0.f, zt = 0.f;
+        const int tgt = row < p.M ? p.lse_target[row] : -1;
+#pragma unroll 1
+        for (int c0 = 0; c0 < Cfg::ACC_COLS; c0 += 32) {
+          uint32_t r[32];
+          tc::tmem_ld32(t_row + (uint32_t)c0, r);
+          epi_lse_chunk(p, r, col_base + c0, scale, tgt, m, s, zt);
+        }
+        if (row < p.M) {
+          p.lse_parts[(int64_t)row * p.lse_stride + part] = make_float2(m, s);
+          if (tgt >= col_base && tgt < col_base + Cfg::ACC_COLS) p.lse_tgt[row] = zt;
+        }
       } else {
 #pragma unroll 1
         for (int c0 = 0; c0 < Cfg::ACC_COLS; c0 += 32) {
@@ -386,6 +399,7 @@ inline int tc2_gemm_launch(rpo_ctx* c, const bf16* A, const bf16* W, void* C, in
   p.tiles_m = (M + tm - 1) / tm; p.tiles_n = (N + 255) / 256; p.kb_total = K / TC_BK;
   int splits = (M <= 128 && c->gemm_bn == 0) ? 1 : tc2_splits(c, M, N, K, allow_split);
   if (tc_epi_fused(epi) && p.tiles_m * p.tiles_n * 8 > TC_CTR_CAPACITY) splits = 1;
+  if (epi == TC_NLSE) splits = 1;
   p.kb_per_split = (p.kb_total + splits - 1) / splits;
   splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
   if (splits > 1 && (size_t)splits * M * N > c->ws.partial_elems) { splits = 1; p.kb_per_split = p.kb_total; }
@@ -393,6 +407,7 @@ inline int tc2_gemm_launch(rpo_ctx* c, const bf16* A, const bf16* W, void* C, in
   p.split_stride = (int64_t)M * N; p.status = c->d_status;
   tc_fill_fuse(c, p, fuse);
   p.ssq_out_parts = rm == 128 ? p.tiles_n : 2 * p.tiles_n;
+  p.lse_stride = p.ssq_out_parts;
   if (fuse) fuse->ssq_out_parts = p.ssq_out_parts;
   if (splits > 1 && !tc_epi_fused(epi)) { epi = TC_PARTIAL; if (splits_out) *splits_out = splits; }
   const CUtensorMap* ma = tc_map(c, A, M, K, rm);
@@ -408,6 +423,7 @@ inline int tc2_gemm_launch(rpo_ctx* c, const bf16* A, const bf16* W, void* C, in
       case TC_NSWIGLU: return tc2_launch<TC_NSWIGLU, 64>(c, ma, mw, p);
       case TC_QKV_ROPE: return tc2_launch<TC_QKV_ROPE, 64>(c, ma, mw, p);
       case TC_ADD_NORM: return tc2_launch<TC_ADD_NORM, 64>(c, ma, mw, p);
+      case TC_NLSE: return tc2_launch<TC_NLSE, 64>(c, ma, mw, p);
       default: return tc2_launch<TC_PARTIAL, 64>(c, ma, mw, p);
     }
   }
@@ -420,6 +436,7 @@ inline int tc2_gemm_launch(rpo_ctx* c, const bf16* A, const bf16* W, void* C, in
     case TC_NSWIGLU: return tc2_launch<TC_NSWIGLU, 128>(c, ma, mw, p);
     case TC_QKV_ROPE: return tc2_launch<TC_QKV_ROPE, 128>(c, ma, mw, p);
     case TC_ADD_NORM: return tc2_launch<TC_ADD_NORM, 128>(c, ma, mw, p);
+    case TC_NLSE: return tc2_launch<TC_NLSE, 128>(c, ma, mw, p);
     default: return tc2_launch<TC_PARTIAL, 128>(c, ma, mw, p);
   }
 }

@@ -525,4 +525,39 @@ __global__ void logprob_rows_kernel(const float* __restrict__ logits, int row0, 
   }
 }
 
+// Target token of every head-row of a teacher-forced pass (row i of the launch = head row row0 + i =
+// (sequence, suffix position)); -1 beyond the sequence's length.
+__global__ void lse_targets_kernel(int row0, int n_rows, int V, int S, const int32_t* __restrict__ tokens,
+                                   const int32_t* __restrict__ lens, int seq0, int32_t* __restrict__ target) {
+  pdl_prologue();
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_rows) return;
+  const int hr = row0 + i, s = hr / S, j = hr % S;
+  const int64_t o = (int64_t)(seq0 + s) * S + j;
+  target[i] = (j < lens[seq0 + s]) ? min(max(tokens[o], 0), V - 1) : -1;
+}
+
+// log pi of the target per head-row from the output head's per-unit (max, sum of exponentials) and the
+// target's z: log pi = (z_t - M) - log sum_u s_u exp(m_u - M), M = max_u m_u.  A warp per row; rows
+// without a target get 0.
+__global__ void lse_merge_rows_kernel(const float2* __restrict__ parts, int n_parts, const float* __restrict__ zt,
+                                      const int32_t* __restrict__ target, int row0, int n_rows, int S, int seq0,
+                                      float* __restrict__ out) {
+  pdl_prologue();
+  const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (i >= n_rows) return;
+  const int hr = row0 + i, s = hr / S, j = hr % S;
+  const int64_t o = (int64_t)(seq0 + s) * S + j;
+  if (target[i] < 0) { if (lane == 0) out[o] = 0.f; return; }
+  const float2* p = parts + (int64_t)i * n_parts;
+  float m = -INFINITY;
+  for (int u = lane; u < n_parts; u += 32) m = fmaxf(m, p[u].x);
+#pragma unroll
+  for (int k = 16; k > 0; k >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, k));
+  float sum = 0.f;
+  for (int u = lane; u < n_parts; u += 32) { const float2 q = p[u]; sum += q.y * __expf(q.x - m); }
+  sum = warp_sum(sum);
+  if (lane == 0) out[o] = (zt[i] - m) - logf(sum);
+}
+
 }  // namespace rpo

@@ -305,6 +305,9 @@ extern "C" int rpo_create(rpo_ctx** out, const rpo_shape* shape, const rpo_limit
   ALLOC(w.t_base, (size_t)nseq * 4);
   ALLOC(w.state_idx, (size_t)nseq * 4);
   ALLOC(w.done_idx, (size_t)nseq * 4);
+  ALLOC(w.lse_parts, (size_t)w.HR * 2 * ceil_div(V, 256) * sizeof(float2));
+  ALLOC(w.lse_tgt, (size_t)w.HR * 4);
+  ALLOC(w.lse_target, (size_t)w.HR * 4);
   ALLOC(w.slot_idx, (size_t)nseq * 4);
   ALLOC(w.step_ctr, 16);
   ALLOC(w.seq_ids, (size_t)nseq * 8);
@@ -424,9 +427,10 @@ static int gemm_fused(rpo_ctx* c, const bf16* A, const bf16* W, void* C, int M, 
   if (M <= 0) return RPO_OK;
   ProfScope ps(c, KC_GEMM);
   static const char* labels[] = {"gemm", "gemm", "gemm", "gemm", "gemm", "gemm (1/rms, float32 store: output head)",
-                                 "gemm (1/rms, SwiGLU: gate/up)", "gemm (1/rms, RoPE, KV append: qkv)", "gemm (residual add, next norm: O / down)"};
+                                 "gemm (1/rms, SwiGLU: gate/up)", "gemm (1/rms, RoPE, KV append: qkv)", "gemm (residual add, next norm: O / down)",
+                                 "gemm (1/rms, 1/T, log-sum-exp parts: output head of the log-prob pass)"};
   prof_begin(c, labels[tc_epi]);
-  const int rc = tc2_wanted(c, M, N, K, true) ? tc2_gemm_launch(c, A, W, C, M, N, K, tc_epi, ldc, true, nullptr, &fuse)
+  const int rc = (tc_epi == TC_NLSE || tc2_wanted(c, M, N, K, true)) ? tc2_gemm_launch(c, A, W, C, M, N, K, tc_epi, ldc, true, nullptr, &fuse)
                                               : tc_gemm_launch(c, A, W, C, M, N, K, tc_epi, ldc, true, nullptr, &fuse);
   prof_end(c);
   c->launches++;
@@ -1224,6 +1228,24 @@ static int logprobs_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, 
         const int nr = std::min(w.HR, head_rows - r0);
         gather_head_rows_kernel<<<nr, 128, 0, st>>>(w.x, c->d_x_last, w.slot_idx, r0, nr, S, d, w.xh);
         c->launches++;
+        if (!d_logits_dbg && fused_layers(c, 1 << 20) && (c->use_fused_lse == 2 || (c->use_fused_lse && tc2_wanted(c, nr, V, d, false)))) {
+          // the output head keeps, per row and column unit, the running maximum, the sum of exponentials and the
+          // target's logit: the [nr, V] logits never reach memory
+          lse_targets_kernel<<<ceil_div(nr, 256), 256, 0, st>>>(r0, nr, V, S, d_tokens, d_lens, s0, w.lse_target);
+          c->launches++;
+          {
+            ProfScope ps(c, KC_NORM);
+            LAUNCH(c, norm_prep_kernel, nr, 128, 0, (const float*)w.xh, (const float*)c->gf, (bf16*)w.hh, w.ssq_h, nr, d);
+          }
+          TcFuse f;
+          f.ssq_in = w.ssq_h; f.ssq_in_parts = 1; f.norm_dim = d; f.eps = c->shape.rms_eps;
+          f.lse_parts = (float2*)w.lse_parts; f.lse_tgt = w.lse_tgt; f.lse_target = w.lse_target; f.lse_inv_T = inv_T;
+          if ((rc = gemm_fused(c, (const bf16*)w.hh, (const bf16*)c->lm_head, nullptr, nr, V, d, TC_NLSE, V, f)) != RPO_OK) break;
+          lse_merge_rows_kernel<<<ceil_div(nr, 8), 256, 0, st>>>((const float2*)w.lse_parts, f.ssq_out_parts, w.lse_tgt, w.lse_target,
+                                                                 r0, nr, S, s0, d_out);
+          c->launches++;
+          continue;
+        }
         if ((rc = head<T>(c, nr)) != RPO_OK) break;
         logprob_rows_kernel<<<nr, 512, 0, st>>>(w.logits, r0, nr, V, S, d_tokens, d_lens, s0, inv_T, d_out, d_logits_dbg);
         c->launches++;
@@ -1463,6 +1485,7 @@ extern "C" int rpo_set_option(rpo_ctx* c, const char* name, int32_t value) {
   }
   else if (!strcmp(name, "fused_split_limit")) c->fused_split_limit = value;
   else if (!strcmp(name, "use_tc5_attention")) c->use_tc5_attention = value;
+  else if (!strcmp(name, "use_fused_lse")) c->use_fused_lse = value;
   else if (!strcmp(name, "use_tc5_decode")) c->use_tc5_decode = value;
   else if (!strcmp(name, "use_gemm_pairs")) c->use_gemm_pairs = value;
   else if (!strcmp(name, "use_cluster_merge")) c->use_cluster_merge = value;

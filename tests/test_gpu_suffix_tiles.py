@@ -56,6 +56,16 @@ def _check_against_oracle(sh_d, w, lens, G, S, forced, eos, stops, fast=1, scale
         ctx.token_logprobs(groups, G, S, dev_i32(t), dev_i32(l), pol)
         torch.cuda.synchronize()
         pol = pol.cpu().numpy()
+        if fast >= 1:
+            # the same pass with the output head that keeps (max, sum of exponentials, target logit) per tile instead of
+            # writing the logits: forced here, since this vocabulary is too small for it to be chosen
+            ctx.set_option("use_fused_lse", 2)
+            pol2 = torch.zeros((n_g * G, S), dtype=torch.float32, device=DEV)
+            ctx.token_logprobs(groups, G, S, dev_i32(t), dev_i32(l), pol2)
+            torch.cuda.synchronize()
+            pol2 = pol2.cpu().numpy()
+            assert np.array_equal(pol2 == 0.0, pol == 0.0) and float(np.max(np.abs(pol2 - pol))) <= 2e-5
+            pol = pol2                                # the comparison with the oracle below runs on the fused result
         worst = [0.0, 0.0, 0.0]
         for g in range(n_g):
             sl = slice(g * G, (g + 1) * G)
