@@ -380,12 +380,20 @@ def run_config(args, name, steps, warmup, rank, local_rank, world, dist, headlin
         dgemm_ms, dgemm_n = prof["decode"]["gemm"]
         mgemm_ms = prof["prefill"]["gemm"][0] + prof["logprobs"]["gemm"][0]
         mgemm_n = prof["prefill"]["gemm"][1] + prof["logprobs"]["gemm"][1]
+        # DRAM bytes per launch of the two GEMM roles, from ncu captures of these very shapes (profiles/gemm_tc2_*_cfg4_reduced.txt,
+        # profiles/decode_small_kernels_cfg4_reduced.txt); only for the workload they were taken on, null elsewhere
+        traffic_many = traffic_decode = None
+        traffic_note = None
+        if name == "cfg4_7b_32x8" and shape["n_layers"] == 28 and not args.chunk:
+            traffic_many = (437.8e6 + 800.9e6 + 4292.8e6 + 3864.2e6) / 4            # QKV, O, gate/up, down of a 16384-row chunk
+            traffic_decode = (28 * (34.9e6 + 27.5e6 + 281.8e6 + 149.9e6) + 1242.3e6) / (28 * 4 + 1)   # a forward's 113 launches
+            traffic_note = "dram__bytes_read.sum + dram__bytes_write.sum per launch, mean over the launches of one layer (decode: one forward), ncu capture of the same shapes on the 2-layer cut"
         if dgemm_n:
             # weight-streaming GEMMs of the decode forwards: algorithmic bytes = every layer matrix + lm_head once per forward
             per_launch = ab["weights"] * (S - 1) / dgemm_n
             ach = per_launch / (dgemm_ms / dgemm_n * 1e-3) / 1e9
             roofline_decode = {"bound": "hbm", "kernel": "gemm_tc_kernel / gemm_tc2_kernel, decode forwards (weight streaming)",
-                               "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": None,
+                               "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": traffic_decode, "traffic_source": traffic_note,
                                "algorithmic_bytes_per_launch": per_launch, "launches": dgemm_n, "ms_per_launch": dgemm_ms / dgemm_n,
                                "share_of_step": dgemm_ms / (ms_per_step), "peak_source": peaks["source"] + ": copy bandwidth",
                                "tensor_tflops": 2.0 * B * (ab["weights"] / esz) * (S - 1) / (dgemm_ms * 1e-3) / 1e12}
@@ -395,7 +403,7 @@ def run_config(args, name, steps, warmup, rank, local_rank, world, dist, headlin
             ach = flops / (mgemm_ms * 1e-3) / 1e12
             roofline_many = {"bound": "tensor", "kernel": "gemm_tc2_kernel (CTA pairs), prefill and teacher-forced passes",
                              "achieved": ach, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_sustained"],
-                             "traffic": None, "algorithmic_flops_per_launch": flops / mgemm_n, "launches": mgemm_n,
+                             "traffic": traffic_many, "traffic_source": traffic_note, "algorithmic_flops_per_launch": flops / mgemm_n, "launches": mgemm_n,
                              "ms_per_launch": mgemm_ms / mgemm_n, "share_of_step": mgemm_ms / ms_per_step,
                              "frac_of_burst_peak": ach / peaks["bf16_tflops"],
                              "peak_source": peaks["source"] + ": sustained cuBLAS bf16 (the kernel runs inside a seconds-long step)"}
