@@ -315,6 +315,8 @@ int rpo_counters(rpo_ctx* ctx, int64_t* kernel_launches, int64_t* free_kv_blocks
  * "use_tc5_decode" (tcgen05 decode attention when a group's rows of one KV head fit a 64-row
  * tile; default 0: the mma.sync kernel measured faster), "use_fused_layers" (RMSNorm / RoPE / KV append / SwiGLU / residual add as GEMM
  * epilogues in passes whose products do not split K, default 1; 2 = also where they split),
+ * "use_tc5_pipelined" (the pipelined variant of the tcgen05 prefill attention: 64-key tiles, running output in
+ * tensor memory; default 0: measured 6-9 % slower),
  * "use_fused_lse" (rpo_token_logprobs: the output head keeps, per row and tile, the running maximum,
  * the sum of exponentials and the target's logit instead of writing the logits; default 1 = where the
  * CTA-pair kernel serves the output head, 2 = always, 0 = never; calls that ask for d_logits_dbg always

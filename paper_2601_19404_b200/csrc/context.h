@@ -110,6 +110,7 @@ struct rpo_ctx {
   int use_fused_layers = 1;           // 16-bit models: RMSNorm / RoPE / KV append / SwiGLU / residual as GEMM epilogues
   int use_tcgen05 = 1, use_tc_attention = 1, use_graph = 1;
   int use_tc5_attention = 1;          // tcgen05 attention for many-row passes
+  int use_tc5_pipelined = 0;          //   its pipelined variant (64-key tiles, running output in tensor memory)
   int use_fused_lse = 1;              // token log-probs: the output head keeps (max, sum exp, target) per tile instead of writing logits
   int use_tc5_decode = 0;             // tcgen05 decode attention (head_dim 128, <= 64 rows per group and KV head): parity-green, but
                                       // measured 5-25 % slower per launch than the mma.sync kernel (1.8 us per 64-key tile): off by default

@@ -14,6 +14,7 @@
 #include "attn_tc.cuh"
 #include "attn_tc5.cuh"
 #include "attn_dec5.cuh"
+#include "attn_pre5.cuh"
 #include "context.h"
 #include "gemm_tc.cuh"
 #include "gemm_tc2.cuh"
@@ -534,6 +535,13 @@ static int attention(rpo_ctx* c, int layer, int rows) {
         f.seqs = (const SeqDesc*)w.seqs; f.block_table = c->d_block_table; f.pool = kv_pool<bf16>(c); f.layer = layer;
         f.hq = s.n_q_heads; f.hkv = s.n_kv_heads; f.scale_log2 = scale * 1.4426950408889634f; f.tiles = (const int2*)w.tiles;
         f.q_col0 = 0; f.status = c->d_status;
+        if (c->use_tc5_pipelined) {                    // 64-key tiles, O accumulated in tensor memory
+          static bool p5_attr[64] = {};
+          if (tc_first_use_on_device(c, p5_attr))
+            CUDA_TRY(cudaFuncSetAttribute(flash_prefill_tc5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P5_SMEM));
+          LAUNCH(c, flash_prefill_tc5_kernel, dim3(s.n_q_heads, c->attn_tiles), 320, P5_SMEM, *qm, f);
+          return RPO_OK;
+        }
         static bool attr_done[64] = {};
         if (tc_first_use_on_device(c, attr_done))
           CUDA_TRY(cudaFuncSetAttribute(flash_attn_tc5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, T5_SMEM));
@@ -1486,6 +1494,7 @@ extern "C" int rpo_set_option(rpo_ctx* c, const char* name, int32_t value) {
   else if (!strcmp(name, "fused_split_limit")) c->fused_split_limit = value;
   else if (!strcmp(name, "use_tc5_attention")) c->use_tc5_attention = value;
   else if (!strcmp(name, "use_fused_lse")) c->use_fused_lse = value;
+  else if (!strcmp(name, "use_tc5_pipelined")) c->use_tc5_pipelined = value;
   else if (!strcmp(name, "use_tc5_decode")) c->use_tc5_decode = value;
   else if (!strcmp(name, "use_gemm_pairs")) c->use_gemm_pairs = value;
   else if (!strcmp(name, "use_cluster_merge")) c->use_cluster_merge = value;

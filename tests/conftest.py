@@ -23,7 +23,7 @@ def pytest_collection_modifyitems(config, items):
     if config.pluginmanager.hasplugin("timeout"):
         for it in items:
             if "gpu" in it.keywords and it.get_closest_marker("timeout") is None:
-                it.add_marker(pytest.mark.timeout(600, method="thread"))
+                it.add_marker(pytest.mark.timeout(int(os.environ.get("RPO_GPU_TEST_TIMEOUT", "600")), method="thread"))
     try:
         import torch
         has_gpu = torch.cuda.is_available()

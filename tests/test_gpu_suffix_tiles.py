@@ -38,6 +38,7 @@ def _check_against_oracle(sh_d, w, lens, G, S, forced, eos, stops, fast=1, scale
         ctx.set_option("use_tcgen05", min(fast, 1)); ctx.set_option("use_tc_attention", min(fast, 1))
         ctx.set_option("use_fused_layers", 2 if fast == 2 else 1)      # 2: fused GEMM epilogues forced
         ctx.set_option("use_tc5_decode", 1 if fast == 3 else 0)        # 3: the tcgen05 decode attention
+        ctx.set_option("use_tc5_pipelined", 1 if fast == 4 else 0)     # 4: the pipelined tcgen05 attention in prefill / log-prob passes
         ctx.init_weights(0, 0.02)
         if scale_qk is not None:                       # sharper attention: the same scaled q/k weights on both sides
             for l in range(sh.n_layers):
@@ -86,8 +87,8 @@ def _check_against_oracle(sh_d, w, lens, G, S, forced, eos, stops, fast=1, scale
         return worst
 
 
-@pytest.mark.parametrize("fast", [3, 2, 1, 0], ids=["tcgen05_decode_attention", "tensor_core_fused_epilogues", "tensor_core_kernels",
-                                                    "cuda_core_kernels"])
+@pytest.mark.parametrize("fast", [4, 3, 2, 1, 0], ids=["tcgen05_pipelined_prefill_attention", "tcgen05_decode_attention", "tensor_core_fused_epilogues",
+                                                       "tensor_core_kernels", "cuda_core_kernels"])
 def test_ragged_long_prefixes_and_multi_tile_suffixes_with_stops(fast):
     """Prefixes of 1100 / 37 / 650 tokens (several prefix splits for the long ones, none for the
     short one), G = 6, 230 suffix tokens = 4 key tiles per sequence; stops inside the first tile, on a
@@ -110,7 +111,7 @@ def test_full_path_shape_short_prompt_long_generation():
     G, S, eos = 8, 300, 7
     stops = {3: 290, 9: 70}
     forced = _forced_with_stops(len(lens) * G, S, sh.vocab, eos, stops, seed=32)
-    for fast in (3, 2, 1):
+    for fast in (4, 3, 2, 1):
         _check_against_oracle(SHAPE, w, lens, G, S, forced, eos, stops, fast=fast)
 
 
@@ -130,5 +131,5 @@ def test_sharp_attention_makes_single_keys_matter():
     stops = {2: 100}
     forced = _forced_with_stops(len(lens) * G, S, sh.vocab, eos, stops, seed=33)
     worst = {f: _check_against_oracle(SHAPE, w, lens, G, S, forced, eos, stops, fast=f, scale_qk=3.0, tol=(9e-2, 6e-2))
-             for f in (3, 2, 1, 0)}
-    assert all(worst[f][0] <= 1.5 * worst[0][0] + 5e-3 for f in (1, 2, 3)), worst
+             for f in (4, 3, 2, 1, 0)}
+    assert all(worst[f][0] <= 1.5 * worst[0][0] + 5e-3 for f in (1, 2, 3, 4)), worst
