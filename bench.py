@@ -338,6 +338,26 @@ def run_config(args, name, steps, warmup, rank, local_rank, world, dist, headlin
         ctx.close()
         return out
 
+    # ---- headline only: the decode forwards one at a time (rpo_decode_wave with one position per call, CUDA events
+    #      around each call): the per-step distribution behind the mean above, suffix length growing from 1 to S
+    step_stats = None
+    if not args.no_profile:
+        groups = ctx.prefill_prefix(d_toks, off, group_ids)
+        w_out = torch.zeros((B, 1), dtype=torch.int32, device=dev)
+        w_len = torch.zeros(B, dtype=torch.int32, device=dev)
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(S + 1)]
+        torch.cuda.synchronize()
+        evs[0].record(stream)
+        for j in range(S):
+            ctx.decode_wave(groups, G, 1, S, smp, w_out, w_len)
+            evs[j + 1].record(stream)
+        torch.cuda.synchronize()
+        ctx.release_groups(groups)
+        per = np.array([evs[j].elapsed_time(evs[j + 1]) for j in range(S)])
+        step_stats = {"p50": float(np.percentile(per, 50)), "p95": float(np.percentile(per, 95)), "min": float(per.min()),
+                      "max": float(per.max()), "n": int(S),
+                      "how": "one rpo_decode_wave call per suffix position (one forward + lm_head + sampler, launched eagerly, no graph)"}
+
     # ---- headline only: end to end through the host-buffer call (pinned host memory, copies timed)
     e2e = None
     if not args.no_e2e:
@@ -416,6 +436,7 @@ def run_config(args, name, steps, warmup, rank, local_rank, world, dist, headlin
             roofline, other = roofline_decode, roofline_many
         roofline_decode = other
     out.update({"e2e": e2e, "roofline": roofline, "roofline_second_kernel": roofline_decode, "kernel_classes": phases,
+                "decode_step_ms": step_stats,
                 "gpu_launches": int(launches), "clocks": clk, "device_status": ctx.device_status()})
     ctx.close()
     return out
@@ -476,7 +497,7 @@ def main():
                    "parallelism": f"groups sharded over {world} rank(s), no collective in the step"},
     }
     for k in ("phases_ms", "decode_hbm", "prefill_tensor", "logprobs_tensor", "roofline", "roofline_second_kernel", "kernel_classes",
-              "e2e", "gpu_launches", "clocks", "device_status"):
+              "decode_step_ms", "e2e", "gpu_launches", "clocks", "device_status"):
         if k in head:
             out[k] = head[k]
     # the other configurations, same kernels, their own (fewer) steps; one GPU only
