@@ -456,7 +456,7 @@ inline int tc_launch(rpo_ctx* c, const CUtensorMap* ma, const CUtensorMap* mw, c
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr; cfg.numAttrs = c->use_pdl ? 1 : 0;
+  cfg.attrs = attr; cfg.numAttrs = c->pdl_now() ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, EPI>, *ma, *mw, p) == cudaSuccess ? RPO_OK : RPO_ERR_CUDA;
 }
 

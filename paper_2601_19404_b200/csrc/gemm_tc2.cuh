@@ -346,7 +346,7 @@ inline int tc2_launch(rpo_ctx* c, const CUtensorMap* ma, const CUtensorMap* mw, 
   }
   const int clusters = std::min(p.tiles_m * p.tiles_n * p.splits, max_clusters);
   cfg.gridDim = dim3(2 * clusters);
-  cfg.numAttrs = c->use_pdl ? 2 : 1;
+  cfg.numAttrs = c->pdl_now() ? 2 : 1;
   return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI, RM>, *ma, *mw, p) == cudaSuccess ? RPO_OK : RPO_ERR_CUDA;
 }
 

@@ -65,13 +65,15 @@ static void prof_end(rpo_ctx* c) {
 // Every kernel of the library starts with pdl_prologue() (or places pdl_wait() itself), so it may be
 // launched with programmatic stream serialization: its CTAs are scheduled while the previous
 // kernel drains, which hides launch latency between the many short kernels of a decode step.
+// By default that attribute is set only while a decode step is being captured into its graph (rpo_ctx::pdl_now):
+// on eagerly launched kernels it was associated with rare hangs of 512-sequence rollouts.
 template <typename... KArgs, typename... Args>
 static cudaError_t launch_kernel(rpo_ctx* c, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
   cudaLaunchAttribute attr[2];
   int n_attr = 0;
-  if (c->use_pdl) {
+  if (c->pdl_now()) {
     attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
     ++n_attr;
@@ -1095,7 +1097,9 @@ static int decode_t(rpo_ctx* c, int n_groups, const rpo_group* groups, int G, in
       const int64_t l0 = c->launches;
       cudaGraph_t graph = nullptr;
       CUDA_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+      c->capturing = true;
       const int rc = enqueue_step();
+      c->capturing = false;
       const cudaError_t ce = cudaStreamEndCapture(st, &graph);
       const int64_t per_step = c->launches - l0;
       c->launches = l0;
