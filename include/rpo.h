@@ -307,9 +307,10 @@ int rpo_counters(rpo_ctx* ctx, int64_t* kernel_launches, int64_t* free_kv_blocks
 /* Runtime switches (tests/benchmarks): name = "use_tcgen05" (bf16 GEMMs on the tensor-core
  * kernel, default 1), "use_tc_attention" (tensor-core attention kernels, default 1),
  * "use_graph" (CUDA graph per decode step, default 1), "use_pdl" (programmatic dependent launch
- * between the library's kernels: 0 off, 1 = inside the captured decode-step graphs only (default), 2 = on
- * every launch -- not recommended: with 2, a rollout of 512 sequences stopped making progress about once
- * in thirty calls on B200 / driver 580, never with 0 or 1), "use_tc5_attention" (tcgen05 attention for
+ * between the library's kernels: 0 off, 1 = in prefill / log-prob passes and inside the captured decode-step
+ * graphs (default), 2 = also on the eagerly launched kernels of a decode call -- not recommended: with 2, a
+ * rollout of 512 sequences stopped making progress about once in thirty calls on B200 / driver 580, never
+ * with 0 or 1), "use_tc5_attention" (tcgen05 attention for
  * many-row passes at head_dim 128, default 1), "use_gemm_pairs" (256 x 256 GEMM tiles on CTA
  * pairs for passes of more than 128 rows, default 1), "use_cluster_merge" (decode attention:
  * the prefix splits of a work item form a thread-block cluster and merge through distributed

@@ -120,9 +120,10 @@ struct rpo_ctx {
                                       // (measured slower than partials + merge kernel at 8 splits: off by default)
   int launch_cluster_x = 0;           // cluster width of the next launch (0: none); cleared by the launch
   int use_pdl = 1;                    // programmatic dependent launch between the library's kernels: 0 off, 1 inside the
-                                      // captured decode-step graphs only, 2 on every launch
+                                      // captured decode-step graphs and in the many-row passes (prefill, log-probs), 2 on
+                                      // every launch (also the eagerly launched parts of a decode call)
   bool capturing = false;             // a decode-step graph is being captured
-  bool pdl_now() const { return use_pdl >= 2 || (use_pdl == 1 && capturing); }
+  bool pdl_now() const { return use_pdl == 2 || (use_pdl == 1 && (capturing || prof_phase != 1)); }
   int use_gemm_pairs = 1;             // 256 x 256 tiles on CTA pairs (cta_group::2) for many-row GEMMs
   int use_gemm_pairs_small = 1;       // pair tiles with 64 rows per CTA for wide matrices at up to 128 rows
   int gemm_bn = 0, gemm_splits = 0;   // > 0: override the GEMM planner (tests, sweeps); 384 / 512 = pair tiles with 64 / 128 rows per CTA

@@ -65,8 +65,9 @@ static void prof_end(rpo_ctx* c) {
 // Every kernel of the library starts with pdl_prologue() (or places pdl_wait() itself), so it may be
 // launched with programmatic stream serialization: its CTAs are scheduled while the previous
 // kernel drains, which hides launch latency between the many short kernels of a decode step.
-// By default that attribute is set only while a decode step is being captured into its graph (rpo_ctx::pdl_now):
-// on eagerly launched kernels it was associated with rare hangs of 512-sequence rollouts.
+// By default that attribute is set in the many-row passes and while a decode step is being captured into its graph
+// (rpo_ctx::pdl_now), not on the eagerly launched kernels of a decode call: there it was associated with rare hangs
+// of 512-sequence rollouts.
 template <typename... KArgs, typename... Args>
 static cudaError_t launch_kernel(rpo_ctx* c, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
   cudaLaunchConfig_t cfg = {};
