@@ -442,6 +442,41 @@ def run_config(args, name, steps, warmup, rank, local_rank, world, dist, headlin
     return out
 
 
+def cache_init_leg(local_rank):
+    """Cache initialisation (Section 3.1, Eq. 1) with continuous batching on the 1.5B-class decoder: 64 requests with
+    512-token prompts, 256 generated tokens each (random weights almost never draw the EOS id, so every response runs to
+    the limit), batches of 32, waves of 32 tokens.  Timed twice on the host clock around synchronised calls: waves that
+    run the decoder over prompt + generated tokens again (prefill + decode per wave), and waves on kept state
+    (rpo_decode_wave: one prefill per request)."""
+    import torch
+    import paper_2601_19404_b200 as rpo
+    from paper_2601_19404_b200 import binding, cache_init
+    shape = dict(workloads.SHAPES["qwen1.5b-class"])
+    n_req, prompt, max_len, wave, mb = 64, 512, 256, 32, 32
+    lens = np.full(n_req, prompt, dtype=np.int32)
+    toks, off = workloads.prefix_tokens(lens, shape["vocab"], seed=7)
+    prompts = [toks[off[k]:off[k + 1]] for k in range(n_req)]
+    blocks = mb * (-(-(prompt + max_len) // 16)) + mb * (-(-max_len // 16)) + 64
+    out = {"workload": f"{n_req} requests x {prompt}-token prompts, {max_len} generated tokens, batch {mb}, waves of {wave}, 1.5B-class"}
+    torch.cuda.set_device(local_rank)
+    with rpo.Context(binding.shape_from_dict(shape), blocks, max_groups=mb, max_seqs=mb, max_chunk_tokens=mb * (prompt + max_len),
+                     max_positions=prompt + max_len + 1) as ctx:
+        ctx.init_weights(seed=0, std=0.02)
+        smp = rpo.Sampler(1.0, 0.95, False, 2, 0)
+        for name in ("re_prefill", "resumable"):
+            for rep in range(2):                                   # the first pass warms up (graphs, tensor maps)
+                torch.cuda.synchronize(); t0 = time.perf_counter()
+                if name == "re_prefill":
+                    got, st = cache_init.schedule(prompts, cache_init.library_engine(ctx, smp), mb, wave, max_len, smp.eos_id)
+                else:
+                    got, st = cache_init.schedule_resumable(prompts, cache_init.LibrarySession(ctx, smp, max_len), mb, wave, max_len, smp.eos_id)
+                torch.cuda.synchronize(); dt = time.perf_counter() - t0
+            out[name] = {"tokens_per_s": st["useful_tokens"] / dt, "seconds": dt, "waves": st["waves"], "tokens": st["useful_tokens"]}
+        out["device_status"] = ctx.device_status()
+    out["resumable_over_re_prefill"] = out["resumable"]["tokens_per_s"] / out["re_prefill"]["tokens_per_s"]
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -516,6 +551,8 @@ def main():
             others["cfg5_partial_over_full"] = {"wall_time_ratio": part["ms_per_step"] / full["ms_per_step"],
                                                 "generated_token_ratio": part["suffix"] / full["suffix"]}
         out["other_configs"] = others
+        if rank == 0:
+            out["cache_init"] = cache_init_leg(local_rank)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(args.config, args.ref_prefix, args.ref_suffix, args.ref_layers)
     if rank == 0:
